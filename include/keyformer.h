@@ -1,0 +1,149 @@
+/*
+ * keyformer.h -- C ABI of the B200 (sm_100a) Keyformer score-and-evict library.
+ *
+ * The library keeps, per (layer, batch row, head), a KV cache of at most k
+ * entries together with each entry's original token position and accumulated
+ * Keyformer score f_theta, and implements the two phases of Algorithm 1 of the
+ * Keyformer paper:
+ *
+ *   prompt phase      kf_prefill_score_prune   (Algorithm 1 with m <- n; section 3.4)
+ *   generation phase  kf_decode_step           (Algorithm 1 with m <- k; section 3.4)
+ *
+ * Conventions
+ *   - Every pointer whose name starts with d_ is a DEVICE pointer, h_ a HOST pointer.
+ *   - All device buffers, the workspace included, are owned by the caller; the
+ *     context owns host metadata only and kf_destroy frees no device memory.
+ *   - Q/K/V tensors are IEEE binary16 ("fp16"), contiguous, row-major in the
+ *     shapes stated per call.  Scores are binary32.
+ *   - Work is enqueued on the CUDA stream passed as `stream` (a cudaStream_t cast
+ *     to void*; NULL = the default stream).  No call synchronises except
+ *     kf_poll_error and the *_host variants' final wait when asked to.
+ *   - Return value 0 = success, negative = one of the KF_E* codes; on an error
+ *     detected on the host nothing has been enqueued.
+ *   - There is no CPU fallback: without a CUDA device every compute call
+ *     returns KF_ECUDA.
+ */
+#ifndef KEYFORMER_B200_H
+#define KEYFORMER_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KF_OK        0
+#define KF_EINVAL   -1   /* bad argument or configuration                         */
+#define KF_ENOSPC   -2   /* workspace too small                                   */
+#define KF_ESTATE   -3   /* call out of order (decode before prefill, ...)        */
+#define KF_ECUDA    -4   /* a CUDA runtime call failed / no device                */
+#define KF_ETIMEOUT -5   /* a bounded device-side wait ran out (error word)       */
+#define KF_EBOUNDS  -6   /* a device-side bounds check failed (error word)        */
+
+/* Logit adjustment zeta of Eq. 4 (section 4.4.3 lists the alternatives). */
+#define KF_NOISE_GUMBEL 0   /* zeta = -ln(-ln u), standard Gumbel, Eq. 7 (the method) */
+#define KF_NOISE_NONE   1   /* zeta = 0 (accumulated-attention score, H2O-like)      */
+#define KF_NOISE_CONST  2   /* zeta = noise_const                                     */
+
+#define KF_BIAS_NONE  0
+#define KF_BIAS_ALIBI 1     /* x_ij += -slope_h * (i - j) on ORIGINAL token positions (section 4.4.2) */
+
+typedef struct kf_ctx kf_ctx;
+
+/* Inputs of Algorithm 1 (cache size k, recent window w, generation length T,
+ * tau_init, tau_end) plus the tensor geometry. */
+typedef struct kf_config {
+  int32_t n_layers;        /* L >= 1                                              */
+  int32_t batch;           /* B >= 1 (beams are batch rows)                       */
+  int32_t n_heads;         /* H >= 1                                              */
+  int32_t head_dim;        /* d in {64, 128, 256}                                 */
+  int32_t budget_k;        /* k >= 1 : KV cache entries kept per (layer, b, head) */
+  int32_t recent_w;        /* 0 <= w <= k : most recent tokens always kept        */
+  int32_t max_prompt_len;  /* largest n accepted by kf_prefill_score_prune        */
+  int32_t gen_len_T;       /* T >= 0 : delta_tau = (tau_end - tau_init) / T (Eq. 12); 0 = constant tau_init */
+  float   tau_init;        /* > 0, paper default 1                                */
+  float   tau_end;         /* > 0, paper default 2                                */
+  uint64_t noise_seed;     /* Philox key                                          */
+  int32_t noise_mode;      /* KF_NOISE_*                                          */
+  int32_t bias_mode;       /* KF_BIAS_*                                           */
+  const float* h_alibi_slopes; /* HOST [H], read during kf_create when bias_mode == KF_BIAS_ALIBI */
+  float   logit_scale;     /* 0 => 1/sqrt(d) (Eq. 1 / Eq. 4)                      */
+  float   noise_const;     /* c of KF_NOISE_CONST                                 */
+  int32_t decode_splits;   /* 0 = choose automatically; else CTAs per unit in the decode kernel */
+  int32_t decode_direct_loads; /* 0 = K/V tiles staged in shared memory by bulk async copies (default); 1 = plain 128-bit global loads */
+} kf_config;
+
+/* Bytes of device workspace kf_create needs for this configuration
+ * (KV cache, positions, scores, kernel scratch).  Returns 0 if the
+ * configuration is invalid. */
+size_t kf_workspace_bytes(const kf_config* cfg);
+
+/* Build a context over a caller-owned device workspace of at least
+ * kf_workspace_bytes(cfg) bytes, 256-byte aligned.  Clears the cache state
+ * (asynchronously, on `stream`).  *out receives the context. */
+int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, void* stream, kf_ctx** out);
+
+/* Prompt phase of Algorithm 1 (t = 0, temperature tau_init; section 3.4).
+ * For every (batch row, head) of `layer`: causal logits x_ij = scale * Q_i.K_j
+ * (+ bias), y_ij = (x_ij + zeta_ij) / tau_init, row-wise softmax (Eq. 11), sum
+ * over query rows into f_theta(j); keep the w most recent positions plus the
+ * top-(k-w) of the others by f_theta (ties: lower position), and store the
+ * kept K/V rows, positions and scores in ascending position order.  If
+ * n_prompt <= k everything is kept.
+ *   d_q, d_k, d_v : DEVICE fp16 [B][H][n_prompt][d], read only.
+ *   d_score_opt   : DEVICE fp32 [B][H][n_prompt] or NULL; receives f_theta
+ *                   before pruning.
+ * Must be called once per layer before that layer's first kf_decode_step. */
+int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
+                           const void* d_q, const void* d_k, const void* d_v,
+                           float* d_score_opt, void* stream);
+
+/* One generation step of Algorithm 1 (t = step >= 1; section 3.4) for every
+ * (batch row, head) of `layer`.  The new token (original position
+ * p = n_prompt + step - 1) joins the cached entries, so m = len + 1 logits:
+ *   out   = sum_j softmax(x)_j V_j                       (Eq. 1; no noise, temperature 1)
+ *   z_j   = softmax_j((x_j + zeta_j) / tau_step)          (Eq. 4, 11; tau of Eq. 12, clamped at T)
+ *   f_theta(j) += z_j                                     (the new token starts from 0)
+ *   if m > k: evict the entry with the smallest f_theta among those not in
+ *   the w most recent (ties: the higher position leaves); the new token's
+ *   row takes the freed slot.  Slot order is therefore arbitrary; the
+ *   position array identifies the entries.
+ *   d_q, d_knew, d_vnew : DEVICE fp16 [B][H][d].
+ *   d_out               : DEVICE fp16 [B][H][d].
+ *   d_score_opt         : DEVICE fp32 [B][H][k+1] or NULL; receives z for the
+ *                         slots [0, len) followed by the new token at index len.
+ * Steps of a layer must be issued in increasing order starting from 1. */
+int kf_decode_step(kf_ctx* ctx, int32_t layer, int32_t step,
+                   const void* d_q, const void* d_knew, const void* d_vnew,
+                   void* d_out, float* d_score_opt, void* stream);
+
+/* Same step with HOST buffers (pinned memory recommended): copies q, k_new,
+ * v_new to the device, runs the step and copies `out` back, all on `stream`.
+ * If `wait` is non-zero the call returns after the stream has drained. */
+int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
+                        const void* h_q, const void* h_knew, const void* h_vnew,
+                        void* h_out, int32_t wait, void* stream);
+
+/* Borrowed DEVICE pointers into the workspace for one layer:
+ *   K, V fp16 [B][H][k][d]; pos int32 [B][H][k] (original positions; -1 marks a slot left empty by the prompt phase);
+ *   acc fp32 [B][H][k] (f_theta); len int32 [B][H] (entries in use).  Any may be NULL. */
+int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V,
+                  const int32_t** d_pos, const float** d_acc, const int32_t** d_len);
+
+/* Waits for `stream`, then returns and clears the device error word:
+ * 0, KF_ETIMEOUT or KF_EBOUNDS. */
+int kf_poll_error(kf_ctx* ctx, void* stream);
+
+/* Number of kernel launches this context has enqueued so far. */
+int64_t kf_launch_count(const kf_ctx* ctx);
+
+/* Frees host metadata.  The workspace stays with the caller. */
+int kf_destroy(kf_ctx* ctx);
+
+const char* kf_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KEYFORMER_B200_H */

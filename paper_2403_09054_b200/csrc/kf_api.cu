@@ -1,0 +1,318 @@
+// C ABI of the library (see include/keyformer.h): configuration checks,
+// workspace carving, temperature schedule (Eq. 12) and kernel launches.
+#include "keyformer.h"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kf_decode.cuh"
+#include "kf_prefill.cuh"
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+struct Layout {
+  size_t K, V, acc, pos, len;          // per-layer strides are kv_layer / sc_layer / len_layer
+  size_t y_scratch, partials, counters, err, slopes;
+  size_t acc_full, idx, staging;
+  size_t total;
+  size_t kv_layer, sc_layer, len_layer; // bytes per layer
+  int units, max_splits;
+};
+
+bool config_ok(const kf_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->batch < 1 || c->n_heads < 1) return false;
+  if (c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256) return false;
+  if (c->budget_k < 1 || c->recent_w < 0 || c->recent_w > c->budget_k) return false;
+  if (c->max_prompt_len < 1 || c->gen_len_T < 0) return false;
+  if (!(c->tau_init > 0.f) || !(c->tau_end > 0.f)) return false;
+  if (c->noise_mode < KF_NOISE_GUMBEL || c->noise_mode > KF_NOISE_CONST) return false;
+  if (c->bias_mode != KF_BIAS_NONE && c->bias_mode != KF_BIAS_ALIBI) return false;
+  if (c->bias_mode == KF_BIAS_ALIBI && !c->h_alibi_slopes) return false;
+  if (c->logit_scale < 0.f || c->decode_splits < 0) return false;
+  if (c->decode_direct_loads != 0 && c->decode_direct_loads != 1) return false;
+  if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
+  return true;
+}
+
+int tiles_of(int k) { return (k + kf::decode_tile_rows() - 1) / kf::decode_tile_rows(); }
+
+Layout make_layout(const kf_config* c) {
+  Layout L{};
+  const size_t units = (size_t)c->batch * c->n_heads;
+  const size_t k = (size_t)c->budget_k, d = (size_t)c->head_dim, nl = (size_t)c->n_layers;
+  L.units = (int)units;
+  L.max_splits = std::max(1, std::min(64, (tiles_of(c->budget_k) + 3) / 4));
+  if (c->decode_splits > 0) L.max_splits = std::max(L.max_splits, (int)c->decode_splits);
+  L.kv_layer = align_up(units * k * d * 2);
+  L.sc_layer = align_up(units * k * 4);
+  L.len_layer = align_up(units * 4);
+  size_t off = 0;
+  L.K = off; off += nl * L.kv_layer;
+  L.V = off; off += nl * L.kv_layer;
+  L.acc = off; off += nl * L.sc_layer;
+  L.pos = off; off += nl * L.sc_layer;
+  L.len = off; off += nl * L.len_layer;
+  L.y_scratch = off; off += align_up(units * (k + 1) * 4);
+  L.partials = off; off += align_up(units * (size_t)L.max_splits * (4 + d) * 4);
+  L.counters = off; off += align_up(units * 4);
+  L.err = off; off += ALIGN;
+  L.slopes = off; off += align_up((size_t)c->n_heads * 4);
+  L.acc_full = off; off += align_up(units * (size_t)c->max_prompt_len * 4);
+  L.idx = off; off += align_up(units * k * 4);
+  L.staging = off; off += 4 * align_up(units * d * 2);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+struct kf_ctx {
+  kf_config cfg;
+  Layout lay;
+  unsigned char* ws;
+  kf::PhiloxKeys pk;
+  float scale;
+  std::vector<int32_t> n_prompt;   // per layer, -1 before prefill
+  std::vector<int32_t> last_step;  // per layer
+  int64_t launches;
+  bool staged;
+};
+
+extern "C" {
+
+size_t kf_workspace_bytes(const kf_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return make_layout(cfg).total;
+}
+
+int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, void* stream, kf_ctx** out) {
+  if (!out) return KF_EINVAL;
+  *out = nullptr;
+  if (!config_ok(cfg) || !d_workspace) return KF_EINVAL;
+  if (((uintptr_t)d_workspace) % ALIGN != 0) return KF_EINVAL;
+  const Layout lay = make_layout(cfg);
+  if (workspace_bytes < lay.total) return KF_ENOSPC;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return KF_ECUDA;
+  kf_ctx* ctx = new (std::nothrow) kf_ctx();
+  if (!ctx) return KF_EINVAL;
+  ctx->cfg = *cfg;
+  ctx->cfg.h_alibi_slopes = nullptr;  // copied below; the caller's array is not referenced later
+  ctx->lay = lay;
+  ctx->ws = static_cast<unsigned char*>(d_workspace);
+  ctx->pk = kf::philox_expand_key(cfg->noise_seed);
+  ctx->scale = cfg->logit_scale > 0.f ? cfg->logit_scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
+  ctx->n_prompt.assign(cfg->n_layers, -1);
+  ctx->last_step.assign(cfg->n_layers, 0);
+  ctx->launches = 0;
+  ctx->staged = cfg->decode_direct_loads == 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemsetAsync(ctx->ws + lay.acc, 0, lay.y_scratch - lay.acc, st);  // acc, pos, len
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + lay.counters, 0, lay.slopes - lay.counters, st);  // counters, err
+  if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI)
+    e = cudaMemcpyAsync(ctx->ws + lay.slopes, cfg->h_alibi_slopes, (size_t)cfg->n_heads * 4, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI) e = cudaStreamSynchronize(st);  // host array may go away
+  if (e != cudaSuccess) { delete ctx; return KF_ECUDA; }
+  *out = ctx;
+  return KF_OK;
+}
+
+int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
+                           const void* d_q, const void* d_k, const void* d_v,
+                           float* d_score_opt, void* stream) {
+  if (!ctx || !d_q || !d_k || !d_v) return KF_EINVAL;
+  const kf_config& c = ctx->cfg;
+  if (layer < 0 || layer >= c.n_layers) return KF_EINVAL;
+  if (n_prompt < 1 || n_prompt > c.max_prompt_len) return KF_EINVAL;
+  const Layout& L = ctx->lay;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* acc_full = d_score_opt ? d_score_opt : reinterpret_cast<float*>(ctx->ws + L.acc_full);
+  int* err = reinterpret_cast<int*>(ctx->ws + L.err);
+  if (cudaMemsetAsync(acc_full, 0, (size_t)L.units * n_prompt * 4, st) != cudaSuccess) return KF_ECUDA;
+
+  kf::PrefillParams P{};
+  P.Q = static_cast<const __half*>(d_q);
+  P.K = static_cast<const __half*>(d_k);
+  P.acc_full = acc_full;
+  P.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
+  P.err = err;
+  P.n = n_prompt; P.H = c.n_heads; P.layer = layer; P.noise_mode = c.noise_mode; P.bias_mode = c.bias_mode;
+  P.scale = ctx->scale;
+  P.inv_tau = (float)(1.0 / (double)c.tau_init);  // the prompt phase is iteration t = 0 of Eq. 12
+  P.noise_const = c.noise_const;
+  P.pk = ctx->pk;
+  if (kf::launch_prefill_score_simt(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+
+  kf::SelectParams S{};
+  S.acc_full = acc_full;
+  S.idx = reinterpret_cast<int32_t*>(ctx->ws + L.idx);
+  S.len = reinterpret_cast<int32_t*>(ctx->ws + L.len + (size_t)layer * L.len_layer);
+  S.err = err;
+  S.n = n_prompt; S.k = c.budget_k; S.w = c.recent_w;
+  if (kf::launch_prefill_select(S, L.units, st) != cudaSuccess) return KF_ECUDA;
+
+  kf::GatherParams G{};
+  G.K = static_cast<const __half*>(d_k);
+  G.V = static_cast<const __half*>(d_v);
+  G.acc_full = acc_full;
+  G.idx = S.idx;
+  G.Kc = reinterpret_cast<__half*>(ctx->ws + L.K + (size_t)layer * L.kv_layer);
+  G.Vc = reinterpret_cast<__half*>(ctx->ws + L.V + (size_t)layer * L.kv_layer);
+  G.pos = reinterpret_cast<int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer);
+  G.acc = reinterpret_cast<float*>(ctx->ws + L.acc + (size_t)layer * L.sc_layer);
+  G.n = n_prompt; G.k = c.budget_k;
+  if (kf::launch_prefill_gather(G, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+
+  ctx->launches += 3;
+  ctx->n_prompt[layer] = n_prompt;
+  ctx->last_step[layer] = 0;
+  return KF_OK;
+}
+
+static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q, const void* d_knew,
+                       const void* d_vnew, void* d_out, float* d_score_opt, cudaStream_t st) {
+  const kf_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  kf::DecodeParams P{};
+  P.K = reinterpret_cast<const __half*>(ctx->ws + L.K + (size_t)layer * L.kv_layer);
+  P.V = reinterpret_cast<const __half*>(ctx->ws + L.V + (size_t)layer * L.kv_layer);
+  P.acc = reinterpret_cast<float*>(ctx->ws + L.acc + (size_t)layer * L.sc_layer);
+  P.pos = reinterpret_cast<int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer);
+  P.len = reinterpret_cast<int32_t*>(ctx->ws + L.len + (size_t)layer * L.len_layer);
+  P.q = static_cast<const __half*>(d_q);
+  P.knew = static_cast<const __half*>(d_knew);
+  P.vnew = static_cast<const __half*>(d_vnew);
+  P.out = static_cast<__half*>(d_out);
+  P.score_opt = d_score_opt;
+  P.y_scratch = reinterpret_cast<float*>(ctx->ws + L.y_scratch);
+  P.partials = reinterpret_cast<float*>(ctx->ws + L.partials);
+  P.counters = reinterpret_cast<unsigned int*>(ctx->ws + L.counters);
+  P.err = reinterpret_cast<int*>(ctx->ws + L.err);
+  P.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
+  P.k = c.budget_k; P.w = c.recent_w;
+  P.p = ctx->n_prompt[layer] + step - 1;
+
+  // split the slots of a unit over CTAs so that the grid fills the 148 SMs several times over
+  const int tiles = tiles_of(c.budget_k);
+  int splits = c.decode_splits;
+  if (splits <= 0) {
+    const int target_ctas = 148 * 8;
+    splits = (target_ctas + L.units - 1) / L.units;
+  }
+  splits = std::max(1, std::min(splits, std::min(L.max_splits, (tiles + 3) / 4)));
+  int tps = (tiles + splits - 1) / splits;
+  tps = (tps + 3) / 4 * 4;  // whole rounds of the CTA's four warps
+  splits = (tiles + tps - 1) / tps;
+  P.splits = splits; P.tiles_per_split = tps;
+  P.H = c.n_heads; P.layer = layer; P.noise_mode = c.noise_mode; P.bias_mode = c.bias_mode;
+  P.scale = ctx->scale;
+  // Eq. 12 with t = step, clamped at T; T = 0 keeps tau_init
+  double tau = c.tau_init;
+  if (c.gen_len_T > 0) {
+    const int t = std::min(step, c.gen_len_T);
+    tau = (double)c.tau_init + (double)t * (((double)c.tau_end - (double)c.tau_init) / (double)c.gen_len_T);
+  }
+  P.inv_tau = (float)(1.0 / tau);
+  P.noise_const = c.noise_const;
+  P.pk = ctx->pk;
+  if (kf::launch_decode(P, c.head_dim, L.units, ctx->staged, st) != cudaSuccess) return KF_ECUDA;
+  ctx->launches += 1;
+  ctx->last_step[layer] = step;
+  return KF_OK;
+}
+
+static int decode_check(kf_ctx* ctx, int32_t layer, int32_t step) {
+  if (!ctx) return KF_EINVAL;
+  if (layer < 0 || layer >= ctx->cfg.n_layers || step < 1) return KF_EINVAL;
+  if (ctx->n_prompt[layer] < 0) return KF_ESTATE;
+  if (step != ctx->last_step[layer] + 1) return KF_ESTATE;
+  return KF_OK;
+}
+
+int kf_decode_step(kf_ctx* ctx, int32_t layer, int32_t step,
+                   const void* d_q, const void* d_knew, const void* d_vnew,
+                   void* d_out, float* d_score_opt, void* stream) {
+  const int rc = decode_check(ctx, layer, step);
+  if (rc != KF_OK) return rc;
+  if (!d_q || !d_knew || !d_vnew || !d_out) return KF_EINVAL;
+  return decode_impl(ctx, layer, step, d_q, d_knew, d_vnew, d_out, d_score_opt, static_cast<cudaStream_t>(stream));
+}
+
+int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
+                        const void* h_q, const void* h_knew, const void* h_vnew,
+                        void* h_out, int32_t wait, void* stream) {
+  const int rc = decode_check(ctx, layer, step);
+  if (rc != KF_OK) return rc;
+  if (!h_q || !h_knew || !h_vnew || !h_out) return KF_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Layout& L = ctx->lay;
+  const size_t bytes = (size_t)L.units * ctx->cfg.head_dim * 2;
+  const size_t stride = align_up(bytes);
+  unsigned char* sq = ctx->ws + L.staging;
+  unsigned char* sk = sq + stride;
+  unsigned char* sv = sk + stride;
+  unsigned char* so = sv + stride;
+  if (cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return KF_ECUDA;
+  if (cudaMemcpyAsync(sk, h_knew, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return KF_ECUDA;
+  if (cudaMemcpyAsync(sv, h_vnew, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return KF_ECUDA;
+  const int rc2 = decode_impl(ctx, layer, step, sq, sk, sv, so, nullptr, st);
+  if (rc2 != KF_OK) return rc2;
+  if (cudaMemcpyAsync(h_out, so, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KF_ECUDA;
+  if (wait && cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
+  return KF_OK;
+}
+
+int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V,
+                  const int32_t** d_pos, const float** d_acc, const int32_t** d_len) {
+  if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return KF_EINVAL;
+  const Layout& L = ctx->lay;
+  if (d_K) *d_K = ctx->ws + L.K + (size_t)layer * L.kv_layer;
+  if (d_V) *d_V = ctx->ws + L.V + (size_t)layer * L.kv_layer;
+  if (d_pos) *d_pos = reinterpret_cast<const int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer);
+  if (d_acc) *d_acc = reinterpret_cast<const float*>(ctx->ws + L.acc + (size_t)layer * L.sc_layer);
+  if (d_len) *d_len = reinterpret_cast<const int32_t*>(ctx->ws + L.len + (size_t)layer * L.len_layer);
+  return KF_OK;
+}
+
+int kf_poll_error(kf_ctx* ctx, void* stream) {
+  if (!ctx) return KF_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, ctx->ws + ctx->lay.err, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return KF_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
+  if (word != 0) {
+    if (cudaMemsetAsync(ctx->ws + ctx->lay.err, 0, sizeof(int), st) != cudaSuccess) return KF_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
+  }
+  return word;
+}
+
+int64_t kf_launch_count(const kf_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int kf_destroy(kf_ctx* ctx) {
+  if (!ctx) return KF_EINVAL;
+  delete ctx;
+  return KF_OK;
+}
+
+const char* kf_strerror(int code) {
+  switch (code) {
+    case KF_OK: return "ok";
+    case KF_EINVAL: return "invalid argument or configuration";
+    case KF_ENOSPC: return "workspace too small";
+    case KF_ESTATE: return "call out of order";
+    case KF_ECUDA: return "CUDA runtime error or no device";
+    case KF_ETIMEOUT: return "a bounded device-side wait ran out";
+    case KF_EBOUNDS: return "a device-side bounds check failed";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

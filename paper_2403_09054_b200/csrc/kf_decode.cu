@@ -1,0 +1,441 @@
+// Generation-phase kernel (Algorithm 1, t >= 1): one launch per layer call does
+//   logits -> attention output + Gumbel-softmax score -> accumulate -> evict -> replace.
+//
+// Grid = (splits, units); a unit is one (batch row, head).  Each CTA streams a
+// contiguous range of cache slots exactly once: every warp owns 32-row tiles,
+// fetched into a private shared-memory ring by 1-D bulk async copies
+// (cp.async.bulk + mbarrier, no multicast), computes the logits x_j = q.K_j
+// once and uses them twice -- for the value-weighted output (Eq. 1) and for
+// the score softmax of (x_j + zeta_j) / tau (Eq. 4, 11).  The CTA that
+// finishes a unit last (ticket counter, no waiting) merges the split partials,
+// normalises the scores, adds them into f_theta, picks the entry to evict and
+// writes the new token's row into the freed slot.
+#include "kf_decode.cuh"
+
+namespace kf {
+
+namespace {
+
+constexpr int TILE_ROWS = 32;
+
+__device__ __forceinline__ float dot8(const uint4& kv, const float (&qf)[8]) {
+  const __half2* h = reinterpret_cast<const __half2*>(&kv);
+  float s = 0.f;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float2 f = __half22float2(h[c]);
+    s = fmaf(f.x, qf[2 * c], s);
+    s = fmaf(f.y, qf[2 * c + 1], s);
+  }
+  return s;
+}
+
+__device__ __forceinline__ void axpy8(float (&o)[8], float a, const uint4& vv) {
+  const __half2* h = reinterpret_cast<const __half2*>(&vv);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float2 f = __half22float2(h[c]);
+    o[2 * c] = fmaf(a, f.x, o[2 * c]);
+    o[2 * c + 1] = fmaf(a, f.y, o[2 * c + 1]);
+  }
+}
+
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ uint4 ld_shared_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)));
+  return v;
+}
+
+__device__ __forceinline__ float noise_for(const DecodeParams& P, uint32_t b, uint32_t lh, uint32_t i, uint32_t j) {
+  if (P.noise_mode == 0) return gumbel_from_word(noise_word(P.pk, b, lh, i, j));
+  if (P.noise_mode == 2) return P.noise_const;
+  return 0.f;
+}
+
+__device__ __forceinline__ unsigned long long evict_key(float a, int pos) {
+  // smallest key = smallest accumulated score; equal scores: the higher position leaves
+  return ((unsigned long long)__float_as_uint(a) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)pos);
+}
+
+// Work of the CTA that closes a unit: merge splits, normalise, accumulate, evict, replace.
+template <int D, int NT>
+__device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
+  __shared__ float sh_scalar[8];
+  __shared__ unsigned long long sh_key[NT / 32];
+  __shared__ int sh_victim;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = P.H;
+  const uint32_t b = (uint32_t)(u / H), h = (uint32_t)(u % H), lh = (uint32_t)P.layer * H + h;
+  const __half* q = P.q + (size_t)u * D;
+  const __half* kn = P.knew + (size_t)u * D;
+  const __half* vn = P.vnew + (size_t)u * D;
+  constexpr int PSTRIDE = 4 + D;
+  const float* part = P.partials + (size_t)u * P.splits * PSTRIDE;
+
+  if (warp == 0) {
+    float s = 0.f;
+    for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[c]), __half2float(kn[c]), s);
+    s = warp_sum(s);
+    if (lane == 0) {
+      const float x_new = s * P.scale;  // bias(p, p) = 0
+      const float y_new = (x_new + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
+      float mx = x_new, my = y_new;
+      for (int sp = 0; sp < P.splits; ++sp) {
+        mx = fmaxf(mx, __ldcg(part + sp * PSTRIDE + 0));
+        my = fmaxf(my, __ldcg(part + sp * PSTRIDE + 2));
+      }
+      float lx = fast_exp2((x_new - mx) * LOG2E), ly = fast_exp2((y_new - my) * LOG2E);
+      for (int sp = 0; sp < P.splits; ++sp) {
+        const float m_s = __ldcg(part + sp * PSTRIDE + 0), l_s = __ldcg(part + sp * PSTRIDE + 1);
+        const float n_s = __ldcg(part + sp * PSTRIDE + 2), k_s = __ldcg(part + sp * PSTRIDE + 3);
+        if (l_s > 0.f) lx = fmaf(l_s, fast_exp2((m_s - mx) * LOG2E), lx);
+        if (k_s > 0.f) ly = fmaf(k_s, fast_exp2((n_s - my) * LOG2E), ly);
+      }
+      sh_scalar[0] = mx; sh_scalar[1] = 1.f / lx; sh_scalar[2] = my; sh_scalar[3] = 1.f / ly;
+      sh_scalar[4] = x_new; sh_scalar[5] = y_new;
+    }
+  }
+  __syncthreads();
+  const float mx = sh_scalar[0], inv_lx = sh_scalar[1], my = sh_scalar[2], inv_ly = sh_scalar[3];
+  const float x_new = sh_scalar[4], y_new = sh_scalar[5];
+
+  // attention output (Eq. 1): merged partial sums plus the new token's own value row
+  for (int c = tid; c < D; c += NT) {
+    float o = fast_exp2((x_new - mx) * LOG2E) * __half2float(vn[c]);
+    for (int sp = 0; sp < P.splits; ++sp) {
+      const float m_s = __ldcg(part + sp * PSTRIDE + 0), l_s = __ldcg(part + sp * PSTRIDE + 1);
+      if (l_s > 0.f) o = fmaf(__ldcg(part + sp * PSTRIDE + 4 + c), fast_exp2((m_s - mx) * LOG2E), o);
+    }
+    P.out[(size_t)u * D + c] = __float2half_rn(o * inv_lx);
+  }
+
+  // score (Eq. 11), accumulation and the eviction candidate
+  float* acc = P.acc + (size_t)u * P.k;
+  int32_t* pos = P.pos + (size_t)u * P.k;
+  const float* ys = P.y_scratch + (size_t)u * (P.k + 1);
+  float* sc = P.score_opt ? P.score_opt + (size_t)u * (P.k + 1) : nullptr;
+  unsigned long long best = ~0ull;
+  const int cutoff = P.p - P.w;  // entries with pos <= cutoff are outside the recent window
+  for (int j = tid; j < len; j += NT) {
+    const float z = fast_exp2((__ldcg(ys + j) - my) * LOG2E) * inv_ly;
+    const float a = acc[j] + z;
+    acc[j] = a;
+    if (sc) sc[j] = z;
+    const int pj = pos[j];
+    if (pj <= cutoff) {
+      const unsigned long long key = evict_key(a, pj);
+      best = key < best ? key : best;
+    }
+  }
+  const float z_new = fast_exp2((y_new - my) * LOG2E) * inv_ly;
+  if (sc && tid == 0) sc[len] = z_new;
+  const unsigned long long key_new = evict_key(z_new, P.p);
+
+  if (len < P.k) {  // cache not full yet: append
+    if (tid == 0) { pos[len] = P.p; acc[len] = z_new; P.len[u] = len + 1; }
+    __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + len) * D;
+    __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + len) * D;
+    for (int c = tid; c < D; c += NT) { Kr[c] = kn[c]; Vr[c] = vn[c]; }
+    return;
+  }
+
+  if (P.w == 0) best = key_new < best ? key_new : best;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+    best = other < best ? other : best;
+  }
+  if (lane == 0) sh_key[warp] = best;
+  if (tid == 0) sh_victim = -1;
+  __syncthreads();
+  best = sh_key[0];
+#pragma unroll
+  for (int wi = 1; wi < NT / 32; ++wi) best = sh_key[wi] < best ? sh_key[wi] : best;
+  if (best == ~0ull) {  // cannot happen for 0 <= w <= k; flag it instead of guessing
+    if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
+    return;
+  }
+  if (best == key_new && P.w == 0) return;  // the new token itself has the lowest score: it is not stored
+  const int victim_pos = (int)(0xFFFFFFFFu - (uint32_t)(best & 0xFFFFFFFFull));
+  for (int j = tid; j < len; j += NT)
+    if (pos[j] == victim_pos) sh_victim = j;
+  __syncthreads();
+  const int jv = sh_victim;
+  if (jv < 0) {
+    if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
+    return;
+  }
+  if (tid == 0) { pos[jv] = P.p; acc[jv] = z_new; }
+  __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + jv) * D;
+  __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + jv) * D;
+  for (int c = tid; c < D; c += NT) { Kr[c] = kn[c]; Vr[c] = vn[c]; }
+}
+
+template <int D, int NW, bool STAGED, int NSTAGE>
+__global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__ DecodeParams P) {
+  constexpr int LPR = D / 8;          // lanes that share one row (16 bytes each)
+  constexpr int NLD = LPR;            // 128-bit loads per lane and 32-row tile
+  constexpr int NT = NW * 32;
+  constexpr int TILE_BYTES = TILE_ROWS * D * 2;
+  constexpr int PSTRIDE = 4 + D;
+
+  extern __shared__ __align__(128) unsigned char dyn_smem[];
+  __shared__ float sh_m[NW], sh_l[NW], sh_my[NW], sh_ly[NW];
+  __shared__ float sh_o[NW][D];
+  __shared__ unsigned int sh_ticket;
+
+  const int s = blockIdx.x, u = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int sub = lane % LPR, grp = lane / LPR;
+  const int len = P.len[u];
+  const int row_begin = s * P.tiles_per_split * TILE_ROWS;
+  const int row_end = min(len, row_begin + P.tiles_per_split * TILE_ROWS);
+  const int n_tiles = row_end > row_begin ? (row_end - row_begin + TILE_ROWS - 1) / TILE_ROWS : 0;
+  const int my_tiles = n_tiles > warp ? (n_tiles - warp + NW - 1) / NW : 0;
+  const __half* Ku = P.K + (size_t)u * P.k * D;
+  const __half* Vu = P.V + (size_t)u * P.k * D;
+  const int32_t* pos_u = P.pos + (size_t)u * P.k;
+  const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
+  const float slope = (P.bias_mode == 1 && P.slopes) ? P.slopes[h] : 0.f;
+
+  float qf[8];
+  {
+    const uint4 qv = *reinterpret_cast<const uint4*>(P.q + (size_t)u * D + sub * 8);
+    const __half2* hq = reinterpret_cast<const __half2*>(&qv);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float2 f = __half22float2(hq[c]);
+      qf[2 * c] = f.x; qf[2 * c + 1] = f.y;
+    }
+  }
+
+  // warp-private ring of shared-memory slots filled by bulk async copies
+  unsigned char* ring = dyn_smem + (size_t)warp * NSTAGE * TILE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(dyn_smem + (size_t)NW * NSTAGE * TILE_BYTES) + warp * NSTAGE;
+  const int n_items = 2 * my_tiles;  // K tile, V tile, K tile, ...
+  bool failed = false;
+  auto item_rows = [&](int it) {
+    const int tb = row_begin + (warp + (it >> 1) * NW) * TILE_ROWS;
+    return min(TILE_ROWS, row_end - tb);
+  };
+  auto issue = [&](int it) {
+    if (lane == 0) {
+      const int tb = row_begin + (warp + (it >> 1) * NW) * TILE_ROWS;
+      const uint32_t bytes = (uint32_t)item_rows(it) * D * 2;
+      const __half* src = ((it & 1) ? Vu : Ku) + (size_t)tb * D;
+      uint64_t* bar = bars + (it % NSTAGE);
+      mbar_expect_tx(bar, bytes);
+      bulk_load(ring + (size_t)(it % NSTAGE) * TILE_BYTES, src, bytes, bar);
+    }
+  };
+  if constexpr (STAGED) {
+    if (lane == 0) {
+      for (int i = 0; i < NSTAGE; ++i) mbar_init(bars + i, 1);
+      mbar_fence_init();
+    }
+    __syncwarp();
+    for (int it = 0; it < NSTAGE && it < n_items; ++it) issue(it);
+  }
+
+  float m_x = -INFINITY, l_x = 0.f, m_y = -INFINITY, l_y = 0.f;
+  float o[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) o[c] = 0.f;
+
+  int consumed = 0;  // items whose slot has been released (STAGED)
+  for (int ti = 0; ti < my_tiles; ++ti) {
+    const int tile_base = row_begin + (warp + ti * NW) * TILE_ROWS;
+    const int rows = min(TILE_ROWS, row_end - tile_base);
+
+    // ---- logits: lane r ends up with x of row tile_base + r
+    float x_mine = 0.f;
+    if constexpr (STAGED) {
+      const int it = 2 * ti;
+      const bool ok = mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
+      if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+      const unsigned char* slot = ring + (size_t)(it % NSTAGE) * TILE_BYTES;
+#pragma unroll
+      for (int i = 0; i < NLD; ++i) {
+        const int r = grp * LPR + i;
+        float part = 0.f;
+        if (r < rows) part = dot8(ld_shared_v4(slot + (size_t)r * D * 2 + sub * 16), qf);
+#pragma unroll
+        for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+        if (sub == i) x_mine = part;
+      }
+      __syncwarp();
+      consumed = it + 1;
+      if (it + NSTAGE < n_items) issue(it + NSTAGE);
+    } else {
+      constexpr int CH = NLD < 8 ? NLD : 8;
+#pragma unroll
+      for (int i0 = 0; i0 < NLD; i0 += CH) {
+        uint4 kv[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          const int r = grp * LPR + i0 + i;
+          kv[i] = r < rows ? ld_nc_v4(Ku + (size_t)(tile_base + r) * D + sub * 8) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          float part = dot8(kv[i], qf);
+#pragma unroll
+          for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+          if (sub == i0 + i) x_mine = part;
+        }
+      }
+    }
+
+    // ---- per-row work: bias, noise, the two running softmaxes
+    const bool valid = lane < rows;
+    const int row = tile_base + lane;
+    float x = -INFINITY, y = -INFINITY;
+    if (valid) {
+      const int pj = pos_u[row];
+      x = fmaf(x_mine, P.scale, -slope * (float)(P.p - pj));
+      y = (x + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)pj)) * P.inv_tau;
+      P.y_scratch[(size_t)u * (P.k + 1) + row] = y;
+    }
+    const float mx_new = fmaxf(m_x, warp_max(x));
+    const float my_new = fmaxf(m_y, warp_max(y));
+    const float corr_x = fast_exp2((m_x - mx_new) * LOG2E);   // 0 on the first tile (m_x = -inf)
+    const float corr_y = fast_exp2((m_y - my_new) * LOG2E);
+    const float pr = valid ? fast_exp2((x - mx_new) * LOG2E) : 0.f;
+    const float ey = valid ? fast_exp2((y - my_new) * LOG2E) : 0.f;
+    l_x = fmaf(l_x, corr_x, warp_sum(pr));
+    l_y = fmaf(l_y, corr_y, warp_sum(ey));
+    m_x = mx_new; m_y = my_new;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) o[c] *= corr_x;
+
+    // ---- value accumulation
+    if constexpr (STAGED) {
+      const int it = 2 * ti + 1;
+      const bool ok = mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
+      if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+      const unsigned char* slot = ring + (size_t)(it % NSTAGE) * TILE_BYTES;
+#pragma unroll
+      for (int i = 0; i < NLD; ++i) {
+        const int r = grp * LPR + i;
+        const float a = __shfl_sync(0xffffffffu, pr, r);
+        if (r < rows) axpy8(o, a, ld_shared_v4(slot + (size_t)r * D * 2 + sub * 16));
+      }
+      __syncwarp();
+      consumed = it + 1;
+      if (it + NSTAGE < n_items) issue(it + NSTAGE);
+    } else {
+      constexpr int CH = NLD < 8 ? NLD : 8;
+#pragma unroll
+      for (int i0 = 0; i0 < NLD; i0 += CH) {
+        uint4 vv[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          const int r = grp * LPR + i0 + i;
+          vv[i] = r < rows ? ld_nc_v4(Vu + (size_t)(tile_base + r) * D + sub * 8) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          const float a = __shfl_sync(0xffffffffu, pr, grp * LPR + i0 + i);
+          axpy8(o, a, vv[i]);
+        }
+      }
+    }
+  }
+
+  if constexpr (STAGED) {
+    if (failed) {
+      // a copy did not land in time: flag it, then give every copy still in flight a second bounded wait
+      if (lane == 0) atomicExch(P.err, ERR_TIMEOUT);
+      const int issued = min(n_items, consumed + NSTAGE);
+      for (int it = consumed; it < issued; ++it)
+        (void)mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
+    }
+  }
+
+  // ---- merge the warps of this CTA
+#pragma unroll
+  for (int off = LPR; off < 32; off <<= 1) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) o[c] += __shfl_xor_sync(0xffffffffu, o[c], off);
+  }
+  if (grp == 0) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) sh_o[warp][sub * 8 + c] = o[c];
+  }
+  if (lane == 0) { sh_m[warp] = m_x; sh_l[warp] = l_x; sh_my[warp] = m_y; sh_ly[warp] = l_y; }
+  __syncthreads();
+  float* part = P.partials + ((size_t)u * P.splits + s) * PSTRIDE;
+  {
+    float M = -INFINITY, MY = -INFINITY;
+#pragma unroll
+    for (int wi = 0; wi < NW; ++wi) { M = fmaxf(M, sh_m[wi]); MY = fmaxf(MY, sh_my[wi]); }
+    float sc[NW];
+#pragma unroll
+    for (int wi = 0; wi < NW; ++wi) sc[wi] = sh_l[wi] > 0.f ? fast_exp2((sh_m[wi] - M) * LOG2E) : 0.f;
+    for (int c = tid; c < D; c += NT) {
+      float acc_o = 0.f;
+#pragma unroll
+      for (int wi = 0; wi < NW; ++wi) acc_o = fmaf(sh_o[wi][c], sc[wi], acc_o);
+      part[4 + c] = acc_o;
+    }
+    if (tid == 0) {
+      float L = 0.f, LY = 0.f;
+#pragma unroll
+      for (int wi = 0; wi < NW; ++wi) {
+        L = fmaf(sh_l[wi], sc[wi], L);
+        if (sh_ly[wi] > 0.f) LY = fmaf(sh_ly[wi], fast_exp2((sh_my[wi] - MY) * LOG2E), LY);
+      }
+      part[0] = M; part[1] = L; part[2] = MY; part[3] = LY;
+    }
+  }
+
+  // ---- the CTA that arrives last closes the unit (no CTA ever waits for another)
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) sh_ticket = atomicAdd(P.counters + u, 1u);
+  __syncthreads();
+  if (sh_ticket != (unsigned)(P.splits - 1)) return;
+  __threadfence();
+  if (tid == 0) P.counters[u] = 0u;  // ready for the next launch
+  combine_and_evict<D, NT>(P, u, len);
+}
+
+template <int D, int NW, bool STAGED, int NSTAGE>
+cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
+  constexpr size_t smem = STAGED ? (size_t)NW * NSTAGE * (TILE_ROWS * D * 2) + (size_t)NW * NSTAGE * 8 : 0;
+  auto kern = decode_kernel<D, NW, STAGED, NSTAGE>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid((unsigned)P.splits, (unsigned)units);
+  kern<<<grid, NW * 32, smem, stream>>>(P);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int decode_tile_rows() { return TILE_ROWS; }
+
+cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, bool staged, cudaStream_t stream) {
+  switch (head_dim) {
+    case 64:
+      return staged ? launch_one<64, 4, true, 4>(P, units, stream) : launch_one<64, 4, false, 1>(P, units, stream);
+    case 128:
+      return staged ? launch_one<128, 4, true, 3>(P, units, stream) : launch_one<128, 4, false, 1>(P, units, stream);
+    case 256:
+      return staged ? launch_one<256, 4, true, 2>(P, units, stream) : launch_one<256, 4, false, 1>(P, units, stream);
+    default:
+      return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace kf

@@ -1,0 +1,34 @@
+// Launch interface of the generation-phase kernel (see kf_decode.cu).
+#pragma once
+
+#include "kf_common.cuh"
+
+namespace kf {
+
+struct DecodeParams {
+  const __half* K;        // [units][k][d] cache of this layer
+  const __half* V;
+  float* acc;             // [units][k]  accumulated score f_theta
+  int32_t* pos;           // [units][k]  original token positions
+  int32_t* len;           // [units]     entries in use
+  const __half* q;        // [units][d]
+  const __half* knew;     // [units][d]
+  const __half* vnew;     // [units][d]
+  __half* out;            // [units][d]
+  float* score_opt;       // [units][k+1] or null
+  float* y_scratch;       // [units][k+1] adjusted logits (x + zeta) / tau
+  float* partials;        // [units][splits][4 + d]
+  unsigned int* counters; // [units] arrival tickets, zero between launches
+  int* err;               // device error word
+  const float* slopes;    // [H] ALiBi slopes or null
+  int32_t k, w, p;        // budget, recent window, position of the query token
+  int32_t splits, tiles_per_split;
+  int32_t H, layer, noise_mode, bias_mode;
+  float scale, inv_tau, noise_const;
+  PhiloxKeys pk;
+};
+
+int decode_tile_rows();
+cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, bool staged, cudaStream_t stream);
+
+}  // namespace kf

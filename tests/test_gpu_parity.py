@@ -1,0 +1,119 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2403_09054_b200 as kf
+import workloads as W
+from tests import lockstep
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _wl(**kw):
+    base = dict(name="t", n_layers=1, batch=2, n_heads=3, head_dim=64, prompt_len=100, budget_k=40, recent_w=10,
+                gen_len_T=12, data_seed=11, noise_seed=5)
+    base.update(kw)
+    return W.Workload(**base)
+
+
+@pytest.mark.parametrize("d", [64, 128, 256])
+@pytest.mark.parametrize("direct", [0, 1])
+def test_small_odd_shapes(d, direct):
+    wl = _wl(head_dim=d, prompt_len=157, budget_k=71, recent_w=13)
+    r = lockstep.run_workload(wl, gpu_kwargs=dict(decode_direct_loads=direct))
+    assert r["max_out_err"] < 2e-3
+
+
+@pytest.mark.parametrize("k,w,n", [(33, 0, 90), (32, 32, 90), (64, 1, 65), (40, 10, 30), (40, 10, 40), (1, 0, 5), (1, 1, 5)])
+def test_edge_budgets(k, w, n):
+    wl = _wl(prompt_len=n, budget_k=k, recent_w=w, gen_len_T=14)
+    lockstep.run_workload(wl)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 5])
+def test_split_counts(splits):
+    wl = _wl(head_dim=128, prompt_len=700, budget_k=517, recent_w=100, gen_len_T=6)
+    lockstep.run_workload(wl, gpu_kwargs=dict(decode_splits=splits))
+
+
+@pytest.mark.parametrize("noise", ["none", "const"])
+def test_other_adjustments(noise):
+    lockstep.run_workload(_wl(head_dim=128), noise=noise)
+
+
+def test_zero_noise_tau_one_scores_are_attention_weights():
+    wl = _wl(head_dim=128, tau_init=1.0, tau_end=1.0, gen_len_T=3)
+    gpu = lockstep.make_gpu(wl, noise_mode=kf.KF_NOISE_NONE)
+    q, k, v = W.make_prompt(wl, 0, DEV)
+    gpu.kf_prefill_score_prune(0, q, k, v)
+    K, V, pos, acc, ln = gpu.kf_view_state(0)
+    Kb, Vb = K.clone().float(), V.clone().float()
+    qs, kn, vn = W.make_step(wl, 0, 1, DEV)
+    out = torch.empty_like(qs)
+    score = torch.zeros(wl.batch, wl.n_heads, wl.budget_k + 1, device=DEV)
+    gpu.kf_decode_step(0, 1, qs, kn, vn, out, score_out=score)
+    torch.cuda.synchronize()
+    assert torch.allclose(score.sum(-1), torch.ones_like(score.sum(-1)), atol=1e-5)
+    Vall = torch.cat([Vb, vn.float()[:, :, None, :]], dim=2)
+    rebuilt = torch.einsum("bhm,bhmd->bhd", score, Vall)
+    assert (rebuilt - out.float()).abs().max() < 2e-3 * out.float().abs().max()
+
+
+def test_alibi_and_rotary_workloads_scaled_down():
+    lockstep.run_workload(W.get_config("c3_mpt").scaled(n_heads=4, prompt_len=600, budget_k=300, recent_w=75, gen_len_T=10))
+    lockstep.run_workload(W.get_config("c2_gptj").scaled(n_heads=2, prompt_len=300, budget_k=150, recent_w=37, gen_len_T=10))
+
+
+def test_heavy_hitter_multi_layer_scaled_down():
+    wl = W.get_config("c4_cerebras").scaled(n_layers=3, batch=2, n_heads=4, prompt_len=400, budget_k=200, recent_w=50, gen_len_T=8)
+    lockstep.run_workload(wl)
+
+
+def test_config1_full():
+    wl = W.get_config("c1_tiny")
+    r = lockstep.run_workload(wl)
+    print("c1", r)
+
+
+def test_call_order_and_argument_errors():
+    wl = _wl()
+    gpu = lockstep.make_gpu(wl)
+    q, kn, vn = W.make_step(wl, 0, 1, DEV)
+    out = torch.empty_like(q)
+    with pytest.raises(kf.KeyformerError) as e:
+        gpu.kf_decode_step(0, 1, q, kn, vn, out)
+    assert e.value.code == kf.KF_ESTATE
+    Q, K, V = W.make_prompt(wl, 0, DEV)
+    gpu.kf_prefill_score_prune(0, Q, K, V)
+    with pytest.raises(kf.KeyformerError) as e:
+        gpu.kf_decode_step(0, 2, q, kn, vn, out)
+    assert e.value.code == kf.KF_ESTATE
+    with pytest.raises(kf.KeyformerError) as e:
+        gpu.kf_decode_step(5, 1, q, kn, vn, out)
+    assert e.value.code == kf.KF_EINVAL
+    gpu.kf_decode_step(0, 1, q, kn, vn, out)
+    assert gpu.kf_poll_error() == 0
+    assert gpu.kf_launch_count() == 4
+
+
+def test_host_buffer_variant_matches_device_variant():
+    wl = _wl(head_dim=128)
+    a, b = lockstep.make_gpu(wl), lockstep.make_gpu(wl)
+    Q, K, V = W.make_prompt(wl, 0, DEV)
+    a.kf_prefill_score_prune(0, Q, K, V)
+    b.kf_prefill_score_prune(0, Q, K, V)
+    for s in range(1, 4):
+        q, kn, vn = W.make_step(wl, 0, s, DEV)
+        out_a = torch.empty_like(q)
+        a.kf_decode_step(0, s, q, kn, vn, out_a)
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, kn, vn))
+        out_b = torch.empty_like(hq).pin_memory()
+        b.kf_decode_step_host(0, s, hq, hk, hv, out_b, wait=True)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a.cpu(), out_b)
+    sa, sb = a.kf_view_state(0), b.kf_view_state(0)
+    torch.cuda.synchronize()
+    for x, y in zip(sa, sb):
+        assert torch.equal(x, y)
