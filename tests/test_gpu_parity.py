@@ -115,5 +115,8 @@ def test_host_buffer_variant_matches_device_variant():
         assert torch.equal(out_a.cpu(), out_b)
     sa, sb = a.kf_view_state(0), b.kf_view_state(0)
     torch.cuda.synchronize()
-    for x, y in zip(sa, sb):
-        assert torch.equal(x, y)
+    for name, x, y in zip("K V pos acc len".split(), sa, sb):
+        if name == "acc":   # prompt scores are summed with floating-point atomics: order-dependent rounding
+            assert torch.allclose(x, y, rtol=1e-5, atol=1e-6)
+        else:
+            assert torch.equal(x, y)
