@@ -191,7 +191,7 @@ def run_ours(args, wl):
                        gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
                        bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
                        alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None,
-                       decode_splits=args.splits, decode_direct_loads=args.direct)
+                       decode_splits=args.splits)
     t_pre = time.perf_counter()
     for l in range(wl.n_layers):
         q, k, v = W.make_prompt(wl_r, l, dev)
@@ -274,7 +274,7 @@ def run_ours(args, wl):
             "config": {"workload": wl.name, "layers": L, "batch": B, "heads": H, "head_dim": d, "prompt": wl.prompt_len,
                        "budget_k": wl.budget_k, "recent_w": wl.recent_w, "tokens_per_s": value * B,
                        "l2": "inputs larger than L2 (KV state %.1f GB per GPU)" % (2 * L * B * H * wl.budget_k * d * 2 / 1e9),
-                       "prefill_s": t_pre, "decode_splits": args.splits, "direct_loads": args.direct},
+                       "prefill_s": t_pre, "decode_splits": args.splits},
             "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": abytes,
@@ -301,7 +301,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4_cerebras")
     ap.add_argument("--splits", type=int, default=0)
-    ap.add_argument("--direct", type=int, default=0)
     ap.add_argument("--cpu-units", type=int, default=512)
     ap.add_argument("--cpu-steps", type=int, default=64)
     ap.add_argument("--traffic", type=float, default=None,

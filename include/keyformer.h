@@ -71,7 +71,7 @@ typedef struct kf_config {
   float   logit_scale;     /* 0 => 1/sqrt(d) (Eq. 1 / Eq. 4)                      */
   float   noise_const;     /* c of KF_NOISE_CONST                                 */
   int32_t decode_splits;   /* 0 = choose automatically; else CTAs per unit in the decode kernel */
-  int32_t decode_direct_loads; /* 0 = K/V tiles staged in shared memory by bulk async copies (default); 1 = plain 128-bit global loads */
+  int32_t reserved;        /* must be 0                                           */
 } kf_config;
 
 /* Bytes of device workspace kf_create needs for this configuration

@@ -30,7 +30,7 @@ class kf_config(C.Structure):
         ("tau_init", C.c_float), ("tau_end", C.c_float), ("noise_seed", C.c_uint64),
         ("noise_mode", C.c_int32), ("bias_mode", C.c_int32), ("h_alibi_slopes", C.POINTER(C.c_float)),
         ("logit_scale", C.c_float), ("noise_const", C.c_float),
-        ("decode_splits", C.c_int32), ("decode_direct_loads", C.c_int32),
+        ("decode_splits", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -85,8 +85,7 @@ def kf_strerror(code: int) -> str:
 
 def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_prompt_len, gen_len_T,
                 tau_init=1.0, tau_end=2.0, noise_seed=0, noise_mode=KF_NOISE_GUMBEL, bias_mode=KF_BIAS_NONE,
-                alibi_slopes=None, logit_scale=0.0, noise_const=0.5772, decode_splits=0,
-                decode_direct_loads=0):
+                alibi_slopes=None, logit_scale=0.0, noise_const=0.5772, decode_splits=0):
     """Fill a kf_config; returns (config, keepalive) where keepalive holds the slopes array."""
     cfg = kf_config()
     cfg.n_layers, cfg.batch, cfg.n_heads, cfg.head_dim = n_layers, batch, n_heads, head_dim
@@ -99,7 +98,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
         keep = np.ascontiguousarray(alibi_slopes, dtype=np.float32)
         cfg.h_alibi_slopes = keep.ctypes.data_as(C.POINTER(C.c_float))
     cfg.logit_scale, cfg.noise_const = logit_scale, noise_const
-    cfg.decode_splits, cfg.decode_direct_loads = decode_splits, decode_direct_loads
+    cfg.decode_splits, cfg.reserved = decode_splits, 0
     return cfg, keep
 
 

@@ -36,7 +36,7 @@ bool config_ok(const kf_config* c) {
   if (c->bias_mode != KF_BIAS_NONE && c->bias_mode != KF_BIAS_ALIBI) return false;
   if (c->bias_mode == KF_BIAS_ALIBI && !c->h_alibi_slopes) return false;
   if (c->logit_scale < 0.f || c->decode_splits < 0) return false;
-  if (c->decode_direct_loads != 0 && c->decode_direct_loads != 1) return false;
+  if (c->reserved != 0) return false;
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
   return true;
 }
@@ -82,7 +82,6 @@ struct kf_ctx {
   std::vector<int32_t> n_prompt;   // per layer, -1 before prefill
   std::vector<int32_t> last_step;  // per layer
   int64_t launches;
-  bool staged;
 };
 
 extern "C" {
@@ -112,7 +111,6 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
   ctx->n_prompt.assign(cfg->n_layers, -1);
   ctx->last_step.assign(cfg->n_layers, 0);
   ctx->launches = 0;
-  ctx->staged = cfg->decode_direct_loads == 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(ctx->ws + lay.acc, 0, lay.y_scratch - lay.acc, st);  // acc, pos, len
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + lay.counters, 0, lay.slopes - lay.counters, st);  // counters, err
@@ -222,7 +220,7 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.inv_tau = (float)(1.0 / tau);
   P.noise_const = c.noise_const;
   P.pk = ctx->pk;
-  if (kf::launch_decode(P, c.head_dim, L.units, ctx->staged, st) != cudaSuccess) return KF_ECUDA;
+  if (kf::launch_decode(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
   ctx->launches += 1;
   ctx->last_step[layer] = step;
   return KF_OK;

@@ -18,18 +18,6 @@ namespace {
 
 constexpr int TILE_ROWS = 32;
 
-__device__ __forceinline__ float dot8(const uint4& kv, const float (&qf)[8]) {
-  const __half2* h = reinterpret_cast<const __half2*>(&kv);
-  float s = 0.f;
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    const float2 f = __half22float2(h[c]);
-    s = fmaf(f.x, qf[2 * c], s);
-    s = fmaf(f.y, qf[2 * c + 1], s);
-  }
-  return s;
-}
-
 __device__ __forceinline__ void axpy8(float (&o)[8], float a, const uint4& vv) {
   const __half2* h = reinterpret_cast<const __half2*>(&vv);
 #pragma unroll
@@ -38,20 +26,6 @@ __device__ __forceinline__ void axpy8(float (&o)[8], float a, const uint4& vv) {
     o[2 * c] = fmaf(a, f.x, o[2 * c]);
     o[2 * c + 1] = fmaf(a, f.y, o[2 * c + 1]);
   }
-}
-
-__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-
-__device__ __forceinline__ uint4 ld_shared_v4(const void* p) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)));
-  return v;
 }
 
 __device__ __forceinline__ float noise_for(const DecodeParams& P, uint32_t b, uint32_t lh, uint32_t i, uint32_t j) {
@@ -179,10 +153,34 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   for (int c = tid; c < D; c += NT) { Kr[c] = kn[c]; Vr[c] = vn[c]; }
 }
 
-template <int D, int NW, bool STAGED, int NSTAGE>
+// Warp-wide maximum in one instruction (f32 redux is an sm_100a feature).
+__device__ __forceinline__ float warp_max_redux(float v) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+  return r;
+}
+
+// acc += sum over the 8 binary16 pairs of a 16-byte chunk; products are exact in binary32 and
+// each fma rounds once (mixed-precision fma, an sm_100 instruction: no separate conversions).
+__device__ __forceinline__ void dot8_mixed(float& acc, const uint4& kv, const uint4& qv) {
+  const uint32_t kw[4] = {kv.x, kv.y, kv.z, kv.w};
+  const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    asm("{\n\t.reg .b16 kl, kh, ql, qh;\n\t"
+        "mov.b32 {kl, kh}, %1;\n\t"
+        "mov.b32 {ql, qh}, %2;\n\t"
+        "fma.rn.f32.f16 %0, kl, ql, %0;\n\t"
+        "fma.rn.f32.f16 %0, kh, qh, %0;\n\t}"
+        : "+f"(acc) : "r"(kw[c]), "r"(qw[c]));
+  }
+}
+
+template <int D, int NW, int NSTAGE>
 __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__ DecodeParams P) {
-  constexpr int LPR = D / 8;          // lanes that share one row (16 bytes each)
-  constexpr int NLD = LPR;            // 128-bit loads per lane and 32-row tile
+  constexpr int CPR = D / 8;          // 16-byte chunks per row
+  constexpr int LPR = CPR;            // lanes that share one row in the value phase
+  constexpr int NLD = LPR;            // 128-bit loads per lane and 32-row value tile
   constexpr int NT = NW * 32;
   constexpr int TILE_BYTES = TILE_ROWS * D * 2;
   constexpr int PSTRIDE = 4 + D;
@@ -190,6 +188,7 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   extern __shared__ __align__(128) unsigned char dyn_smem[];
   __shared__ float sh_m[NW], sh_l[NW], sh_my[NW], sh_ly[NW];
   __shared__ float sh_o[NW][D];
+  __shared__ __align__(16) __half sh_q[D];
   __shared__ unsigned int sh_ticket;
 
   const int s = blockIdx.x, u = blockIdx.y;
@@ -206,161 +205,138 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
   const float slope = (P.bias_mode == 1 && P.slopes) ? P.slopes[h] : 0.f;
 
-  float qf[8];
-  {
-    const uint4 qv = *reinterpret_cast<const uint4*>(P.q + (size_t)u * D + sub * 8);
-    const __half2* hq = reinterpret_cast<const __half2*>(&qv);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const float2 f = __half22float2(hq[c]);
-      qf[2 * c] = f.x; qf[2 * c + 1] = f.y;
-    }
-  }
-
   // warp-private ring of shared-memory slots filled by bulk async copies
   unsigned char* ring = dyn_smem + (size_t)warp * NSTAGE * TILE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(dyn_smem + (size_t)NW * NSTAGE * TILE_BYTES) + warp * NSTAGE;
   const int n_items = 2 * my_tiles;  // K tile, V tile, K tile, ...
   bool failed = false;
-  auto item_rows = [&](int it) {
-    const int tb = row_begin + (warp + (it >> 1) * NW) * TILE_ROWS;
-    return min(TILE_ROWS, row_end - tb);
-  };
+  auto tile_base_of = [&](int ti) { return row_begin + (warp + ti * NW) * TILE_ROWS; };
   auto issue = [&](int it) {
     if (lane == 0) {
-      const int tb = row_begin + (warp + (it >> 1) * NW) * TILE_ROWS;
-      const uint32_t bytes = (uint32_t)item_rows(it) * D * 2;
+      const int tb = tile_base_of(it >> 1);
+      const uint32_t bytes = (uint32_t)min(TILE_ROWS, row_end - tb) * D * 2;
       const __half* src = ((it & 1) ? Vu : Ku) + (size_t)tb * D;
       uint64_t* bar = bars + (it % NSTAGE);
       mbar_expect_tx(bar, bytes);
       bulk_load(ring + (size_t)(it % NSTAGE) * TILE_BYTES, src, bytes, bar);
     }
   };
-  if constexpr (STAGED) {
-    if (lane == 0) {
-      for (int i = 0; i < NSTAGE; ++i) mbar_init(bars + i, 1);
-      mbar_fence_init();
-    }
-    __syncwarp();
-    for (int it = 0; it < NSTAGE && it < n_items; ++it) issue(it);
+  if (lane == 0) {
+    for (int i = 0; i < NSTAGE; ++i) mbar_init(bars + i, 1);
+    mbar_fence_init();
   }
+  __syncwarp();
+  for (int it = 0; it < NSTAGE && it < n_items; ++it) issue(it);
 
-  float m_x = -INFINITY, l_x = 0.f, m_y = -INFINITY, l_y = 0.f;
+  if (tid < D / 8)
+    reinterpret_cast<uint4*>(sh_q)[tid] = reinterpret_cast<const uint4*>(P.q + (size_t)u * D)[tid];
+  __syncthreads();
+
+  float m_x = -INFINITY, l_x = 0.f, m_y = -INFINITY, l_y = 0.f;  // l_* are per-lane partial sums
   float o[8];
 #pragma unroll
   for (int c = 0; c < 8; ++c) o[c] = 0.f;
+  int pos_next = 0;
+  if (my_tiles > 0) {
+    const int tb = tile_base_of(0);
+    pos_next = (tb + lane < row_end) ? pos_u[tb + lane] : 0;
+  }
 
-  int consumed = 0;  // items whose slot has been released (STAGED)
+  int consumed = 0;  // ring items whose slot has been released
   for (int ti = 0; ti < my_tiles; ++ti) {
-    const int tile_base = row_begin + (warp + ti * NW) * TILE_ROWS;
+    const int tile_base = tile_base_of(ti);
     const int rows = min(TILE_ROWS, row_end - tile_base);
+    const int pj = pos_next;
+    if (ti + 1 < my_tiles) {
+      const int tb = tile_base_of(ti + 1);
+      pos_next = (tb + lane < row_end) ? pos_u[tb + lane] : 0;
+    }
 
-    // ---- logits: lane r ends up with x of row tile_base + r
-    float x_mine = 0.f;
-    if constexpr (STAGED) {
+    // ---- logits: lane r computes x of row tile_base + r.  Chunks are visited in a rotated
+    //      order ((c + lane) mod CPR) so that the 16-byte reads of a quarter warp hit distinct banks.
+    float x_mine;
+    {
       const int it = 2 * ti;
       const bool ok = mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
       if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-      const unsigned char* slot = ring + (size_t)(it % NSTAGE) * TILE_BYTES;
+      const unsigned char* krow = ring + (size_t)(it % NSTAGE) * TILE_BYTES + (size_t)lane * D * 2;
+      const unsigned char* qb = reinterpret_cast<const unsigned char*>(sh_q);
+      float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int i = 0; i < NLD; ++i) {
-        const int r = grp * LPR + i;
-        float part = 0.f;
-        if (r < rows) part = dot8(ld_shared_v4(slot + (size_t)r * D * 2 + sub * 16), qf);
+      for (int c0 = 0; c0 < CPR; c0 += 4) {
+        uint4 kv[4], qv[4];
 #pragma unroll
-        for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-        if (sub == i) x_mine = part;
+        for (int g = 0; g < 4; ++g) {
+          const int ch = (c0 + g + lane) & (CPR - 1);
+          kv[g] = *reinterpret_cast<const uint4*>(krow + ch * 16);
+          qv[g] = *reinterpret_cast<const uint4*>(qb + ch * 16);
+        }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) dot8_mixed(part[g], kv[g], qv[g]);
       }
+      x_mine = (part[0] + part[1]) + (part[2] + part[3]);
       __syncwarp();
       consumed = it + 1;
       if (it + NSTAGE < n_items) issue(it + NSTAGE);
-    } else {
-      constexpr int CH = NLD < 8 ? NLD : 8;
-#pragma unroll
-      for (int i0 = 0; i0 < NLD; i0 += CH) {
-        uint4 kv[CH];
-#pragma unroll
-        for (int i = 0; i < CH; ++i) {
-          const int r = grp * LPR + i0 + i;
-          kv[i] = r < rows ? ld_nc_v4(Ku + (size_t)(tile_base + r) * D + sub * 8) : make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int i = 0; i < CH; ++i) {
-          float part = dot8(kv[i], qf);
-#pragma unroll
-          for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-          if (sub == i0 + i) x_mine = part;
-        }
-      }
     }
 
-    // ---- per-row work: bias, noise, the two running softmaxes
+    // ---- per-row work: bias, noise, the two running softmaxes (warp-common maxima, per-lane sums)
     const bool valid = lane < rows;
-    const int row = tile_base + lane;
     float x = -INFINITY, y = -INFINITY;
     if (valid) {
-      const int pj = pos_u[row];
       x = fmaf(x_mine, P.scale, -slope * (float)(P.p - pj));
       y = (x + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)pj)) * P.inv_tau;
-      P.y_scratch[(size_t)u * (P.k + 1) + row] = y;
+      P.y_scratch[(size_t)u * (P.k + 1) + tile_base + lane] = y;
     }
-    const float mx_new = fmaxf(m_x, warp_max(x));
-    const float my_new = fmaxf(m_y, warp_max(y));
+    const float mx_new = fmaxf(m_x, warp_max_redux(x));
+    const float my_new = fmaxf(m_y, warp_max_redux(y));
     const float corr_x = fast_exp2((m_x - mx_new) * LOG2E);   // 0 on the first tile (m_x = -inf)
     const float corr_y = fast_exp2((m_y - my_new) * LOG2E);
     const float pr = valid ? fast_exp2((x - mx_new) * LOG2E) : 0.f;
     const float ey = valid ? fast_exp2((y - my_new) * LOG2E) : 0.f;
-    l_x = fmaf(l_x, corr_x, warp_sum(pr));
-    l_y = fmaf(l_y, corr_y, warp_sum(ey));
+    l_x = fmaf(l_x, corr_x, pr);
+    l_y = fmaf(l_y, corr_y, ey);
     m_x = mx_new; m_y = my_new;
 #pragma unroll
     for (int c = 0; c < 8; ++c) o[c] *= corr_x;
 
-    // ---- value accumulation
-    if constexpr (STAGED) {
+    // ---- value accumulation: LPR lanes share a row, each owns 8 columns
+    {
       const int it = 2 * ti + 1;
       const bool ok = mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
       if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-      const unsigned char* slot = ring + (size_t)(it % NSTAGE) * TILE_BYTES;
+      const unsigned char* slot = ring + (size_t)(it % NSTAGE) * TILE_BYTES + sub * 16;
+      constexpr int CH = NLD < 4 ? NLD : 4;
 #pragma unroll
-      for (int i = 0; i < NLD; ++i) {
-        const int r = grp * LPR + i;
-        const float a = __shfl_sync(0xffffffffu, pr, r);
-        if (r < rows) axpy8(o, a, ld_shared_v4(slot + (size_t)r * D * 2 + sub * 16));
+      for (int i0 = 0; i0 < NLD; i0 += CH) {
+        uint4 vv[CH];
+        float a[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          const int r = grp * LPR + i0 + i;
+          a[i] = __shfl_sync(0xffffffffu, pr, r);
+          vv[i] = r < rows ? *reinterpret_cast<const uint4*>(slot + (size_t)r * D * 2) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < CH; ++i) axpy8(o, a[i], vv[i]);
       }
       __syncwarp();
       consumed = it + 1;
       if (it + NSTAGE < n_items) issue(it + NSTAGE);
-    } else {
-      constexpr int CH = NLD < 8 ? NLD : 8;
-#pragma unroll
-      for (int i0 = 0; i0 < NLD; i0 += CH) {
-        uint4 vv[CH];
-#pragma unroll
-        for (int i = 0; i < CH; ++i) {
-          const int r = grp * LPR + i0 + i;
-          vv[i] = r < rows ? ld_nc_v4(Vu + (size_t)(tile_base + r) * D + sub * 8) : make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int i = 0; i < CH; ++i) {
-          const float a = __shfl_sync(0xffffffffu, pr, grp * LPR + i0 + i);
-          axpy8(o, a, vv[i]);
-        }
-      }
     }
   }
 
-  if constexpr (STAGED) {
-    if (failed) {
-      // a copy did not land in time: flag it, then give every copy still in flight a second bounded wait
-      if (lane == 0) atomicExch(P.err, ERR_TIMEOUT);
-      const int issued = min(n_items, consumed + NSTAGE);
-      for (int it = consumed; it < issued; ++it)
-        (void)mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
-    }
+  if (failed) {
+    // a copy did not land in time: flag it, then give every copy still in flight a second bounded wait
+    if (lane == 0) atomicExch(P.err, ERR_TIMEOUT);
+    const int issued = min(n_items, consumed + NSTAGE);
+    for (int it = consumed; it < issued; ++it)
+      (void)mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
   }
 
-  // ---- merge the warps of this CTA
+  // ---- merge the lanes, then the warps of this CTA
+  l_x = warp_sum(l_x);
+  l_y = warp_sum(l_y);
 #pragma unroll
   for (int off = LPR; off < 32; off <<= 1) {
 #pragma unroll
@@ -408,10 +384,10 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   combine_and_evict<D, NT>(P, u, len);
 }
 
-template <int D, int NW, bool STAGED, int NSTAGE>
+template <int D, int NW, int NSTAGE>
 cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
-  constexpr size_t smem = STAGED ? (size_t)NW * NSTAGE * (TILE_ROWS * D * 2) + (size_t)NW * NSTAGE * 8 : 0;
-  auto kern = decode_kernel<D, NW, STAGED, NSTAGE>;
+  constexpr size_t smem = (size_t)NW * NSTAGE * (TILE_ROWS * D * 2) + (size_t)NW * NSTAGE * 8;
+  auto kern = decode_kernel<D, NW, NSTAGE>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -425,16 +401,12 @@ cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
 
 int decode_tile_rows() { return TILE_ROWS; }
 
-cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, bool staged, cudaStream_t stream) {
+cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
   switch (head_dim) {
-    case 64:
-      return staged ? launch_one<64, 4, true, 4>(P, units, stream) : launch_one<64, 4, false, 1>(P, units, stream);
-    case 128:
-      return staged ? launch_one<128, 4, true, 3>(P, units, stream) : launch_one<128, 4, false, 1>(P, units, stream);
-    case 256:
-      return staged ? launch_one<256, 4, true, 2>(P, units, stream) : launch_one<256, 4, false, 1>(P, units, stream);
-    default:
-      return cudaErrorInvalidValue;
+    case 64: return launch_one<64, 4, 4>(P, units, stream);
+    case 128: return launch_one<128, 4, 3>(P, units, stream);
+    case 256: return launch_one<256, 4, 2>(P, units, stream);
+    default: return cudaErrorInvalidValue;
   }
 }
 

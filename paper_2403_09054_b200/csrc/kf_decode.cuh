@@ -29,6 +29,6 @@ struct DecodeParams {
 };
 
 int decode_tile_rows();
-cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, bool staged, cudaStream_t stream);
+cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 
 }  // namespace kf

@@ -41,8 +41,7 @@ def test_workspace_size_covers_the_cache():
 
 @pytest.mark.parametrize("bad", [dict(head_dim=96), dict(budget_k=0), dict(recent_w=65), dict(recent_w=-1),
                                  dict(tau_init=0.0), dict(tau_end=-1.0), dict(n_layers=0), dict(gen_len_T=-1),
-                                 dict(noise_mode=7), dict(bias_mode=1), dict(max_prompt_len=0),
-                                 dict(decode_direct_loads=2)])
+                                 dict(noise_mode=7), dict(bias_mode=1), dict(max_prompt_len=0)])
 def test_invalid_configurations_are_rejected(bad):
     assert kf.kf_workspace_bytes(_cfg(**bad)) == 0
 
