@@ -91,22 +91,40 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
     P.out[(size_t)u * D + c] = __float2half_rn(o * inv_lx);
   }
 
-  // score (Eq. 11), accumulation and the eviction candidate
-  float* acc = P.acc + (size_t)u * P.k;
-  int32_t* pos = P.pos + (size_t)u * P.k;
-  const float* ys = P.y_scratch + (size_t)u * (P.k + 1);
-  float* sc = P.score_opt ? P.score_opt + (size_t)u * (P.k + 1) : nullptr;
+  // score (Eq. 11), accumulation and the eviction candidate.  Loads are issued in batches so
+  // that a thread has several cache lines in flight instead of one round trip per entry.
+  float* __restrict__ acc = P.acc + (size_t)u * P.k;
+  int32_t* __restrict__ pos = P.pos + (size_t)u * P.k;
+  const float* __restrict__ ys = P.y_scratch + (size_t)u * (P.k + 1);
+  float* __restrict__ sc = P.score_opt ? P.score_opt + (size_t)u * (P.k + 1) : nullptr;
   unsigned long long best = ~0ull;
+  int best_j = -1;
   const int cutoff = P.p - P.w;  // entries with pos <= cutoff are outside the recent window
-  for (int j = tid; j < len; j += NT) {
-    const float z = fast_exp2((__ldcg(ys + j) - my) * LOG2E) * inv_ly;
-    const float a = acc[j] + z;
-    acc[j] = a;
-    if (sc) sc[j] = z;
-    const int pj = pos[j];
-    if (pj <= cutoff) {
-      const unsigned long long key = evict_key(a, pj);
-      best = key < best ? key : best;
+  constexpr int BATCH = 8;
+  for (int j0 = tid; j0 < len; j0 += NT * BATCH) {
+    float yv[BATCH], av[BATCH];
+    int pv[BATCH];
+#pragma unroll
+    for (int i = 0; i < BATCH; ++i) {
+      const int j = j0 + i * NT;
+      const bool in = j < len;
+      yv[i] = in ? __ldcg(ys + j) : 0.f;
+      av[i] = in ? acc[j] : 0.f;
+      pv[i] = in ? pos[j] : 0x7fffffff;
+    }
+#pragma unroll
+    for (int i = 0; i < BATCH; ++i) {
+      const int j = j0 + i * NT;
+      if (j < len) {
+        const float z = fast_exp2((yv[i] - my) * LOG2E) * inv_ly;
+        const float a = av[i] + z;
+        acc[j] = a;
+        if (sc) sc[j] = z;
+        if (pv[i] <= cutoff) {
+          const unsigned long long key = evict_key(a, pv[i]);
+          if (key < best) { best = key; best_j = j; }
+        }
+      }
     }
   }
   const float z_new = fast_exp2((y_new - my) * LOG2E) * inv_ly;
@@ -121,6 +139,7 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
     return;
   }
 
+  const unsigned long long mine = best;
   if (P.w == 0) best = key_new < best ? key_new : best;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -138,12 +157,10 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
     return;
   }
   if (best == key_new && P.w == 0) return;  // the new token itself has the lowest score: it is not stored
-  const int victim_pos = (int)(0xFFFFFFFFu - (uint32_t)(best & 0xFFFFFFFFull));
-  for (int j = tid; j < len; j += NT)
-    if (pos[j] == victim_pos) sh_victim = j;
+  if (mine == best) sh_victim = best_j;      // keys are unique (positions are), so exactly one thread owns it
   __syncthreads();
   const int jv = sh_victim;
-  if (jv < 0) {
+  if (jv < 0 || jv >= len) {
     if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
     return;
   }
