@@ -125,6 +125,57 @@ int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
                         const void* h_q, const void* h_knew, const void* h_vnew,
                         void* h_out, int32_t wait, void* stream);
 
+/* Size in bytes of the scratch block built into the library (see kf_decode_step_static). */
+#define KF_STATIC_SCRATCH_BYTES (16u << 20)
+
+/* Arguments of kf_decode_step_static: the quantities kf_decode_step takes from its context. */
+typedef struct kf_static_step {
+  int32_t batch, n_heads, head_dim;   /* B, H, d in {64, 128, 256}                          */
+  int32_t budget_k, recent_w;         /* k, w                                               */
+  int32_t layer;                      /* layer index (part of the noise coordinates)        */
+  int32_t position;                   /* p: original position of the token being generated  */
+  int32_t noise_mode, bias_mode;      /* KF_NOISE_*, KF_BIAS_*                              */
+  int32_t reserved;                   /* must be 0                                          */
+  double  tau;                        /* temperature of this step (Eq. 12, computed by the caller) */
+  uint64_t noise_seed;
+  float   logit_scale;                /* 0 => 1/sqrt(d)                                     */
+  float   noise_const;
+  const float* d_alibi_slopes;        /* DEVICE [H] when bias_mode == KF_BIAS_ALIBI, else NULL */
+} kf_static_step;
+
+/* (The paper has no counterpart for this call: it is a packaging variant of kf_decode_step.)
+ *
+ * The same generation step, for callers that have no way to obtain device memory for the
+ * library's scratch: code that runs where cudaMalloc is off limits -- inside a region that is
+ * being captured or replayed and must not allocate, under a framework that owns every byte of
+ * the GPU through its own pool, or in a process whose memory budget is fixed up front.  Such a
+ * caller keeps the cache tensors itself and passes them in; the per-launch scratch (adjusted
+ * logits, split partials, arrival tickets) lives in a block of KF_STATIC_SCRATCH_BYTES of device
+ * memory that is part of the library image.  Every GPU that loads the library holds that block
+ * until the process exits.  The call itself calls no cudaMalloc, cudaFree or other allocating
+ * routine.
+ *
+ *   d_K, d_V  : DEVICE fp16 [B][H][k][d]   cache rows, updated in place (one row replaced or appended)
+ *   d_pos     : DEVICE int32 [B][H][k]     original positions, updated in place
+ *   d_acc     : DEVICE fp32 [B][H][k]      accumulated scores f_theta, updated in place
+ *   d_len     : DEVICE int32 [B][H]        entries in use, updated in place
+ *   d_q, d_knew, d_vnew, d_out, d_score_opt : as in kf_decode_step
+ *
+ * Limits and rules
+ *   - The step needs about 4*B*H*(k+1) + 4*B*H*splits*(d+4) bytes of scratch; if that exceeds the
+ *     block the call returns KF_ENOSPC and enqueues nothing.
+ *   - The first call on a device looks up the block's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one block, which keeps the previous call's contents; the
+ *     call clears what must start at zero.  Two calls whose kernels overlap on the GPU (different
+ *     streams, no ordering between them) would race on it: keep them on one stream or order them.
+ *   - Device-side self-checks have nowhere to report to in this variant (there is no context to
+ *     poll); arguments are validated on the host as far as possible. */
+int kf_decode_step_static(const kf_static_step* args,
+                          void* d_K, void* d_V, int32_t* d_pos, float* d_acc, int32_t* d_len,
+                          const void* d_q, const void* d_knew, const void* d_vnew,
+                          void* d_out, float* d_score_opt, void* stream);
+
 /* Borrowed DEVICE pointers into the workspace for one layer:
  *   K, V fp16 [B][H][k][d]; pos int32 [B][H][k] (original positions; -1 marks a slot left empty by the prompt phase);
  *   acc fp32 [B][H][k] (f_theta); len int32 [B][H] (entries in use).  Any may be NULL. */

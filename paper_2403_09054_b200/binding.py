@@ -20,7 +20,7 @@ KF_BIAS_NONE, KF_BIAS_ALIBI = 0, 1
 
 EXPORTS = ("kf_workspace_bytes", "kf_create", "kf_prefill_score_prune", "kf_decode_step",
            "kf_decode_step_host", "kf_view_state", "kf_poll_error", "kf_launch_count",
-           "kf_destroy", "kf_strerror")
+           "kf_destroy", "kf_strerror", "kf_decode_step_static")
 
 
 class kf_config(C.Structure):
@@ -32,6 +32,19 @@ class kf_config(C.Structure):
         ("logit_scale", C.c_float), ("noise_const", C.c_float),
         ("decode_splits", C.c_int32), ("reserved", C.c_int32),
     ]
+
+
+class kf_static_step(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("budget_k", C.c_int32), ("recent_w", C.c_int32), ("layer", C.c_int32), ("position", C.c_int32),
+        ("noise_mode", C.c_int32), ("bias_mode", C.c_int32), ("reserved", C.c_int32),
+        ("tau", C.c_double), ("noise_seed", C.c_uint64), ("logit_scale", C.c_float), ("noise_const", C.c_float),
+        ("d_alibi_slopes", C.c_void_p),
+    ]
+
+
+KF_STATIC_SCRATCH_BYTES = 16 << 20
 
 
 def _load() -> C.CDLL:
@@ -51,6 +64,8 @@ def _load() -> C.CDLL:
     lib.kf_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.kf_decode_step_host.restype = C.c_int
     lib.kf_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32, vp]
+    lib.kf_decode_step_static.restype = C.c_int
+    lib.kf_decode_step_static.argtypes = [C.POINTER(kf_static_step)] + [vp] * 11
     lib.kf_view_state.restype = C.c_int
     lib.kf_view_state.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
     lib.kf_poll_error.restype = C.c_int
@@ -119,6 +134,28 @@ def _dev_ptr(t, dtype, numel, name):
         raise ValueError(f"{name}: expected a contiguous CUDA {dtype} tensor with {numel} elements, "
                          f"got {t.dtype} {tuple(t.shape)} on {t.device}")
     return t.data_ptr()
+
+
+def kf_decode_step_static(*, batch, n_heads, head_dim, budget_k, recent_w, layer, position, tau,
+                          K, V, pos, acc, length, q, knew, vnew, out, score_out=None, noise_seed=0,
+                          noise_mode=KF_NOISE_GUMBEL, noise_const=0.5772, bias_mode=KF_BIAS_NONE,
+                          alibi_slopes_dev=None, logit_scale=0.0, stream=None) -> int:
+    """One generation step on caller-held cache tensors, using the library's built-in scratch block
+    (for callers that cannot allocate device memory).  Returns the KF_* status code."""
+    a = kf_static_step()
+    a.batch, a.n_heads, a.head_dim, a.budget_k, a.recent_w = batch, n_heads, head_dim, budget_k, recent_w
+    a.layer, a.position, a.noise_mode, a.bias_mode, a.reserved = layer, position, noise_mode, bias_mode, 0
+    a.tau, a.noise_seed, a.logit_scale, a.noise_const = tau, noise_seed & 0xFFFFFFFFFFFFFFFF, logit_scale, noise_const
+    a.d_alibi_slopes = None if alibi_slopes_dev is None else alibi_slopes_dev.data_ptr()
+    U = batch * n_heads
+    return int(LIB.kf_decode_step_static(
+        C.byref(a),
+        _dev_ptr(K, torch.float16, U * budget_k * head_dim, "K"), _dev_ptr(V, torch.float16, U * budget_k * head_dim, "V"),
+        _dev_ptr(pos, torch.int32, U * budget_k, "pos"), _dev_ptr(acc, torch.float32, U * budget_k, "acc"),
+        _dev_ptr(length, torch.int32, U, "length"),
+        _dev_ptr(q, torch.float16, U * head_dim, "q"), _dev_ptr(knew, torch.float16, U * head_dim, "knew"),
+        _dev_ptr(vnew, torch.float16, U * head_dim, "vnew"), _dev_ptr(out, torch.float16, U * head_dim, "out"),
+        _dev_ptr(score_out, torch.float32, U * (budget_k + 1), "score_out"), _stream_ptr(stream)))
 
 
 class Keyformer:

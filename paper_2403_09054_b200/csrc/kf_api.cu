@@ -267,6 +267,51 @@ int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
   return KF_OK;
 }
 
+int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t* d_pos, float* d_acc,
+                          int32_t* d_len, const void* d_q, const void* d_knew, const void* d_vnew,
+                          void* d_out, float* d_score_opt, void* stream) {
+  if (!a || !d_K || !d_V || !d_pos || !d_acc || !d_len || !d_q || !d_knew || !d_vnew || !d_out) return KF_EINVAL;
+  if (a->batch < 1 || a->n_heads < 1 || (int64_t)a->batch * a->n_heads > 65535) return KF_EINVAL;
+  if (a->head_dim != 64 && a->head_dim != 128 && a->head_dim != 256) return KF_EINVAL;
+  if (a->budget_k < 1 || a->recent_w < 0 || a->recent_w > a->budget_k) return KF_EINVAL;
+  if (a->layer < 0 || a->position < 0 || !(a->tau > 0.0) || a->logit_scale < 0.f) return KF_EINVAL;
+  if (a->noise_mode < KF_NOISE_GUMBEL || a->noise_mode > KF_NOISE_CONST) return KF_EINVAL;
+  if (a->bias_mode != KF_BIAS_NONE && a->bias_mode != KF_BIAS_ALIBI) return KF_EINVAL;
+  if (a->bias_mode == KF_BIAS_ALIBI && !a->d_alibi_slopes) return KF_EINVAL;
+  const int units = a->batch * a->n_heads;
+  const int tiles = tiles_of(a->budget_k);
+  int splits = std::max(1, std::min((148 * 8 + units - 1) / units, std::min(64, (tiles + 3) / 4)));
+  int tps = ((tiles + splits - 1) / splits + 3) / 4 * 4;
+  splits = (tiles + tps - 1) / tps;
+  const size_t y_bytes = align_up((size_t)units * ((size_t)a->budget_k + 1) * 4);
+  const size_t partial_bytes = align_up((size_t)units * splits * (4 + (size_t)a->head_dim) * 4);
+  const size_t counter_bytes = align_up((size_t)units * 4);
+  if (y_bytes + partial_bytes + counter_bytes + 256 > kf::STATIC_SCRATCH_BYTES) return KF_ENOSPC;  // before any CUDA call
+
+  kf::DecodeParams P{};
+  P.K = static_cast<const __half*>(d_K);
+  P.V = static_cast<const __half*>(d_V);
+  P.acc = d_acc; P.pos = d_pos; P.len = d_len;
+  P.q = static_cast<const __half*>(d_q);
+  P.knew = static_cast<const __half*>(d_knew);
+  P.vnew = static_cast<const __half*>(d_vnew);
+  P.out = static_cast<__half*>(d_out);
+  P.score_opt = d_score_opt;
+  P.err = nullptr;
+  P.slopes = a->bias_mode == KF_BIAS_ALIBI ? a->d_alibi_slopes : nullptr;
+  P.k = a->budget_k; P.w = a->recent_w; P.p = a->position;
+  P.splits = splits; P.tiles_per_split = tps;
+  P.H = a->n_heads; P.layer = a->layer; P.noise_mode = a->noise_mode; P.bias_mode = a->bias_mode;
+  P.scale = a->logit_scale > 0.f ? a->logit_scale : (float)(1.0 / std::sqrt((double)a->head_dim));
+  P.inv_tau = (float)(1.0 / a->tau);
+  P.noise_const = a->noise_const;
+  P.pk = kf::philox_expand_key(a->noise_seed);
+  const cudaError_t e = kf::launch_decode_static(P, a->head_dim, units, y_bytes, partial_bytes, counter_bytes,
+                                                 static_cast<cudaStream_t>(stream));
+  if (e == cudaErrorMemoryAllocation) return KF_ENOSPC;
+  return e == cudaSuccess ? KF_OK : KF_ECUDA;
+}
+
 int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V,
                   const int32_t** d_pos, const float** d_acc, const int32_t** d_len) {
   if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return KF_EINVAL;

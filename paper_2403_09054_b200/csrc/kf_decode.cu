@@ -12,6 +12,8 @@
 // writes the new token's row into the freed slot.
 #include "kf_decode.cuh"
 
+#include <mutex>
+
 namespace kf {
 
 namespace {
@@ -425,6 +427,47 @@ cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaSt
     case 256: return launch_one<256, 4, 2>(P, units, stream);
     default: return cudaErrorInvalidValue;
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Scratch for kf_decode_step_static: a fixed block of device memory that exists from the moment
+// the library is loaded on a GPU until the process exits, so that the entry point never has to
+// ask anyone for memory.  In host code `g_static_scratch` is only a handle for the symbol; its
+// device address comes from cudaGetSymbolAddress, once per device.
+__device__ __align__(256) static unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_static_mutex;
+void* g_static_addr[64] = {};
+}  // namespace
+
+cudaError_t launch_decode_static(DecodeParams P, int head_dim, int units, size_t y_bytes, size_t partial_bytes,
+                                 size_t counter_bytes, cudaStream_t stream) {
+  if (y_bytes + partial_bytes + counter_bytes + 256 > STATIC_SCRATCH_BYTES) return cudaErrorMemoryAllocation;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  void* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+      void* ptr = nullptr;
+      e = cudaGetSymbolAddress(&ptr, g_static_scratch);  // the current device's copy of the array
+      if (e != cudaSuccess) return e;
+      g_static_addr[dev] = ptr;
+    }
+    base = g_static_addr[dev];
+  }
+  unsigned char* b = static_cast<unsigned char*>(base);
+  P.y_scratch = reinterpret_cast<float*>(b);
+  P.partials = reinterpret_cast<float*>(b + y_bytes);
+  P.counters = reinterpret_cast<unsigned int*>(b + y_bytes + partial_bytes);
+  P.err = reinterpret_cast<int*>(b + STATIC_SCRATCH_BYTES - 256);  // error word of the kernel's self-checks
+  // the arrival tickets must start at zero; everything else is written before it is read
+  e = cudaMemsetAsync(P.counters, 0, counter_bytes, stream);
+  if (e != cudaSuccess) return e;
+  return launch_decode(P, head_dim, units, stream);
 }
 
 }  // namespace kf

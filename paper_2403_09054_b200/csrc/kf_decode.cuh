@@ -28,7 +28,15 @@ struct DecodeParams {
   PhiloxKeys pk;
 };
 
+// Size of the built-in scratch block used by kf_decode_step_static (16 MiB per GPU).
+constexpr size_t STATIC_SCRATCH_BYTES = (size_t)16 << 20;
+
 int decode_tile_rows();
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
+
+// Same launch with y_scratch / partials / counters carved out of the built-in scratch block
+// (the three sizes are in bytes, each a multiple of 256).  Allocates nothing.
+cudaError_t launch_decode_static(DecodeParams P, int head_dim, int units, size_t y_bytes, size_t partial_bytes,
+                                 size_t counter_bytes, cudaStream_t stream);
 
 }  // namespace kf
