@@ -117,6 +117,16 @@ def max_over_ranks(value: float, world: int, device) -> float:
     return float(t.item())
 
 
+def rank_workload(wl: W.Workload, rank: int) -> W.Workload:
+    """Every rank owns its own batch rows (weak scaling): same shape, different data seed."""
+    return wl.scaled(data_seed=wl.data_seed + 1000 * rank)
+
+
+def whole_job_rate(ms_per_step: float, world: int) -> float:
+    """Steps per second summed over the ranks, from the slowest rank's time per step."""
+    return world * 1e3 / ms_per_step
+
+
 def barrier(world: int):
     if world > 1:
         import torch.distributed as dist
@@ -185,7 +195,7 @@ def run_ours(args, wl):
     rank, world, local = dist_setup(args.gpus)
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
-    wl_r = wl.scaled(data_seed=wl.data_seed + 1000 * rank)   # every rank owns its own batch rows (weak scaling)
+    wl_r = rank_workload(wl, rank)
     gpu = kf.Keyformer(device=dev, n_layers=wl.n_layers, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
                        budget_k=wl.budget_k, recent_w=wl.recent_w, max_prompt_len=wl.prompt_len,
                        gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
@@ -235,7 +245,7 @@ def run_ours(args, wl):
     total_ms = max_over_ranks(total_ms, world, dev)
     assert gpu.kf_poll_error() == 0
     ms_per_step = total_ms / args.steps
-    value = world * 1e3 / ms_per_step
+    value = whole_job_rate(ms_per_step, world)
 
     vec_bytes = B * H * d * 2
     e2e_ms = None
