@@ -46,6 +46,10 @@ extern "C" {
 #define KF_NOISE_NONE   1   /* zeta = 0 (accumulated-attention score, H2O-like)      */
 #define KF_NOISE_CONST  2   /* zeta = noise_const                                     */
 
+/* How kf_prefill_score_prune computes the prompt logits Q K^T. */
+#define KF_PREFILL_TENSOR 0 /* tcgen05 tensor cores, accumulators in tensor memory (default) */
+#define KF_PREFILL_SIMT   1 /* CUDA cores; scores are summed with floating-point atomics     */
+
 #define KF_BIAS_NONE  0
 #define KF_BIAS_ALIBI 1     /* x_ij += -slope_h * (i - j) on ORIGINAL token positions (section 4.4.2) */
 
@@ -71,7 +75,7 @@ typedef struct kf_config {
   float   logit_scale;     /* 0 => 1/sqrt(d) (Eq. 1 / Eq. 4)                      */
   float   noise_const;     /* c of KF_NOISE_CONST                                 */
   int32_t decode_splits;   /* 0 = choose automatically; else CTAs per unit in the decode kernel */
-  int32_t reserved;        /* must be 0                                           */
+  int32_t prefill_impl;    /* KF_PREFILL_*                                        */
 } kf_config;
 
 /* Bytes of device workspace kf_create needs for this configuration

@@ -19,7 +19,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 struct Layout {
   size_t K, V, acc, pos, len;          // per-layer strides are kv_layer / sc_layer / len_layer
   size_t y_scratch, partials, counters, err, slopes;
-  size_t acc_full, idx, staging;
+  size_t acc_full, idx, staging, lse2;
   size_t total;
   size_t kv_layer, sc_layer, len_layer; // bytes per layer
   int units, max_splits;
@@ -36,7 +36,7 @@ bool config_ok(const kf_config* c) {
   if (c->bias_mode != KF_BIAS_NONE && c->bias_mode != KF_BIAS_ALIBI) return false;
   if (c->bias_mode == KF_BIAS_ALIBI && !c->h_alibi_slopes) return false;
   if (c->logit_scale < 0.f || c->decode_splits < 0) return false;
-  if (c->reserved != 0) return false;
+  if (c->prefill_impl != KF_PREFILL_TENSOR && c->prefill_impl != KF_PREFILL_SIMT) return false;
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
   return true;
 }
@@ -67,6 +67,7 @@ Layout make_layout(const kf_config* c) {
   L.acc_full = off; off += align_up(units * (size_t)c->max_prompt_len * 4);
   L.idx = off; off += align_up(units * k * 4);
   L.staging = off; off += 4 * align_up(units * d * 2);
+  L.lse2 = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
   L.total = off;
   return L;
 }
@@ -133,20 +134,37 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float* acc_full = d_score_opt ? d_score_opt : reinterpret_cast<float*>(ctx->ws + L.acc_full);
   int* err = reinterpret_cast<int*>(ctx->ws + L.err);
-  if (cudaMemsetAsync(acc_full, 0, (size_t)L.units * n_prompt * 4, st) != cudaSuccess) return KF_ECUDA;
-
-  kf::PrefillParams P{};
-  P.Q = static_cast<const __half*>(d_q);
-  P.K = static_cast<const __half*>(d_k);
-  P.acc_full = acc_full;
-  P.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
-  P.err = err;
-  P.n = n_prompt; P.H = c.n_heads; P.layer = layer; P.noise_mode = c.noise_mode; P.bias_mode = c.bias_mode;
-  P.scale = ctx->scale;
-  P.inv_tau = (float)(1.0 / (double)c.tau_init);  // the prompt phase is iteration t = 0 of Eq. 12
-  P.noise_const = c.noise_const;
-  P.pk = ctx->pk;
-  if (kf::launch_prefill_score_simt(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+  const float* slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
+  const float inv_tau = (float)(1.0 / (double)c.tau_init);  // the prompt phase is iteration t = 0 of Eq. 12
+  if (c.prefill_impl == KF_PREFILL_TENSOR) {
+    kf::PrefillTcArgs A{};
+    A.Q = static_cast<const __half*>(d_q);
+    A.K = static_cast<const __half*>(d_k);
+    A.lse2 = reinterpret_cast<float*>(ctx->ws + L.lse2);
+    A.acc_full = acc_full;
+    A.slopes = slopes;
+    A.err = err;
+    A.n = n_prompt; A.H = c.n_heads; A.layer = layer; A.noise_mode = c.noise_mode; A.bias_mode = c.bias_mode;
+    A.scale = ctx->scale; A.inv_tau = inv_tau; A.noise_const = c.noise_const;
+    A.pk = ctx->pk;
+    if (kf::launch_prefill_score_tc(A, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+    ctx->launches += 2;
+  } else {
+    if (cudaMemsetAsync(acc_full, 0, (size_t)L.units * n_prompt * 4, st) != cudaSuccess) return KF_ECUDA;
+    kf::PrefillParams P{};
+    P.Q = static_cast<const __half*>(d_q);
+    P.K = static_cast<const __half*>(d_k);
+    P.acc_full = acc_full;
+    P.slopes = slopes;
+    P.err = err;
+    P.n = n_prompt; P.H = c.n_heads; P.layer = layer; P.noise_mode = c.noise_mode; P.bias_mode = c.bias_mode;
+    P.scale = ctx->scale;
+    P.inv_tau = inv_tau;
+    P.noise_const = c.noise_const;
+    P.pk = ctx->pk;
+    if (kf::launch_prefill_score_simt(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+    ctx->launches += 1;
+  }
 
   kf::SelectParams S{};
   S.acc_full = acc_full;
@@ -168,7 +186,7 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
   G.n = n_prompt; G.k = c.budget_k;
   if (kf::launch_prefill_gather(G, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
 
-  ctx->launches += 3;
+  ctx->launches += 2;
   ctx->n_prompt[layer] = n_prompt;
   ctx->last_step[layer] = 0;
   return KF_OK;

@@ -1,5 +1,7 @@
-// Launch interface of the prompt-phase kernels (see kf_prefill_simt.cu).
+// Launch interface of the prompt-phase kernels (see kf_prefill_tc.cu and kf_prefill_simt.cu).
 #pragma once
+
+#include <cuda.h>
 
 #include "kf_common.cuh"
 
@@ -36,6 +38,37 @@ struct GatherParams {
   int32_t n, k;
 };
 
+// Kernel parameters of the tensor-core scoring kernel (both sweeps).
+struct PrefillTcParams {
+  CUtensorMap tmQ;     // fp16 [units][n][d], 64 x 128 boxes, 128-byte swizzle
+  CUtensorMap tmK;
+  float* lse2;         // [units][nblk * 128] log2-domain log-sum-exp of every query row (+inf past n)
+  float* acc_full;     // [units][n] f_theta before pruning
+  const float* slopes; // [H] or null
+  int* err;
+  int32_t n, nblk, H, layer;
+  float a_scale;       // logit scale * log2(e) / tau
+  float c1;            // log2(e) / tau
+  float inv_tau;
+  float const_term;    // constant logit adjustment in the scaled log2 domain (0 without one)
+  PhiloxKeys pk;
+};
+
+// What the caller of the tensor-core scoring provides.
+struct PrefillTcArgs {
+  const __half* Q;     // [units][n][d]
+  const __half* K;
+  float* lse2;         // scratch, prefill_tc_lse_floats(units, n) floats
+  float* acc_full;     // [units][n], fully overwritten
+  const float* slopes;
+  int* err;
+  int32_t n, H, layer, noise_mode, bias_mode;
+  float scale, inv_tau, noise_const;
+  PhiloxKeys pk;
+};
+
+size_t prefill_tc_lse_floats(int units, int n_max);
+cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int units, cudaStream_t stream);
 cudaError_t launch_prefill_score_simt(const PrefillParams& P, int head_dim, int units, cudaStream_t stream);
 cudaError_t launch_prefill_select(const SelectParams& P, int units, cudaStream_t stream);
 cudaError_t launch_prefill_gather(const GatherParams& P, int head_dim, int units, cudaStream_t stream);

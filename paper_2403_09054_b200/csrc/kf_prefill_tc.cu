@@ -1,0 +1,518 @@
+// Prompt-phase scoring on the 5th-generation tensor cores (Algorithm 1, t = 0; section 3.4).
+//
+// The causal logits X = Q K^T are a dense contraction, so they run as tcgen05.mma tiles with
+// the accumulators in tensor memory; everything the method adds on top of them -- the logit
+// adjustment zeta of Eq. 4, the temperature, the row softmax of Eq. 11 and the accumulation of
+// the scores over query rows -- is per-element arithmetic done by the CUDA cores on the
+// accumulator tiles as they are read back.  Two launches of one kernel template:
+//
+//   sweep 1  D = Q_blk K_tile^T : an accumulator lane is a QUERY row, so a thread keeps that
+//            row's running maximum and normaliser in registers; output lse2[i] =
+//            log2 sum_j 2^(y2_ij) with y2 = (x + zeta) log2(e) / tau.
+//   sweep 2  D = K_blk Q_tile^T : the operands swap places, an accumulator lane is a KEY, so a
+//            thread sums z_ij = 2^(y2_ij - lse2[i]) over the queries i >= j in a register and
+//            stores f_theta(j) directly: no atomics, a reproducible summation order.
+//
+// One CTA owns a block of 128 rows of the resident operand and streams 128-row tiles of the
+// other one through a ring of shared-memory stages.  Warp 0 issues the TMA loads (128-byte
+// swizzled boxes, no multicast), warp 1 owns tensor memory and issues the MMAs, warps 2..9 are
+// two groups of four compute warps that take accumulator tiles alternately (a warp can read
+// the 32 accumulator lanes selected by warp id mod 4).  Every wait is bounded; a wait that runs
+// out raises the error word and the CTA drains and frees tensor memory before it leaves.
+#include "kf_prefill.cuh"
+
+#include <cuda.h>
+
+#include <mutex>
+
+namespace kf {
+
+namespace {
+
+constexpr int TC_BM = 128;                    // rows of the resident operand (accumulator lanes)
+constexpr int TC_BN = 128;                    // rows of a streamed tile (accumulator columns)
+constexpr int TC_NCW = 8;                     // compute warps
+constexpr int TC_THREADS = (2 + TC_NCW) * 32;
+constexpr int TC_NACC = 4;                    // accumulator buffers: 4 x 128 columns = all of tensor memory
+constexpr uint32_t TC_TMEM_COLS = 512;
+constexpr uint32_t TC_WAIT_LIMIT = 1u << 21;
+constexpr int TC_BOX_BYTES = 128 * 128;       // one TMA box: 128 rows x 64 binary16
+constexpr int TC_XBUF_FLOATS = 4 * 32 * 4;    // per warp: 4 noise calls x 32 lanes x 4 words
+constexpr float LG2_LN2 = -0.5287663729448977f;  // log2(ln 2)
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, binary16 operands, binary32 accumulation, issued by one thread.
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The barrier receives one arrival once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// 32 lanes x 32 consecutive binary32 columns: thread t of the warp receives lane (base + t).
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  tmem_wait_ld();
+#pragma unroll
+  for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
+}
+
+// Shared-memory matrix descriptor of a K-major operand stored as 128-byte swizzled rows
+// (what a TMA box with CU_TENSOR_MAP_SWIZZLE_128B writes): 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4)      // start address / 16
+         | (1ull << 16)                            // leading byte offset (unused with swizzle) = 1
+         | ((uint64_t)(1024 >> 4) << 32)           // stride byte offset between 8-row groups
+         | (1ull << 46)                            // descriptor version of sm_100
+         | (2ull << 61);                           // 128-byte swizzle
+}
+
+// Instruction descriptor: binary16 A and B, both K-major, binary32 accumulator, M = 128, N = 128.
+constexpr uint32_t UMMA_IDESC = (1u << 4) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+
+// Bounded wait that also gives up when another role of the CTA has already given up.
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < TC_WAIT_LIMIT; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if (it > 32) {
+      __nanosleep(40);
+      if ((it & 127u) == 0u && *abort_flag) return false;
+    }
+  }
+  return false;
+}
+
+// ------------------------------------------------------------------ the logit adjustment
+// Same u as uniform_from_word(): ((r >> 9) + 1/2) / 2^23, built without an int->float conversion.
+__device__ __forceinline__ float uniform_from_word_bits(uint32_t r) {
+  return __uint_as_float((r >> 9) | 0x3f800000u) - 0.99999994f;   // [1, 2) grid minus (1 - 2^-24): exact
+}
+// -log2(u), relative error of a few 1e-6 (the series takes over where the fast logarithm loses accuracy).
+__device__ __forceinline__ float neg_lg2_uniform(float u) {
+  const float v = 1.0f - u;
+  const float series = v * fmaf(v, fmaf(v, fmaf(v, 0.25f, 0.33333334f), 0.5f), 1.0f) * LOG2E;
+  const float direct = -__log2f(u);
+  return v < 0.03125f ? series : direct;
+}
+// The four noise terms of one Philox call in the scaled log2 domain:
+//   zeta * log2(e) / tau = -(log2(-log2 u) + log2 ln 2) / tau     with zeta = -ln(-ln u)   (Eq. 7)
+__device__ __forceinline__ float4 noise_terms(const PhiloxKeys& pk, uint32_t jgroup, uint32_t i, uint32_t lh, uint32_t b,
+                                              float neg_inv_tau, float offset) {
+  const uint4 r = philox4x32_10(jgroup, i, lh, b, pk);
+  float4 t;
+  t.x = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.x))), neg_inv_tau, offset);
+  t.y = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.y))), neg_inv_tau, offset);
+  t.z = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.z))), neg_inv_tau, offset);
+  t.w = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.w))), neg_inv_tau, offset);
+  return t;
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int D, int NST, bool SWEEP2, bool NOISE, bool ALIBI>
+__global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constant__ PrefillTcParams P) {
+  constexpr int OP_BYTES = TC_BM * D * 2;  // one operand block: D / 64 boxes
+  constexpr int KCH = D / 64;              // 64-column boxes per operand row
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* sR = smem;                                  // resident operand
+  unsigned char* sS = smem + OP_BYTES;                       // NST stages of the streamed operand
+  float* xbuf = reinterpret_cast<float*>(sS + (size_t)NST * OP_BYTES);  // [TC_NCW][TC_XBUF_FLOATS] noise exchange
+  float* lse_s = xbuf + TC_NCW * TC_XBUF_FLOATS;             // [TC_NCW][2][128] lse2 of the current query tile
+  float* comb = lse_s + TC_NCW * 2 * 128;                    // [2][128] hand-over between the two compute groups
+  uint64_t* bars = reinterpret_cast<uint64_t*>(comb + 2 * 128);
+  uint64_t* r_full = bars;
+  uint64_t* s_full = bars + 1;
+  uint64_t* s_empty = s_full + NST;
+  uint64_t* t_full = s_empty + NST;
+  uint64_t* t_empty = t_full + TC_NACC;
+  uint64_t* drain = t_empty + TC_NACC;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* issued_slot = const_cast<int*>(abort_flag) + 1;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int u = blockIdx.y;
+  const int nblk = P.nblk;
+  const int Rb = SWEEP2 ? (int)blockIdx.x : nblk - 1 - (int)blockIdx.x;   // the longest CTAs of a unit start first
+  const int t_begin = SWEEP2 ? Rb : 0;
+  const int n_tiles = SWEEP2 ? nblk - Rb : Rb + 1;
+  const CUtensorMap* mapR = SWEEP2 ? &P.tmK : &P.tmQ;
+  const CUtensorMap* mapS = SWEEP2 ? &P.tmQ : &P.tmK;
+
+  if (tid == 0) {
+    mbar_init(r_full, 1);
+    for (int s = 0; s < NST; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, 1); }
+    for (int a = 0; a < TC_NACC; ++a) { mbar_init(t_full + a, 1); mbar_init(t_empty + a, 4); }
+    mbar_init(drain, 1);
+    *abort_flag = 0;
+    *issued_slot = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, TC_TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // per-thread results of the compute warps
+  float row_m = -INFINITY, row_l = 0.f;   // sweep 1: running maximum / normaliser of this query row
+  float col_sum = 0.f;                    // sweep 2: f_theta partial of this key
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(r_full, OP_BYTES);
+      for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sR + kc * TC_BOX_BYTES, mapR, kc * 64, Rb * TC_BM, u, r_full);
+      int it = 0;
+      for (; it < n_tiles; ++it) {
+        const int s = it % NST;
+        if (it >= NST && !wait_bar(s_empty + s, (uint32_t)((it / NST - 1) & 1), abort_flag)) {
+          *abort_flag = 1;
+          atomicExch(P.err, ERR_TIMEOUT);
+          break;
+        }
+        mbar_expect_tx(s_full + s, OP_BYTES);
+        unsigned char* dst = sS + (size_t)s * OP_BYTES;
+        for (int kc = 0; kc < KCH; ++kc) tma_load_3d(dst + kc * TC_BOX_BYTES, mapS, kc * 64, (t_begin + it) * TC_BN, u, s_full + s);
+      }
+      *issued_slot = it;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = wait_bar(r_full, 0, abort_flag);
+      const uint32_t r_addr = smem_u32(sR);
+      for (int it = 0; ok && it < n_tiles; ++it) {
+        const int s = it % NST, a = it % TC_NACC;
+        ok = wait_bar(s_full + s, (uint32_t)((it / NST) & 1), abort_flag);
+        if (ok && it >= TC_NACC) ok = wait_bar(t_empty + a, (uint32_t)((it / TC_NACC - 1) & 1), abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t s_addr = smem_u32(sS + (size_t)s * OP_BYTES);
+        const uint32_t d_addr = tmem_base + (uint32_t)(a * TC_BN);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (uint32_t)((kk >> 2) * TC_BOX_BYTES + (kk & 3) * 32);  // box, then 16 columns = 32 bytes
+          umma_f16(d_addr, umma_smem_desc(r_addr + off), umma_smem_desc(s_addr + off), UMMA_IDESC, kk > 0 ? 1u : 0u);
+        }
+        umma_commit(s_empty + s);   // the stage may be refilled once these MMAs have read it
+        umma_commit(t_full + a);    // the accumulator tile is complete
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicExch(P.err, ERR_TIMEOUT);
+      }
+      umma_commit(drain);           // nothing of this thread's MMAs is in flight once this lands
+      (void)wait_bar(drain, 0, abort_flag);
+    }
+  } else {
+    // ------------------------------------------------------------ compute warps
+    const int cw = warp - 2;            // 0..7
+    const int grp = cw >> 2;            // which accumulator tiles: it = grp, grp + 2, ...
+    const int quarter = warp & 3;       // accumulator lanes this warp may read
+    const int row = quarter * 32 + lane;               // row of the resident block owned by this thread
+    const int g_row = Rb * TC_BM + row;                // query i (sweep 1) or key j (sweep 2)
+    const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
+    const float A = P.a_scale;
+    const float neg_inv_tau = -P.inv_tau;
+    const float n_off = NOISE ? neg_inv_tau * LG2_LN2 : P.const_term;   // additive term common to all logits
+    float sb = 0.f;
+    if (ALIBI) sb = P.slopes[h] * P.c1;
+    float* my_x = xbuf + cw * TC_XBUF_FLOATS;
+    float* my_lse = lse_s + cw * 256;
+    const float* lse_u = P.lse2 + (size_t)u * nblk * TC_BN;
+    bool ok = true;
+
+    float4 lse_next = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (SWEEP2 && grp < n_tiles) lse_next = reinterpret_cast<const float4*>(lse_u + (size_t)(t_begin + grp) * TC_BN)[lane];
+
+    for (int it = grp, k = 0; it < n_tiles; it += 2, ++k) {
+      const int a = it % TC_NACC;
+      const int t = t_begin + it;
+      const bool diag = (t == Rb);
+      if (SWEEP2) {
+        __syncwarp();
+        reinterpret_cast<float4*>(my_lse + (k & 1) * 128)[lane] = lse_next;
+        if (it + 2 < n_tiles) lse_next = reinterpret_cast<const float4*>(lse_u + (size_t)(t + 2) * TC_BN)[lane];
+        __syncwarp();
+      }
+      ok = wait_bar(t_full + a, (uint32_t)((it / TC_NACC) & 1), abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * TC_BN);
+
+#pragma unroll 1
+      for (int c = 0; c < TC_BN / 32; ++c) {
+        // on the diagonal tile whole 32-column chunks are causally masked for this warp
+        if (diag && (SWEEP2 ? c < quarter : c > quarter)) continue;
+        const bool edge = diag && c == quarter;
+        float v[32];
+        tmem_ld_32x32(t_addr + (uint32_t)(c * 32), v);
+        const int col0 = t * TC_BN + c * 32;   // first key j (sweep 1) / first query i (sweep 2) of the chunk
+
+        if (!SWEEP2) {
+          // ---- thread = query row i; y2_j for 32 keys, then one online-softmax update
+          float bias0 = 0.f;
+          if (ALIBI) bias0 = sb * (float)(col0 - g_row);   // -slope (i - j) log2(e) / tau at e = 0
+          float y[32];
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            float4 nz = make_float4(n_off, n_off, n_off, n_off);
+            if (NOISE) nz = noise_terms(P.pk, (uint32_t)(col0 >> 2) + g, (uint32_t)g_row, lh, b, neg_inv_tau, n_off);
+            const float nn[4] = {nz.x, nz.y, nz.z, nz.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const int e = 4 * g + q;
+              float val = fmaf(v[e], A, nn[q]);
+              if (ALIBI) val += fmaf(sb, (float)e, bias0);
+              y[e] = val;
+            }
+          }
+          if (edge) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) y[e] = e <= lane ? y[e] : -INFINITY;
+          }
+          float cmax = y[0];
+#pragma unroll
+          for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, y[e]);
+          const float m_new = fmaxf(row_m, cmax);
+          const float m_use = m_new == -INFINITY ? 0.f : m_new;
+          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            s0 += fast_exp2(y[e] - m_use);
+            s1 += fast_exp2(y[e + 1] - m_use);
+            s2 += fast_exp2(y[e + 2] - m_use);
+            s3 += fast_exp2(y[e + 3] - m_use);
+          }
+          row_l = fmaf(row_l, fast_exp2(row_m - m_use), (s0 + s1) + (s2 + s3));
+          row_m = m_new;
+        } else {
+          // ---- thread = key j; z_ij for 32 queries, two halves of 16 (one noise exchange each)
+          float bias0 = 0.f;
+          if (ALIBI) bias0 = sb * (float)(g_row - col0);   // -slope (i - j) log2(e) / tau at e = 0
+          const float* lse_t = my_lse + (k & 1) * 128 + c * 32;
+          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            if (NOISE) {
+              // lane L draws the call of key group (L & 7) of this warp and query 4 g + (L >> 3);
+              // afterwards lane L reads word (L & 3) of its own key group (L >> 2) for each query.
+              __syncwarp();
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                const uint32_t jg = (uint32_t)((Rb * TC_BM + quarter * 32) >> 2) + (uint32_t)(lane & 7);
+                const uint32_t qi = (uint32_t)(col0 + half * 16 + 4 * g + (lane >> 3));
+                reinterpret_cast<float4*>(my_x)[g * 32 + lane] = noise_terms(P.pk, jg, qi, lh, b, neg_inv_tau, n_off);
+              }
+              __syncwarp();
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const float4 l4 = reinterpret_cast<const float4*>(lse_t)[half * 4 + g];
+              const float ll[4] = {l4.x, l4.y, l4.z, l4.w};
+              float pp[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const int e = half * 16 + 4 * g + q;
+                const float nz = NOISE ? my_x[(g * 32 + 8 * q + (lane >> 2)) * 4 + (lane & 3)] : n_off;
+                float val = fmaf(v[e], A, nz);
+                if (ALIBI) val += fmaf(-sb, (float)e, bias0);
+                float p = fast_exp2(val - ll[q]);
+                if (edge) p = e >= lane ? p : 0.f;
+                pp[q] = p;
+              }
+              s0 += pp[0]; s1 += pp[1]; s2 += pp[2]; s3 += pp[3];
+            }
+          }
+          col_sum += (s0 + s1) + (s2 + s3);
+        }
+      }
+      // hand the accumulator buffer back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(t_empty + a);
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicExch(P.err, ERR_TIMEOUT);
+    }
+    if (grp == 1) {
+      if (!SWEEP2) { comb[row] = row_m; comb[128 + row] = row_l; }
+      else comb[row] = col_sum;
+    }
+  }
+
+  __syncthreads();
+  if (warp >= 2 && warp < 6) {
+    const int row = (warp & 3) * 32 + lane;
+    const int g_row = Rb * TC_BM + row;
+    if (!SWEEP2) {
+      const float m1 = comb[row], l1 = comb[128 + row];
+      const float m = fmaxf(row_m, m1);
+      float lse = INFINITY;   // rows past the prompt: their scores vanish in sweep 2
+      if (g_row < P.n && m > -INFINITY) {
+        const float l = row_l * fast_exp2(row_m - m) + l1 * fast_exp2(m1 - m);
+        lse = m + log2f(l);
+      }
+      P.lse2[(size_t)u * nblk * TC_BN + g_row] = lse;
+    } else if (g_row < P.n) {
+      P.acc_full[(size_t)u * P.n + g_row] = col_sum + comb[row];
+    }
+  }
+
+  // ---- teardown: on the failure path give the copies still in flight a bounded wait, then free tensor memory
+  if (tid == 0 && *abort_flag) {
+    const int issued = *issued_slot;
+    for (int it = issued > NST ? issued - NST : 0; it < issued; ++it)
+      (void)mbar_wait_bounded(s_full + (it % NST), (uint32_t)((it / NST) & 1), TC_WAIT_LIMIT);
+    (void)mbar_wait_bounded(r_full, 0, TC_WAIT_LIMIT);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TC_TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static std::once_flag once;
+  static EncodeTiledFn fn = nullptr;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// fp16 [units][n][d] viewed as a 3-D tensor (d innermost); boxes of 64 columns x 128 rows, 128-byte swizzle.
+// Rows past n read as zeros, so a block never sees another unit's rows.
+bool make_operand_map(CUtensorMap* map, const __half* base, int units, int n, int d) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)n, (cuuint64_t)units};
+  const cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)n * d * 2};
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, int NST>
+constexpr size_t tc_smem_bytes() {
+  size_t b = 1024 + (size_t)(1 + NST) * TC_BM * D * 2 + (size_t)TC_NCW * TC_XBUF_FLOATS * 4 + (size_t)TC_NCW * 2 * 128 * 4 +
+             2 * 128 * 4 + 32 * 8 + 64;
+  return b < 120 * 1024 ? 120 * 1024 : b;   // one CTA per SM: each takes all of tensor memory
+}
+
+template <int D, int NST, bool SWEEP2>
+cudaError_t launch_variant(const PrefillTcParams& P, int units, bool noise, bool alibi, cudaStream_t st) {
+  constexpr size_t smem = tc_smem_bytes<D, NST>();
+  dim3 grid((unsigned)P.nblk, (unsigned)units);
+  auto go = [&](auto kern) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, TC_THREADS, smem, st>>>(P);
+    return cudaGetLastError();
+  };
+  if (noise) return alibi ? go(prefill_tc<D, NST, SWEEP2, true, true>) : go(prefill_tc<D, NST, SWEEP2, true, false>);
+  return alibi ? go(prefill_tc<D, NST, SWEEP2, false, true>) : go(prefill_tc<D, NST, SWEEP2, false, false>);
+}
+
+}  // namespace
+
+cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int units, cudaStream_t stream) {
+  if (a.n < 1 || units < 1 || units > 65535) return cudaErrorInvalidValue;
+  PrefillTcParams P{};
+  if (!make_operand_map(&P.tmQ, a.Q, units, a.n, head_dim)) return cudaErrorNotSupported;
+  if (!make_operand_map(&P.tmK, a.K, units, a.n, head_dim)) return cudaErrorNotSupported;
+  P.lse2 = a.lse2;
+  P.acc_full = a.acc_full;
+  P.slopes = a.slopes;
+  P.err = a.err;
+  P.n = a.n;
+  P.nblk = (a.n + TC_BM - 1) / TC_BM;
+  P.H = a.H;
+  P.layer = a.layer;
+  P.inv_tau = a.inv_tau;
+  P.c1 = LOG2E * a.inv_tau;
+  P.a_scale = a.scale * P.c1;
+  P.const_term = a.noise_mode == 2 ? a.noise_const * P.c1 : 0.f;
+  P.pk = a.pk;
+  const bool noise = a.noise_mode == 0, alibi = a.bias_mode == 1 && a.slopes != nullptr;
+  cudaError_t e;
+  switch (head_dim) {
+    case 64:
+      e = launch_variant<64, 4, false>(P, units, noise, alibi, stream);
+      if (e == cudaSuccess) e = launch_variant<64, 4, true>(P, units, noise, alibi, stream);
+      return e;
+    case 128:
+      e = launch_variant<128, 3, false>(P, units, noise, alibi, stream);
+      if (e == cudaSuccess) e = launch_variant<128, 3, true>(P, units, noise, alibi, stream);
+      return e;
+    case 256:
+      e = launch_variant<256, 2, false>(P, units, noise, alibi, stream);
+      if (e == cudaSuccess) e = launch_variant<256, 2, true>(P, units, noise, alibi, stream);
+      return e;
+    default:
+      return cudaErrorInvalidValue;
+  }
+}
+
+size_t prefill_tc_lse_floats(int units, int n_max) {
+  return (size_t)units * (size_t)((n_max + TC_BM - 1) / TC_BM) * TC_BM;
+}
+
+}  // namespace kf

@@ -18,11 +18,38 @@ def _wl(**kw):
     return W.Workload(**base)
 
 
+@pytest.mark.parametrize("impl", [kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_SIMT])
 @pytest.mark.parametrize("d", [64, 128, 256])
-def test_small_odd_shapes(d):
+def test_small_odd_shapes(d, impl):
     wl = _wl(head_dim=d, prompt_len=157, budget_k=71, recent_w=13)
-    r = lockstep.run_workload(wl)
+    r = lockstep.run_workload(wl, gpu_kwargs=dict(prefill_impl=impl))
     assert r["max_out_err"] < 2e-3
+
+
+@pytest.mark.parametrize("n", [1, 31, 128, 129, 257, 640, 1000])
+@pytest.mark.parametrize("noise", ["gumbel", "none"])
+def test_prompt_lengths_around_tile_edges(n, noise):
+    """Prompt scoring only (T = 0): one row, a partial tile, exact tiles, several tiles with a ragged tail."""
+    wl = _wl(head_dim=128, prompt_len=n, budget_k=max(1, n // 2), recent_w=max(0, n // 8), gen_len_T=0)
+    lockstep.run_workload(wl, noise=noise)
+
+
+def test_prompt_scores_tensor_core_vs_cuda_core():
+    """The two scoring implementations agree far inside the oracle tolerance, and the tensor-core
+    one is reproducible bit for bit (no atomics)."""
+    wl = _wl(head_dim=128, prompt_len=777, budget_k=300, recent_w=50, positional="alibi")
+    q, k, v = W.make_prompt(wl, 0, DEV)
+    scores = []
+    for impl in (kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_SIMT):
+        gpu = lockstep.make_gpu(wl, prefill_impl=impl)
+        s = torch.empty(wl.batch, wl.n_heads, wl.prompt_len, dtype=torch.float32, device=DEV)
+        gpu.kf_prefill_score_prune(0, q, k, v, score_out=s)
+        assert gpu.kf_poll_error() == 0
+        scores.append(s)
+        gpu.kf_destroy()
+    assert torch.equal(scores[0], scores[1])
+    assert torch.allclose(scores[0], scores[2], rtol=2e-4, atol=1e-6)
+    assert torch.allclose(scores[0].sum(-1), torch.full_like(scores[0].sum(-1), float(wl.prompt_len)), rtol=1e-4)
 
 
 @pytest.mark.parametrize("k,w,n", [(33, 0, 90), (32, 32, 90), (64, 1, 65), (40, 10, 30), (40, 10, 40), (1, 0, 5), (1, 1, 5)])
@@ -94,7 +121,7 @@ def test_call_order_and_argument_errors():
     assert e.value.code == kf.KF_EINVAL
     gpu.kf_decode_step(0, 1, q, kn, vn, out)
     assert gpu.kf_poll_error() == 0
-    assert gpu.kf_launch_count() == 4
+    assert gpu.kf_launch_count() == 5   # prompt phase: 2 scoring sweeps + select + gather; then 1 decode kernel
 
 
 def test_host_buffer_variant_matches_device_variant():
