@@ -303,6 +303,77 @@ def run_ours(args, wl):
     return line
 
 
+# ----------------------------------------------------------------------------- prompt phase
+# Lane-instructions one causal logit needs per sweep when nothing is wasted: Philox4x32-10 shared by four
+# logits (10 rounds x 4 instructions / 4), the 23-bit uniform (3), two logarithms with the u -> 1 repair (6),
+# scale + adjustment (1), subtract + exponential (2), maximum or sum (2).
+PREFILL_LANE_INSTR_PER_LOGIT_SWEEP = 24
+ALU_LANES_PER_SM, N_SM = 128, 148
+
+
+def run_prefill(args, wl):
+    """Times kf_prefill_score_prune (prompt scoring on the tensor cores + select + gather) for one layer."""
+    import paper_2403_09054_b200 as kf
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    n = wl.prompt_len
+    kk = max(1, int(round(n * args.budget_frac)))
+    wl = rank_workload(wl.scaled(budget_k=kk, recent_w=kk // 4), rank)
+    gpu = kf.Keyformer(device=dev, n_layers=1, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
+                       budget_k=wl.budget_k, recent_w=wl.recent_w, max_prompt_len=n, gen_len_T=0,
+                       tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
+                       bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
+                       alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None,
+                       prefill_impl=kf.KF_PREFILL_SIMT if args.prefill_simt else kf.KF_PREFILL_TENSOR)
+    q, k, v = W.make_prompt(wl, 0, dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        gpu.kf_prefill_score_prune(0, q, k, v, stream=stream)
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = gpu.kf_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        gpu.kf_prefill_score_prune(0, q, k, v, stream=stream)
+    e1.record(stream)
+    barrier(world)
+    clocks = sampler.stop()
+    launches = gpu.kf_launch_count() - launches0
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    assert gpu.kf_poll_error() == 0
+    if rank == 0:
+        units = wl.batch * wl.n_heads
+        logits = units * n * (n + 1) // 2
+        lane_instr = 2 * PREFILL_LANE_INSTR_PER_LOGIT_SWEEP * logits
+        sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        peak = N_SM * ALU_LANES_PER_SM * 1965.0e6 / 1e12
+        achieved = lane_instr / (ms * 1e-3) / 1e12
+        line = {
+            "metric": "prompt score-and-prune calls/sec (one layer)", "value": world * 1e3 / ms, "unit": "calls/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16 operands, f32 accumulate and score arithmetic",
+            "data": "synthetic",
+            "config": {"workload": wl.name, "phase": "prefill", "batch": wl.batch, "heads": wl.n_heads,
+                       "head_dim": wl.head_dim, "prompt": n, "budget_k": wl.budget_k, "recent_w": wl.recent_w,
+                       "causal_logits": logits, "G_logits_per_s": logits / ms / 1e6,
+                       "qk_tflops_both_sweeps": 2 * 2 * logits * wl.head_dim / (ms * 1e-3) / 1e12,
+                       "l2": "Q, K, V of the call (%.0f MB) exceed L2" % (3 * units * n * wl.head_dim * 2 / 1e6)},
+            "roofline": {"bound": "alu", "kernel": "prefill_tc (two sweeps)", "achieved": achieved, "peak": peak,
+                         "unit": "T lane-instr/s", "frac": achieved / peak, "traffic": None,
+                         "lane_instr_per_logit_sweep": PREFILL_LANE_INSTR_PER_LOGIT_SWEEP,
+                         "peak_kind": "148 SMs x 128 lanes x 1965 MHz", "sm_mhz_seen": sm_mhz},
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        print(json.dumps(line))
+    gpu.kf_destroy()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -317,11 +388,17 @@ def main():
                     help="DRAM bytes per launch of the decode kernel from an ncu capture (see profiles/)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling a small case)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (profiling a small case)")
+    ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
+                    help="decode: the generation step (the headline metric); prefill: the prompt phase of one layer")
+    ap.add_argument("--budget-frac", type=float, default=0.5, help="prefill phase: k as a fraction of the prompt")
+    ap.add_argument("--prefill-simt", action="store_true", help="prefill phase: CUDA-core scoring instead of tcgen05")
     args = ap.parse_args()
     wl = W.get_config(args.workload)
     if args.layers > 0:
         wl = wl.scaled(n_layers=args.layers, name=f"{wl.name}[layers={args.layers}]")
-    if args.impl == "reference":
+    if args.phase == "prefill" and args.impl == "ours":
+        run_prefill(args, wl)
+    elif args.impl == "reference":
         run_reference(args, wl)
     else:
         run_ours(args, wl)

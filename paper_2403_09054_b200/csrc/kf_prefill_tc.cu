@@ -15,8 +15,8 @@
 //
 // One CTA owns a block of 128 rows of the resident operand and streams 128-row tiles of the
 // other one through a ring of shared-memory stages.  Warp 0 issues the TMA loads (128-byte
-// swizzled boxes, no multicast), warp 1 owns tensor memory and issues the MMAs, warps 2..9 are
-// two groups of four compute warps that take accumulator tiles alternately (a warp can read
+// swizzled boxes, no multicast), warp 1 owns tensor memory and issues the MMAs, the other warps are
+// groups of four compute warps that take accumulator tiles in turn (a warp can read
 // the 32 accumulator lanes selected by warp id mod 4).  Every wait is bounded; a wait that runs
 // out raises the error word and the CTA drains and frees tensor memory before it leaves.
 #include "kf_prefill.cuh"
@@ -24,6 +24,7 @@
 #include <cuda.h>
 
 #include <mutex>
+#include <type_traits>
 
 namespace kf {
 
@@ -31,8 +32,11 @@ namespace {
 
 constexpr int TC_BM = 128;                    // rows of the resident operand (accumulator lanes)
 constexpr int TC_BN = 128;                    // rows of a streamed tile (accumulator columns)
-constexpr int TC_NCW = 8;                     // compute warps
-constexpr int TC_THREADS = (2 + TC_NCW) * 32;
+constexpr int tc_threads(int ng) { return (2 + 4 * ng) * 32; }   // TMA warp + MMA warp + NG groups of 4 compute warps
+#ifndef KF_TC_NG
+#define KF_TC_NG 3
+#endif
+constexpr int TC_NG = KF_TC_NG;               // compute groups for head_dim 64 / 128 (256 leaves room for 2)
 constexpr int TC_NACC = 4;                    // accumulator buffers: 4 x 128 columns = all of tensor memory
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr uint32_t TC_WAIT_LIMIT = 1u << 21;
@@ -121,43 +125,53 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
 }
 
 // ------------------------------------------------------------------ the logit adjustment
-// Same u as uniform_from_word(): ((r >> 9) + 1/2) / 2^23, built without an int->float conversion.
-__device__ __forceinline__ float uniform_from_word_bits(uint32_t r) {
-  return __uint_as_float((r >> 9) | 0x3f800000u) - 0.99999994f;   // [1, 2) grid minus (1 - 2^-24): exact
+__device__ __forceinline__ float fast_lg2(float x) {   // arguments here are normal numbers: no subnormal handling
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
-// -log2(u), relative error of a few 1e-6 (the series takes over where the fast logarithm loses accuracy).
+// Same u as uniform_from_word(): ((r >> 9) + 1/2) / 2^23, built without an int->float conversion:
+// the funnel shift places the 23 random bits under the exponent of 1.0, giving a value of [1, 2).
+__device__ __forceinline__ float uniform_from_word_bits(uint32_t r) {
+  return __uint_as_float(__funnelshift_r(r, 0x7Fu, 9)) - 0.99999994f;   // minus (1 - 2^-24): exact
+}
+// -log2(u).  The fast logarithm has an absolute error near 2^-22, too coarse once u approaches 1;
+// there (v = 1 - u < 2^-8, v exact) two terms of the series of -ln(1 - v) take over.  Relative
+// error below 5e-5 everywhere.
 __device__ __forceinline__ float neg_lg2_uniform(float u) {
   const float v = 1.0f - u;
-  const float series = v * fmaf(v, fmaf(v, fmaf(v, 0.25f, 0.33333334f), 0.5f), 1.0f) * LOG2E;
-  const float direct = -__log2f(u);
-  return v < 0.03125f ? series : direct;
+  const float series = v * fmaf(v, 0.5f * LOG2E, LOG2E);
+  const float direct = -fast_lg2(u);
+  return v < 0.00390625f ? series : direct;
 }
 // The four noise terms of one Philox call in the scaled log2 domain:
 //   zeta * log2(e) / tau = -(log2(-log2 u) + log2 ln 2) / tau     with zeta = -ln(-ln u)   (Eq. 7)
+// `offset` carries -log2(ln 2) / tau plus whatever the caller wants added to all four logits.
 __device__ __forceinline__ float4 noise_terms(const PhiloxKeys& pk, uint32_t jgroup, uint32_t i, uint32_t lh, uint32_t b,
                                               float neg_inv_tau, float offset) {
   const uint4 r = philox4x32_10(jgroup, i, lh, b, pk);
   float4 t;
-  t.x = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.x))), neg_inv_tau, offset);
-  t.y = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.y))), neg_inv_tau, offset);
-  t.z = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.z))), neg_inv_tau, offset);
-  t.w = fmaf(__log2f(neg_lg2_uniform(uniform_from_word_bits(r.w))), neg_inv_tau, offset);
+  t.x = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.x))), neg_inv_tau, offset);
+  t.y = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.y))), neg_inv_tau, offset);
+  t.z = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.z))), neg_inv_tau, offset);
+  t.w = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.w))), neg_inv_tau, offset);
   return t;
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int D, int NST, bool SWEEP2, bool NOISE, bool ALIBI>
-__global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constant__ PrefillTcParams P) {
+template <int D, int NST, int NG, bool SWEEP2, bool NOISE, bool ALIBI>
+__global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_constant__ PrefillTcParams P) {
   constexpr int OP_BYTES = TC_BM * D * 2;  // one operand block: D / 64 boxes
   constexpr int KCH = D / 64;              // 64-column boxes per operand row
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char* sR = smem;                                  // resident operand
   unsigned char* sS = smem + OP_BYTES;                       // NST stages of the streamed operand
-  float* xbuf = reinterpret_cast<float*>(sS + (size_t)NST * OP_BYTES);  // [TC_NCW][TC_XBUF_FLOATS] noise exchange
-  float* lse_s = xbuf + TC_NCW * TC_XBUF_FLOATS;             // [TC_NCW][2][128] lse2 of the current query tile
-  float* comb = lse_s + TC_NCW * 2 * 128;                    // [2][128] hand-over between the two compute groups
-  uint64_t* bars = reinterpret_cast<uint64_t*>(comb + 2 * 128);
+  constexpr int NCW = 4 * NG;                                // compute warps
+  float* xbuf = reinterpret_cast<float*>(sS + (size_t)NST * OP_BYTES);  // [NCW][TC_XBUF_FLOATS] noise exchange
+  float* lse_s = xbuf + NCW * TC_XBUF_FLOATS;                // [NCW][128] lse2 of the current query tile
+  float* comb = lse_s + NCW * 128;                           // [NG - 1][2][128] hand-over between the compute groups
+  uint64_t* bars = reinterpret_cast<uint64_t*>(comb + (NG - 1) * 2 * 128);
   uint64_t* r_full = bars;
   uint64_t* s_full = bars + 1;
   uint64_t* s_empty = s_full + NST;
@@ -196,7 +210,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constan
   const uint32_t tmem_base = *tmem_slot;
 
   // per-thread results of the compute warps
-  float row_m = -INFINITY, row_l = 0.f;   // sweep 1: running maximum / normaliser of this query row
+  float row_m = 0.f, row_l = 0.f;         // sweep 1: reference exponent and sum_j 2^(y2_j - row_m) of this query row
+  bool started = false;
   float col_sum = 0.f;                    // sweep 2: f_theta partial of this key
 
   if (warp == 0) {
@@ -249,7 +264,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constan
   } else {
     // ------------------------------------------------------------ compute warps
     const int cw = warp - 2;            // 0..7
-    const int grp = cw >> 2;            // which accumulator tiles: it = grp, grp + 2, ...
+    const int grp = cw >> 2;            // which accumulator tiles: it = grp, grp + NG, ...
     const int quarter = warp & 3;       // accumulator lanes this warp may read
     const int row = quarter * 32 + lane;               // row of the resident block owned by this thread
     const int g_row = Rb * TC_BM + row;                // query i (sweep 1) or key j (sweep 2)
@@ -260,21 +275,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constan
     float sb = 0.f;
     if (ALIBI) sb = P.slopes[h] * P.c1;
     float* my_x = xbuf + cw * TC_XBUF_FLOATS;
-    float* my_lse = lse_s + cw * 256;
+    float* my_lse = lse_s + cw * 128;
     const float* lse_u = P.lse2 + (size_t)u * nblk * TC_BN;
     bool ok = true;
 
     float4 lse_next = make_float4(0.f, 0.f, 0.f, 0.f);
     if (SWEEP2 && grp < n_tiles) lse_next = reinterpret_cast<const float4*>(lse_u + (size_t)(t_begin + grp) * TC_BN)[lane];
 
-    for (int it = grp, k = 0; it < n_tiles; it += 2, ++k) {
+    for (int it = grp; it < n_tiles; it += NG) {
       const int a = it % TC_NACC;
       const int t = t_begin + it;
       const bool diag = (t == Rb);
       if (SWEEP2) {
         __syncwarp();
-        reinterpret_cast<float4*>(my_lse + (k & 1) * 128)[lane] = lse_next;
-        if (it + 2 < n_tiles) lse_next = reinterpret_cast<const float4*>(lse_u + (size_t)(t + 2) * TC_BN)[lane];
+        reinterpret_cast<float4*>(my_lse)[lane] = lse_next;
+        if (it + NG < n_tiles) lse_next = reinterpret_cast<const float4*>(lse_u + (size_t)(t + NG) * TC_BN)[lane];
         __syncwarp();
       }
       ok = wait_bar(t_full + a, (uint32_t)((it / TC_NACC) & 1), abort_flag);
@@ -292,77 +307,112 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constan
         tmem_ld_32x32(t_addr + (uint32_t)(c * 32), v);
         const int col0 = t * TC_BN + c * 32;   // first key j (sweep 1) / first query i (sweep 2) of the chunk
 
+        // causally masked logits of the diagonal chunk: -inf in, 0 out of every exponential below
+        if (edge) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = (SWEEP2 ? e >= lane : e <= lane) ? v[e] : -INFINITY;
+        }
+
         if (!SWEEP2) {
-          // ---- thread = query row i; y2_j for 32 keys, then one online-softmax update
+          // ---- thread = query row i: add sum_j 2^(y2_j - row_m) over 32 keys to row_l.  The reference
+          //      row_m is not the exact running maximum: any value within 2^+-100 of it serves, so it moves
+          //      only when the sum leaves that range, which saves a max and a subtract per logit.
           float bias0 = 0.f;
           if (ALIBI) bias0 = sb * (float)(col0 - g_row);   // -slope (i - j) log2(e) / tau at e = 0
-          float y[32];
+          if (!started) {
+            row_m = fmaf(v[0], A, n_off + bias0);          // element 0 of a row's first chunk is never masked
+            started = true;
+          }
+          // mode 0: sum of 2^(y2 - ref); mode 1: max of y2 - ref (exact fallback, see below)
+          auto sweep_chunk = [&](float ref, auto mode) -> float {
+            constexpr bool WANT_MAX = decltype(mode)::value;
+            const float off = n_off + bias0 - ref;
+            float r0 = WANT_MAX ? -INFINITY : 0.f, r1 = r0, r2 = r0, r3 = r0;
 #pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            float4 nz = make_float4(n_off, n_off, n_off, n_off);
-            if (NOISE) nz = noise_terms(P.pk, (uint32_t)(col0 >> 2) + g, (uint32_t)g_row, lh, b, neg_inv_tau, n_off);
-            const float nn[4] = {nz.x, nz.y, nz.z, nz.w};
+            for (int g = 0; g < 8; ++g) {
+              float4 nz = make_float4(off, off, off, off);
+              if (NOISE) nz = noise_terms(P.pk, (uint32_t)(col0 >> 2) + g, (uint32_t)g_row, lh, b, neg_inv_tau, off);
+              const float nn[4] = {nz.x, nz.y, nz.z, nz.w};
+              float a4[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int e = 4 * g + q;
-              float val = fmaf(v[e], A, nn[q]);
-              if (ALIBI) val += fmaf(sb, (float)e, bias0);
-              y[e] = val;
+              for (int q = 0; q < 4; ++q) {
+                const int e = 4 * g + q;
+                a4[q] = fmaf(v[e], A, nn[q]);
+                if (ALIBI) a4[q] = fmaf(sb, (float)e, a4[q]);
+              }
+              if (WANT_MAX) {
+                r0 = fmaxf(r0, a4[0]); r1 = fmaxf(r1, a4[1]); r2 = fmaxf(r2, a4[2]); r3 = fmaxf(r3, a4[3]);
+              } else {
+                r0 += fast_exp2(a4[0]); r1 += fast_exp2(a4[1]); r2 += fast_exp2(a4[2]); r3 += fast_exp2(a4[3]);
+              }
+            }
+            return WANT_MAX ? fmaxf(fmaxf(r0, r1), fmaxf(r2, r3)) : (r0 + r1) + (r2 + r3);
+          };
+          float ref = row_m;
+          float sum = sweep_chunk(ref, std::false_type{});
+          if (!(sum < 1e30f)) {
+            // some logit lies about 2^100 or more above the reference: take the chunk's exact maximum instead
+            const float cm = sweep_chunk(ref, std::true_type{});
+            if (cm < INFINITY) {
+              ref += cm;
+              sum = sweep_chunk(ref, std::false_type{});
             }
           }
-          if (edge) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) y[e] = e <= lane ? y[e] : -INFINITY;
+          if (ref != row_m) {
+            row_l *= fast_exp2(row_m - ref);
+            row_m = ref;
           }
-          float cmax = y[0];
-#pragma unroll
-          for (int e = 1; e < 32; ++e) cmax = fmaxf(cmax, y[e]);
-          const float m_new = fmaxf(row_m, cmax);
-          const float m_use = m_new == -INFINITY ? 0.f : m_new;
-          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            s0 += fast_exp2(y[e] - m_use);
-            s1 += fast_exp2(y[e + 1] - m_use);
-            s2 += fast_exp2(y[e + 2] - m_use);
-            s3 += fast_exp2(y[e + 3] - m_use);
+          row_l += sum;
+          if (row_l > 1.8446744e19f) {   // 2^64: keep the sum far from overflow
+            row_l *= 5.4210109e-20f;     // 2^-64
+            row_m += 64.f;
           }
-          row_l = fmaf(row_l, fast_exp2(row_m - m_use), (s0 + s1) + (s2 + s3));
-          row_m = m_new;
         } else {
-          // ---- thread = key j; z_ij for 32 queries, two halves of 16 (one noise exchange each)
+          // ---- thread = key j: add z_ij = 2^(y2_ij - lse2_i) over 32 queries to col_sum
           float bias0 = 0.f;
           if (ALIBI) bias0 = sb * (float)(g_row - col0);   // -slope (i - j) log2(e) / tau at e = 0
-          const float* lse_t = my_lse + (k & 1) * 128 + c * 32;
+          const float* lse_t = my_lse + c * 32;
           float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+          if (NOISE) {
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            if (NOISE) {
-              // lane L draws the call of key group (L & 7) of this warp and query 4 g + (L >> 3);
-              // afterwards lane L reads word (L & 3) of its own key group (L >> 2) for each query.
+            for (int half = 0; half < 2; ++half) {
+              // Lane L draws the Philox call of key group (L & 7) of this warp and query 4 g + (L >> 3) and
+              // folds that query's -lse2 into the four terms; afterwards lane L reads word (L & 3) of its
+              // own key group (L >> 2) for each query.  Both access patterns are bank-conflict free.
               __syncwarp();
 #pragma unroll
               for (int g = 0; g < 4; ++g) {
+                const int ql = half * 16 + 4 * g + (lane >> 3);
                 const uint32_t jg = (uint32_t)((Rb * TC_BM + quarter * 32) >> 2) + (uint32_t)(lane & 7);
-                const uint32_t qi = (uint32_t)(col0 + half * 16 + 4 * g + (lane >> 3));
-                reinterpret_cast<float4*>(my_x)[g * 32 + lane] = noise_terms(P.pk, jg, qi, lh, b, neg_inv_tau, n_off);
+                reinterpret_cast<float4*>(my_x)[g * 32 + lane] =
+                    noise_terms(P.pk, jg, (uint32_t)(col0 + ql), lh, b, neg_inv_tau, n_off - lse_t[ql]);
               }
               __syncwarp();
-            }
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const float4 l4 = reinterpret_cast<const float4*>(lse_t)[half * 4 + g];
+              for (int g = 0; g < 4; ++g) {
+                float pp[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const int e = half * 16 + 4 * g + q;
+                  float arg = fmaf(v[e], A, my_x[(g * 32 + 8 * q + (lane >> 2)) * 4 + (lane & 3)]);
+                  if (ALIBI) arg += fmaf(-sb, (float)e, bias0);
+                  pp[q] = fast_exp2(arg);
+                }
+                s0 += pp[0]; s1 += pp[1]; s2 += pp[2]; s3 += pp[3];
+              }
+            }
+          } else {
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              const float4 l4 = reinterpret_cast<const float4*>(lse_t)[g];
               const float ll[4] = {l4.x, l4.y, l4.z, l4.w};
               float pp[4];
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
-                const int e = half * 16 + 4 * g + q;
-                const float nz = NOISE ? my_x[(g * 32 + 8 * q + (lane >> 2)) * 4 + (lane & 3)] : n_off;
-                float val = fmaf(v[e], A, nz);
-                if (ALIBI) val += fmaf(-sb, (float)e, bias0);
-                float p = fast_exp2(val - ll[q]);
-                if (edge) p = e >= lane ? p : 0.f;
-                pp[q] = p;
+                const int e = 4 * g + q;
+                float arg = fmaf(v[e], A, n_off - ll[q]);
+                if (ALIBI) arg += fmaf(-sb, (float)e, bias0);
+                pp[q] = fast_exp2(arg);
               }
               s0 += pp[0]; s1 += pp[1]; s2 += pp[2]; s3 += pp[3];
             }
@@ -379,9 +429,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constan
       *abort_flag = 1;
       atomicExch(P.err, ERR_TIMEOUT);
     }
-    if (grp == 1) {
-      if (!SWEEP2) { comb[row] = row_m; comb[128 + row] = row_l; }
-      else comb[row] = col_sum;
+    if (grp > 0) {
+      float* mine = comb + (grp - 1) * 256;
+      mine[row] = SWEEP2 ? col_sum : row_m;
+      mine[128 + row] = row_l;
     }
   }
 
@@ -390,16 +441,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc(const __grid_constan
     const int row = (warp & 3) * 32 + lane;
     const int g_row = Rb * TC_BM + row;
     if (!SWEEP2) {
-      const float m1 = comb[row], l1 = comb[128 + row];
-      const float m = fmaxf(row_m, m1);
-      float lse = INFINITY;   // rows past the prompt: their scores vanish in sweep 2
-      if (g_row < P.n && m > -INFINITY) {
-        const float l = row_l * fast_exp2(row_m - m) + l1 * fast_exp2(m1 - m);
-        lse = m + log2f(l);
+      // merge the groups' (reference, sum) pairs; a sum of 0 marks a group that had no tile
+      float m = row_m, l = row_l;
+#pragma unroll
+      for (int g = 1; g < NG; ++g) {
+        const float m1 = comb[(g - 1) * 256 + row], l1 = comb[(g - 1) * 256 + 128 + row];
+        if (l1 > 0.f) {
+          if (l > 0.f) {
+            const float mm = fmaxf(m, m1);
+            l = l * fast_exp2(m - mm) + l1 * fast_exp2(m1 - mm);
+            m = mm;
+          } else {
+            m = m1; l = l1;
+          }
+        }
       }
-      P.lse2[(size_t)u * nblk * TC_BN + g_row] = lse;
+      // rows past the prompt get +inf: their scores vanish in sweep 2
+      P.lse2[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? m + log2f(l) : INFINITY;
     } else if (g_row < P.n) {
-      P.acc_full[(size_t)u * P.n + g_row] = col_sum + comb[row];
+      float total = col_sum;
+#pragma unroll
+      for (int g = 1; g < NG; ++g) total += comb[(g - 1) * 256 + row];
+      P.acc_full[(size_t)u * P.n + g_row] = total;
     }
   }
 
@@ -450,25 +513,26 @@ bool make_operand_map(CUtensorMap* map, const __half* base, int units, int n, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, int NST>
+template <int D, int NST, int NG>
 constexpr size_t tc_smem_bytes() {
-  size_t b = 1024 + (size_t)(1 + NST) * TC_BM * D * 2 + (size_t)TC_NCW * TC_XBUF_FLOATS * 4 + (size_t)TC_NCW * 2 * 128 * 4 +
-             2 * 128 * 4 + 32 * 8 + 64;
+  size_t b = 1024 + (size_t)(1 + NST) * TC_BM * D * 2 + (size_t)4 * NG * TC_XBUF_FLOATS * 4 + (size_t)4 * NG * 128 * 4 +
+             (size_t)(NG - 1) * 2 * 128 * 4 + 32 * 8 + 64;
   return b < 120 * 1024 ? 120 * 1024 : b;   // one CTA per SM: each takes all of tensor memory
 }
 
-template <int D, int NST, bool SWEEP2>
+template <int D, int NST, int NG, bool SWEEP2>
 cudaError_t launch_variant(const PrefillTcParams& P, int units, bool noise, bool alibi, cudaStream_t st) {
-  constexpr size_t smem = tc_smem_bytes<D, NST>();
+  constexpr size_t smem = tc_smem_bytes<D, NST, NG>();
+  static_assert(smem <= 227 * 1024, "shared memory budget of one CTA");
   dim3 grid((unsigned)P.nblk, (unsigned)units);
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, TC_THREADS, smem, st>>>(P);
+    kern<<<grid, tc_threads(NG), smem, st>>>(P);
     return cudaGetLastError();
   };
-  if (noise) return alibi ? go(prefill_tc<D, NST, SWEEP2, true, true>) : go(prefill_tc<D, NST, SWEEP2, true, false>);
-  return alibi ? go(prefill_tc<D, NST, SWEEP2, false, true>) : go(prefill_tc<D, NST, SWEEP2, false, false>);
+  if (noise) return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, true, true>) : go(prefill_tc<D, NST, NG, SWEEP2, true, false>);
+  return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, false, true>) : go(prefill_tc<D, NST, NG, SWEEP2, false, false>);
 }
 
 }  // namespace
@@ -495,16 +559,16 @@ cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int un
   cudaError_t e;
   switch (head_dim) {
     case 64:
-      e = launch_variant<64, 4, false>(P, units, noise, alibi, stream);
-      if (e == cudaSuccess) e = launch_variant<64, 4, true>(P, units, noise, alibi, stream);
+      e = launch_variant<64, 4, TC_NG, false>(P, units, noise, alibi, stream);
+      if (e == cudaSuccess) e = launch_variant<64, 4, TC_NG, true>(P, units, noise, alibi, stream);
       return e;
     case 128:
-      e = launch_variant<128, 3, false>(P, units, noise, alibi, stream);
-      if (e == cudaSuccess) e = launch_variant<128, 3, true>(P, units, noise, alibi, stream);
+      e = launch_variant<128, 3, TC_NG, false>(P, units, noise, alibi, stream);
+      if (e == cudaSuccess) e = launch_variant<128, 3, TC_NG, true>(P, units, noise, alibi, stream);
       return e;
     case 256:
-      e = launch_variant<256, 2, false>(P, units, noise, alibi, stream);
-      if (e == cudaSuccess) e = launch_variant<256, 2, true>(P, units, noise, alibi, stream);
+      e = launch_variant<256, 2, 2, false>(P, units, noise, alibi, stream);
+      if (e == cudaSuccess) e = launch_variant<256, 2, 2, true>(P, units, noise, alibi, stream);
       return e;
     default:
       return cudaErrorInvalidValue;

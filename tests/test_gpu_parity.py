@@ -34,6 +34,14 @@ def test_prompt_lengths_around_tile_edges(n, noise):
     lockstep.run_workload(wl, noise=noise)
 
 
+@pytest.mark.parametrize("scale", [2.0, 16.0])
+def test_prompt_scores_with_extreme_logits(scale):
+    """Logits hundreds of units apart (a scale far above 1/sqrt(d)): the prompt softmax must not overflow,
+    and rows dominated by a single key must still match the oracle."""
+    wl = _wl(head_dim=64, prompt_len=400, budget_k=150, recent_w=20, gen_len_T=2)
+    lockstep.run_workload(wl, logit_scale=scale)
+
+
 def test_prompt_scores_tensor_core_vs_cuda_core():
     """The two scoring implementations agree far inside the oracle tolerance, and the tensor-core
     one is reproducible bit for bit (no atomics)."""
