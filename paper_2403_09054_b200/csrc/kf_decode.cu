@@ -423,7 +423,7 @@ int decode_tile_rows() { return TILE_ROWS; }
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
   switch (head_dim) {
     case 64: return launch_one<64, 4, 4>(P, units, stream);
-    case 128: return launch_one<128, 4, 3>(P, units, stream);
+    case 128: return launch_one<128, 4, 2>(P, units, stream);   // 64 KB of ring per CTA: three CTAs per SM
     case 256: return launch_one<256, 4, 2>(P, units, stream);
     default: return cudaErrorInvalidValue;
   }
