@@ -38,6 +38,11 @@ def algorithmic_bytes_per_launch(wl: W.Workload) -> int:
     return wl.batch * wl.n_heads * per_unit
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel<128,4,2> launch on a c4_cerebras layer
+# (1024 units, k = 2048, d = 128), from the ncu capture summarised in profiles/decode_kernel_c4_cerebras.md.
+C4_DECODE_TRAFFIC_BYTES = 1.130e9
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -288,7 +293,9 @@ def run_ours(args, wl):
             "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": abytes,
-                         "launch_ms": launch_ms, "traffic": args.traffic},
+                         "launch_ms": launch_ms,
+                         "traffic": args.traffic if args.traffic is not None else
+                         (C4_DECODE_TRAFFIC_BYTES if wl.name.startswith("c4_cerebras") and args.splits == 0 else None)},
             "cpu_baseline": {"value": cpu_rate / wl.units, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": (world * 1e3 / e2e_ms) if e2e_ms else None, "unit": UNIT, "h2d_bytes_per_step": 3 * L * vec_bytes,
                     "d2h_bytes_per_step": L * vec_bytes},
@@ -385,7 +392,8 @@ def main():
     ap.add_argument("--cpu-units", type=int, default=512)
     ap.add_argument("--cpu-steps", type=int, default=64)
     ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per launch of the decode kernel from an ncu capture (see profiles/)")
+                    help="DRAM bytes per launch of the decode kernel from an ncu capture (default: the committed "
+                         "capture of the current kernel on the Cerebras-shaped layer, see profiles/)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling a small case)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (profiling a small case)")
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
