@@ -45,6 +45,8 @@ extern "C" {
 #define KF_NOISE_GUMBEL 0   /* zeta = -ln(-ln u), standard Gumbel, Eq. 7 (the method) */
 #define KF_NOISE_NONE   1   /* zeta = 0 (accumulated-attention score, H2O-like)      */
 #define KF_NOISE_CONST  2   /* zeta = noise_const                                     */
+#define KF_NOISE_GAUSS  3   /* zeta = noise_mu + noise_sigma * N(0,1) (the Gaussian alternative of section 4.4.3;
+                               Box-Muller on two Philox words)                        */
 
 /* How kf_prefill_score_prune computes the prompt logits Q K^T. */
 #define KF_PREFILL_TENSOR 0 /* tcgen05 tensor cores, accumulators in tensor memory (default) */
@@ -76,6 +78,8 @@ typedef struct kf_config {
   float   noise_const;     /* c of KF_NOISE_CONST                                 */
   int32_t decode_splits;   /* 0 = choose automatically; else CTAs per unit in the decode kernel */
   int32_t prefill_impl;    /* KF_PREFILL_*                                        */
+  float   noise_mu;        /* mean of KF_NOISE_GAUSS (the paper matches Gumbel's 0.5772)          */
+  float   noise_sigma;     /* standard deviation of KF_NOISE_GAUSS (1.2825 in the paper)         */
 } kf_config;
 
 /* Bytes of device workspace kf_create needs for this configuration

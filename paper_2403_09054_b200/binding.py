@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 KF_OK, KF_EINVAL, KF_ENOSPC, KF_ESTATE, KF_ECUDA, KF_ETIMEOUT, KF_EBOUNDS = 0, -1, -2, -3, -4, -5, -6
-KF_NOISE_GUMBEL, KF_NOISE_NONE, KF_NOISE_CONST = 0, 1, 2
+KF_NOISE_GUMBEL, KF_NOISE_NONE, KF_NOISE_CONST, KF_NOISE_GAUSS = 0, 1, 2, 3
 KF_BIAS_NONE, KF_BIAS_ALIBI = 0, 1
 KF_PREFILL_TENSOR, KF_PREFILL_SIMT = 0, 1
 
@@ -32,6 +32,7 @@ class kf_config(C.Structure):
         ("noise_mode", C.c_int32), ("bias_mode", C.c_int32), ("h_alibi_slopes", C.POINTER(C.c_float)),
         ("logit_scale", C.c_float), ("noise_const", C.c_float),
         ("decode_splits", C.c_int32), ("prefill_impl", C.c_int32),
+        ("noise_mu", C.c_float), ("noise_sigma", C.c_float),
     ]
 
 
@@ -102,7 +103,7 @@ def kf_strerror(code: int) -> str:
 def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_prompt_len, gen_len_T,
                 tau_init=1.0, tau_end=2.0, noise_seed=0, noise_mode=KF_NOISE_GUMBEL, bias_mode=KF_BIAS_NONE,
                 alibi_slopes=None, logit_scale=0.0, noise_const=0.5772, decode_splits=0,
-                prefill_impl=KF_PREFILL_TENSOR):
+                prefill_impl=KF_PREFILL_TENSOR, noise_mu=0.5772, noise_sigma=1.2825):
     """Fill a kf_config; returns (config, keepalive) where keepalive holds the slopes array."""
     cfg = kf_config()
     cfg.n_layers, cfg.batch, cfg.n_heads, cfg.head_dim = n_layers, batch, n_heads, head_dim
@@ -116,6 +117,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
         cfg.h_alibi_slopes = keep.ctypes.data_as(C.POINTER(C.c_float))
     cfg.logit_scale, cfg.noise_const = logit_scale, noise_const
     cfg.decode_splits, cfg.prefill_impl = decode_splits, prefill_impl
+    cfg.noise_mu, cfg.noise_sigma = noise_mu, noise_sigma
     return cfg, keep
 
 

@@ -32,7 +32,8 @@ bool config_ok(const kf_config* c) {
   if (c->budget_k < 1 || c->recent_w < 0 || c->recent_w > c->budget_k) return false;
   if (c->max_prompt_len < 1 || c->gen_len_T < 0) return false;
   if (!(c->tau_init > 0.f) || !(c->tau_end > 0.f)) return false;
-  if (c->noise_mode < KF_NOISE_GUMBEL || c->noise_mode > KF_NOISE_CONST) return false;
+  if (c->noise_mode < KF_NOISE_GUMBEL || c->noise_mode > KF_NOISE_GAUSS) return false;
+  if (c->noise_mode == KF_NOISE_GAUSS && !(c->noise_sigma >= 0.f)) return false;
   if (c->bias_mode != KF_BIAS_NONE && c->bias_mode != KF_BIAS_ALIBI) return false;
   if (c->bias_mode == KF_BIAS_ALIBI && !c->h_alibi_slopes) return false;
   if (c->logit_scale < 0.f || c->decode_splits < 0) return false;
@@ -146,6 +147,7 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
     A.err = err;
     A.n = n_prompt; A.H = c.n_heads; A.layer = layer; A.noise_mode = c.noise_mode; A.bias_mode = c.bias_mode;
     A.scale = ctx->scale; A.inv_tau = inv_tau; A.noise_const = c.noise_const;
+    A.noise_mu = c.noise_mu; A.noise_sigma = c.noise_sigma;
     A.pk = ctx->pk;
     if (kf::launch_prefill_score_tc(A, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
     ctx->launches += 2;
@@ -161,6 +163,7 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
     P.scale = ctx->scale;
     P.inv_tau = inv_tau;
     P.noise_const = c.noise_const;
+    P.noise_mu = c.noise_mu; P.noise_sigma = c.noise_sigma;
     P.pk = ctx->pk;
     if (kf::launch_prefill_score_simt(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
     ctx->launches += 1;
@@ -237,6 +240,7 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   }
   P.inv_tau = (float)(1.0 / tau);
   P.noise_const = c.noise_const;
+  P.noise_mu = c.noise_mu; P.noise_sigma = c.noise_sigma;
   P.pk = ctx->pk;
   if (kf::launch_decode(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
   ctx->launches += 1;

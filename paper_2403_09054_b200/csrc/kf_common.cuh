@@ -80,6 +80,16 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t r) {
   return -LN2 * __log2f(neg_log_uniform(uniform_from_word(r)));
 }
 
+// Standard normal variate by the Box-Muller transform: radius from word a, angle from word b.
+// cos(2 pi u) is evaluated as -cos(2 pi (u - 1/2)) so that the fast cosine sees an angle inside (-pi, pi).
+__device__ __forceinline__ float gauss_from_words(uint32_t ra, uint32_t rb) {
+  const float radius = sqrtf(2.0f * neg_log_uniform(uniform_from_word(ra)));
+  const float angle = 6.2831853071795865f * (uniform_from_word(rb) - 0.5f);
+  return -radius * __cosf(angle);
+}
+// The second word of the Gaussian adjustment comes from a separate counter plane: bit 31 of the batch word.
+constexpr uint32_t GAUSS_PLANE = 0x80000000u;
+
 // ------------------------------------------------------------------ warp reductions
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll

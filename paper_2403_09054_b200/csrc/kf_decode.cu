@@ -33,6 +33,8 @@ __device__ __forceinline__ void axpy8(float (&o)[8], float a, const uint4& vv) {
 __device__ __forceinline__ float noise_for(const DecodeParams& P, uint32_t b, uint32_t lh, uint32_t i, uint32_t j) {
   if (P.noise_mode == 0) return gumbel_from_word(noise_word(P.pk, b, lh, i, j));
   if (P.noise_mode == 2) return P.noise_const;
+  if (P.noise_mode == 3)
+    return fmaf(P.noise_sigma, gauss_from_words(noise_word(P.pk, b, lh, i, j), noise_word(P.pk, b | GAUSS_PLANE, lh, i, j)), P.noise_mu);
   return 0.f;
 }
 

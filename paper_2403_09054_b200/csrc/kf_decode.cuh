@@ -24,7 +24,7 @@ struct DecodeParams {
   int32_t k, w, p;        // budget, recent window, position of the query token
   int32_t splits, tiles_per_split;
   int32_t H, layer, noise_mode, bias_mode;
-  float scale, inv_tau, noise_const;
+  float scale, inv_tau, noise_const, noise_mu, noise_sigma;
   PhiloxKeys pk;
 };
 

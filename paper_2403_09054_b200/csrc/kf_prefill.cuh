@@ -14,7 +14,7 @@ struct PrefillParams {
   const float* slopes; // [H] or null
   int* err;
   int32_t n, H, layer, noise_mode, bias_mode;
-  float scale, inv_tau, noise_const;
+  float scale, inv_tau, noise_const, noise_mu, noise_sigma;
   PhiloxKeys pk;
 };
 
@@ -51,6 +51,7 @@ struct PrefillTcParams {
   float c1;            // log2(e) / tau
   float inv_tau;
   float const_term;    // constant logit adjustment in the scaled log2 domain (0 without one)
+  float gauss_scale;   // noise_sigma * log2(e) / tau (Gaussian adjustment)
   PhiloxKeys pk;
 };
 
@@ -63,7 +64,7 @@ struct PrefillTcArgs {
   const float* slopes;
   int* err;
   int32_t n, H, layer, noise_mode, bias_mode;
-  float scale, inv_tau, noise_const;
+  float scale, inv_tau, noise_const, noise_mu, noise_sigma;
   PhiloxKeys pk;
 };
 

@@ -15,6 +15,8 @@ constexpr int NTH = 256; // 16 x 16 threads, 4 x 4 logits each
 __device__ __forceinline__ float prefill_noise(const PrefillParams& P, uint32_t b, uint32_t lh, uint32_t i, uint32_t j) {
   if (P.noise_mode == 0) return gumbel_from_word(noise_word(P.pk, b, lh, i, j));
   if (P.noise_mode == 2) return P.noise_const;
+  if (P.noise_mode == 3)
+    return fmaf(P.noise_sigma, gauss_from_words(noise_word(P.pk, b, lh, i, j), noise_word(P.pk, b | GAUSS_PLANE, lh, i, j)), P.noise_mu);
   return 0.f;
 }
 

@@ -147,19 +147,32 @@ __device__ __forceinline__ float neg_lg2_uniform(float u) {
 // The four noise terms of one Philox call in the scaled log2 domain:
 //   zeta * log2(e) / tau = -(log2(-log2 u) + log2 ln 2) / tau     with zeta = -ln(-ln u)   (Eq. 7)
 // `offset` carries -log2(ln 2) / tau plus whatever the caller wants added to all four logits.
+// MODE 1 (Gumbel): `mult` = -1 / tau.  MODE 2 (Gaussian alternative of section 4.4.3): the four terms are
+// sigma * N(0,1) * log2(e) / tau with `mult` = sigma * log2(e) / tau and the mean inside `offset`; the angle words
+// come from the counter plane with bit 31 of the batch word set.
+constexpr int NOISE_OFF = 0, NOISE_GUMBEL_T = 1, NOISE_GAUSS_T = 2;
+template <int MODE>
 __device__ __forceinline__ float4 noise_terms(const PhiloxKeys& pk, uint32_t jgroup, uint32_t i, uint32_t lh, uint32_t b,
-                                              float neg_inv_tau, float offset) {
+                                              float mult, float offset) {
   const uint4 r = philox4x32_10(jgroup, i, lh, b, pk);
   float4 t;
-  t.x = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.x))), neg_inv_tau, offset);
-  t.y = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.y))), neg_inv_tau, offset);
-  t.z = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.z))), neg_inv_tau, offset);
-  t.w = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.w))), neg_inv_tau, offset);
+  if (MODE == NOISE_GAUSS_T) {
+    const uint4 a = philox4x32_10(jgroup, i, lh, b | GAUSS_PLANE, pk);
+    t.x = fmaf(gauss_from_words(r.x, a.x), mult, offset);
+    t.y = fmaf(gauss_from_words(r.y, a.y), mult, offset);
+    t.z = fmaf(gauss_from_words(r.z, a.z), mult, offset);
+    t.w = fmaf(gauss_from_words(r.w, a.w), mult, offset);
+  } else {
+    t.x = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.x))), mult, offset);
+    t.y = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.y))), mult, offset);
+    t.z = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.z))), mult, offset);
+    t.w = fmaf(fast_lg2(neg_lg2_uniform(uniform_from_word_bits(r.w))), mult, offset);
+  }
   return t;
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int D, int NST, int NG, bool SWEEP2, bool NOISE, bool ALIBI>
+template <int D, int NST, int NG, bool SWEEP2, int NOISE, bool ALIBI>
 __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_constant__ PrefillTcParams P) {
   constexpr int OP_BYTES = TC_BM * D * 2;  // one operand block: D / 64 boxes
   constexpr int KCH = D / 64;              // 64-column boxes per operand row
@@ -270,8 +283,8 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
     const int g_row = Rb * TC_BM + row;                // query i (sweep 1) or key j (sweep 2)
     const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
     const float A = P.a_scale;
-    const float neg_inv_tau = -P.inv_tau;
-    const float n_off = NOISE ? neg_inv_tau * LG2_LN2 : P.const_term;   // additive term common to all logits
+    const float n_mult = NOISE == NOISE_GAUSS_T ? P.gauss_scale : -P.inv_tau;
+    const float n_off = NOISE == NOISE_GUMBEL_T ? -P.inv_tau * LG2_LN2 : P.const_term;   // additive term common to all logits
     float sb = 0.f;
     if (ALIBI) sb = P.slopes[h] * P.c1;
     float* my_x = xbuf + cw * TC_XBUF_FLOATS;
@@ -331,7 +344,7 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
 #pragma unroll
             for (int g = 0; g < 8; ++g) {
               float4 nz = make_float4(off, off, off, off);
-              if (NOISE) nz = noise_terms(P.pk, (uint32_t)(col0 >> 2) + g, (uint32_t)g_row, lh, b, neg_inv_tau, off);
+              if (NOISE) nz = noise_terms<NOISE>(P.pk, (uint32_t)(col0 >> 2) + g, (uint32_t)g_row, lh, b, n_mult, off);
               const float nn[4] = {nz.x, nz.y, nz.z, nz.w};
               float a4[4];
 #pragma unroll
@@ -385,7 +398,7 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
                 const int ql = half * 16 + 4 * g + (lane >> 3);
                 const uint32_t jg = (uint32_t)((Rb * TC_BM + quarter * 32) >> 2) + (uint32_t)(lane & 7);
                 reinterpret_cast<float4*>(my_x)[g * 32 + lane] =
-                    noise_terms(P.pk, jg, (uint32_t)(col0 + ql), lh, b, neg_inv_tau, n_off - lse_t[ql]);
+                    noise_terms<NOISE>(P.pk, jg, (uint32_t)(col0 + ql), lh, b, n_mult, n_off - lse_t[ql]);
               }
               __syncwarp();
 #pragma unroll
@@ -521,7 +534,7 @@ constexpr size_t tc_smem_bytes() {
 }
 
 template <int D, int NST, int NG, bool SWEEP2>
-cudaError_t launch_variant(const PrefillTcParams& P, int units, bool noise, bool alibi, cudaStream_t st) {
+cudaError_t launch_variant(const PrefillTcParams& P, int units, int noise, bool alibi, cudaStream_t st) {
   constexpr size_t smem = tc_smem_bytes<D, NST, NG>();
   static_assert(smem <= 227 * 1024, "shared memory budget of one CTA");
   dim3 grid((unsigned)P.nblk, (unsigned)units);
@@ -531,8 +544,11 @@ cudaError_t launch_variant(const PrefillTcParams& P, int units, bool noise, bool
     kern<<<grid, tc_threads(NG), smem, st>>>(P);
     return cudaGetLastError();
   };
-  if (noise) return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, true, true>) : go(prefill_tc<D, NST, NG, SWEEP2, true, false>);
-  return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, false, true>) : go(prefill_tc<D, NST, NG, SWEEP2, false, false>);
+  if (noise == NOISE_GUMBEL_T)
+    return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GUMBEL_T, true>) : go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GUMBEL_T, false>);
+  if (noise == NOISE_GAUSS_T)
+    return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GAUSS_T, true>) : go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GAUSS_T, false>);
+  return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, NOISE_OFF, true>) : go(prefill_tc<D, NST, NG, SWEEP2, NOISE_OFF, false>);
 }
 
 }  // namespace
@@ -553,9 +569,11 @@ cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int un
   P.inv_tau = a.inv_tau;
   P.c1 = LOG2E * a.inv_tau;
   P.a_scale = a.scale * P.c1;
-  P.const_term = a.noise_mode == 2 ? a.noise_const * P.c1 : 0.f;
+  P.const_term = a.noise_mode == 2 ? a.noise_const * P.c1 : (a.noise_mode == 3 ? a.noise_mu * P.c1 : 0.f);
+  P.gauss_scale = a.noise_sigma * P.c1;
   P.pk = a.pk;
-  const bool noise = a.noise_mode == 0, alibi = a.bias_mode == 1 && a.slopes != nullptr;
+  const int noise = a.noise_mode == 0 ? NOISE_GUMBEL_T : (a.noise_mode == 3 ? NOISE_GAUSS_T : NOISE_OFF);
+  const bool alibi = a.bias_mode == 1 && a.slopes != nullptr;
   cudaError_t e;
   switch (head_dim) {
     case 64:

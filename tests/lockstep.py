@@ -202,8 +202,8 @@ def run_workload(wl: W.Workload, units_per_layer=None, steps=None, layers=None, 
                  sample_seed=0, check_state_every=1, gpu_kwargs=None, noise="gumbel", logit_scale=0.0):
     """Prefill + `steps` decode steps of `wl` on the GPU in lock step with the oracle.
     Returns a dict of summary numbers."""
-    nm_gpu = {"gumbel": kf.KF_NOISE_GUMBEL, "none": kf.KF_NOISE_NONE, "const": kf.KF_NOISE_CONST}[noise]
-    nm_ref = {"gumbel": ko.NOISE_GUMBEL, "none": ko.NOISE_NONE, "const": ko.NOISE_CONST}[noise]
+    nm_gpu = {"gumbel": kf.KF_NOISE_GUMBEL, "none": kf.KF_NOISE_NONE, "const": kf.KF_NOISE_CONST, "gauss": kf.KF_NOISE_GAUSS}[noise]
+    nm_ref = {"gumbel": ko.NOISE_GUMBEL, "none": ko.NOISE_NONE, "const": ko.NOISE_CONST, "gauss": ko.NOISE_GAUSS}[noise]
     gpu = make_gpu(wl, noise_mode=nm_gpu, logit_scale=logit_scale, **(gpu_kwargs or {}))
     layers = list(range(wl.n_layers)) if layers is None else layers
     steps = wl.gen_len_T if steps is None else steps

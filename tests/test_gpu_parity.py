@@ -72,9 +72,11 @@ def test_split_counts(splits):
     lockstep.run_workload(wl, gpu_kwargs=dict(decode_splits=splits))
 
 
-@pytest.mark.parametrize("noise", ["none", "const"])
-def test_other_adjustments(noise):
-    lockstep.run_workload(_wl(head_dim=128), noise=noise)
+@pytest.mark.parametrize("impl", [kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_SIMT])
+@pytest.mark.parametrize("noise", ["none", "const", "gauss"])
+def test_other_adjustments(noise, impl):
+    lockstep.run_workload(_wl(head_dim=128, prompt_len=300, budget_k=120, recent_w=30), noise=noise,
+                          gpu_kwargs=dict(prefill_impl=impl))
 
 
 def test_zero_noise_tau_one_scores_are_attention_weights():
