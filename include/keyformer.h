@@ -190,6 +190,20 @@ int kf_decode_step_static(const kf_static_step* args,
 int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V,
                   const int32_t** d_pos, const float** d_acc, const int32_t** d_len);
 
+/* Checkpoint of one layer's cache (section 3.3: the reduced KV cache and f_theta are the whole state the
+ * method carries from step to step).  kf_state_bytes gives the size of one layer's image: K, V, f_theta,
+ * positions and entry counts, each block padded to 256 bytes, in that order.  kf_export_state copies the
+ * image to a caller-owned DEVICE buffer and reports how far the layer has come (prompt length, last decode
+ * step); kf_import_state loads an image into a context created with the same configuration and sets that
+ * progress, after which kf_decode_step continues with step last_step + 1 and reproduces the original run
+ * bit for bit (noise and temperature are functions of the coordinates, not of hidden state).  Both are
+ * enqueued on `stream`.  KF_ESTATE if the layer has no prompt yet; KF_ENOSPC if `bytes` is too small. */
+size_t kf_state_bytes(const kf_ctx* ctx);
+int kf_export_state(kf_ctx* ctx, int32_t layer, void* d_dst, size_t bytes,
+                    int32_t* n_prompt, int32_t* last_step, void* stream);
+int kf_import_state(kf_ctx* ctx, int32_t layer, const void* d_src, size_t bytes,
+                    int32_t n_prompt, int32_t last_step, void* stream);
+
 /* Waits for `stream`, then returns and clears the device error word:
  * 0, KF_ETIMEOUT or KF_EBOUNDS. */
 int kf_poll_error(kf_ctx* ctx, void* stream);

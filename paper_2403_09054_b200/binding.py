@@ -21,7 +21,7 @@ KF_PREFILL_TENSOR, KF_PREFILL_SIMT = 0, 1
 
 EXPORTS = ("kf_workspace_bytes", "kf_create", "kf_prefill_score_prune", "kf_decode_step",
            "kf_decode_step_host", "kf_view_state", "kf_poll_error", "kf_launch_count",
-           "kf_destroy", "kf_strerror", "kf_decode_step_static")
+           "kf_destroy", "kf_strerror", "kf_decode_step_static", "kf_state_bytes", "kf_export_state", "kf_import_state")
 
 
 class kf_config(C.Structure):
@@ -68,6 +68,12 @@ def _load() -> C.CDLL:
     lib.kf_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32, vp]
     lib.kf_decode_step_static.restype = C.c_int
     lib.kf_decode_step_static.argtypes = [C.POINTER(kf_static_step)] + [vp] * 11
+    lib.kf_state_bytes.restype = C.c_size_t
+    lib.kf_state_bytes.argtypes = [vp]
+    lib.kf_export_state.restype = C.c_int
+    lib.kf_export_state.argtypes = [vp, i32, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32), vp]
+    lib.kf_import_state.restype = C.c_int
+    lib.kf_import_state.argtypes = [vp, i32, vp, C.c_size_t, i32, i32, vp]
     lib.kf_view_state.restype = C.c_int
     lib.kf_view_state.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
     lib.kf_poll_error.restype = C.c_int
@@ -228,6 +234,20 @@ class Keyformer:
         acc = view(ptrs[3], B * H * k * 4, torch.float32, (B, H, k))
         ln = view(ptrs[4], B * H * 4, torch.int32, (B, H))
         return K, V, pos, acc, ln
+
+    def kf_state_bytes(self) -> int:
+        return int(LIB.kf_state_bytes(self._h))
+
+    def kf_export_state(self, layer, image, stream=None):
+        """Copy one layer's cache image into the uint8 CUDA tensor `image`; returns (n_prompt, last_step)."""
+        n_prompt, last_step = C.c_int32(), C.c_int32()
+        _check(LIB.kf_export_state(self._h, layer, _dev_ptr(image, torch.uint8, image.numel(), "image"), image.numel(),
+                                   C.byref(n_prompt), C.byref(last_step), _stream_ptr(stream)), "kf_export_state")
+        return n_prompt.value, last_step.value
+
+    def kf_import_state(self, layer, image, n_prompt, last_step, stream=None):
+        _check(LIB.kf_import_state(self._h, layer, _dev_ptr(image, torch.uint8, image.numel(), "image"), image.numel(),
+                                   n_prompt, last_step, _stream_ptr(stream)), "kf_import_state")
 
     def kf_poll_error(self, stream=None) -> int:
         return int(LIB.kf_poll_error(self._h, _stream_ptr(stream)))

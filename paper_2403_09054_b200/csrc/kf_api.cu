@@ -346,6 +346,54 @@ int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V
   return KF_OK;
 }
 
+size_t kf_state_bytes(const kf_ctx* ctx) {
+  if (!ctx) return 0;
+  const Layout& L = ctx->lay;
+  return 2 * L.kv_layer + 2 * L.sc_layer + L.len_layer;
+}
+
+// One layer's image: K | V | acc | pos | len, the workspace's own per-layer blocks back to back.
+static int copy_state(kf_ctx* ctx, int32_t layer, unsigned char* image, bool to_image, cudaStream_t st) {
+  const Layout& L = ctx->lay;
+  struct Block { size_t ws_off, bytes; };
+  const Block blocks[5] = {{L.K + (size_t)layer * L.kv_layer, L.kv_layer},   {L.V + (size_t)layer * L.kv_layer, L.kv_layer},
+                           {L.acc + (size_t)layer * L.sc_layer, L.sc_layer}, {L.pos + (size_t)layer * L.sc_layer, L.sc_layer},
+                           {L.len + (size_t)layer * L.len_layer, L.len_layer}};
+  size_t off = 0;
+  for (const Block& b : blocks) {
+    void* dst = to_image ? (void*)(image + off) : (void*)(ctx->ws + b.ws_off);
+    const void* src = to_image ? (const void*)(ctx->ws + b.ws_off) : (const void*)(image + off);
+    if (cudaMemcpyAsync(dst, src, b.bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return KF_ECUDA;
+    off += b.bytes;
+  }
+  return KF_OK;
+}
+
+int kf_export_state(kf_ctx* ctx, int32_t layer, void* d_dst, size_t bytes, int32_t* n_prompt, int32_t* last_step,
+                    void* stream) {
+  if (!ctx || !d_dst || layer < 0 || layer >= ctx->cfg.n_layers) return KF_EINVAL;
+  if (ctx->n_prompt[layer] < 0) return KF_ESTATE;
+  if (bytes < kf_state_bytes(ctx)) return KF_ENOSPC;
+  const int rc = copy_state(ctx, layer, static_cast<unsigned char*>(d_dst), true, static_cast<cudaStream_t>(stream));
+  if (rc != KF_OK) return rc;
+  if (n_prompt) *n_prompt = ctx->n_prompt[layer];
+  if (last_step) *last_step = ctx->last_step[layer];
+  return KF_OK;
+}
+
+int kf_import_state(kf_ctx* ctx, int32_t layer, const void* d_src, size_t bytes, int32_t n_prompt, int32_t last_step,
+                    void* stream) {
+  if (!ctx || !d_src || layer < 0 || layer >= ctx->cfg.n_layers) return KF_EINVAL;
+  if (n_prompt < 1 || last_step < 0) return KF_EINVAL;
+  if (bytes < kf_state_bytes(ctx)) return KF_ENOSPC;
+  const int rc = copy_state(ctx, layer, const_cast<unsigned char*>(static_cast<const unsigned char*>(d_src)), false,
+                            static_cast<cudaStream_t>(stream));
+  if (rc != KF_OK) return rc;
+  ctx->n_prompt[layer] = n_prompt;
+  ctx->last_step[layer] = last_step;
+  return KF_OK;
+}
+
 int kf_poll_error(kf_ctx* ctx, void* stream) {
   if (!ctx) return KF_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

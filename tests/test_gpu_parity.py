@@ -134,6 +134,47 @@ def test_call_order_and_argument_errors():
     assert gpu.kf_launch_count() == 5   # prompt phase: 2 scoring sweeps + select + gather; then 1 decode kernel
 
 
+def test_export_import_state_resumes_bit_exactly():
+    wl = _wl(head_dim=128, n_layers=2, prompt_len=130, budget_k=64, recent_w=16, gen_len_T=10)
+    a = lockstep.make_gpu(wl)
+    for l in range(2):
+        a.kf_prefill_score_prune(l, *W.make_prompt(wl, l, DEV))
+    outs = {}
+
+    def step(gpu, l, s):
+        q, kn, vn = W.make_step(wl, l, s, DEV)
+        out = torch.empty_like(q)
+        gpu.kf_decode_step(l, s, q, kn, vn, out)
+        return out
+
+    for s in range(1, 4):
+        for l in range(2):
+            step(a, l, s)
+    images = []
+    for l in range(2):
+        img = torch.empty(a.kf_state_bytes(), dtype=torch.uint8, device=DEV)
+        images.append((img, a.kf_export_state(l, img)))
+    assert images[0][1] == (130, 3)
+    for s in range(4, 8):
+        for l in range(2):
+            outs[(l, s)] = step(a, l, s)
+    b = lockstep.make_gpu(wl)            # a fresh context continues from the images
+    with pytest.raises(kf.KeyformerError) as e:
+        b.kf_export_state(0, images[0][0])
+    assert e.value.code == kf.KF_ESTATE
+    for l in range(2):
+        img, (n_prompt, last_step) = images[l]
+        b.kf_import_state(l, img, n_prompt, last_step)
+    for s in range(4, 8):
+        for l in range(2):
+            assert torch.equal(step(b, l, s), outs[(l, s)])
+    torch.cuda.synchronize()
+    for l in range(2):
+        for x, y in zip(a.kf_view_state(l), b.kf_view_state(l)):
+            assert torch.equal(x, y)
+    assert a.kf_poll_error() == 0 and b.kf_poll_error() == 0
+
+
 def test_host_buffer_variant_matches_device_variant():
     wl = _wl(head_dim=128)
     a, b = lockstep.make_gpu(wl), lockstep.make_gpu(wl)
