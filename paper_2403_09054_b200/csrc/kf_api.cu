@@ -36,7 +36,7 @@ bool config_ok(const kf_config* c) {
   if (c->noise_mode == KF_NOISE_GAUSS && !(c->noise_sigma >= 0.f)) return false;
   if (c->bias_mode != KF_BIAS_NONE && c->bias_mode != KF_BIAS_ALIBI) return false;
   if (c->bias_mode == KF_BIAS_ALIBI && !c->h_alibi_slopes) return false;
-  if (c->logit_scale < 0.f || c->decode_splits < 0) return false;
+  if (c->logit_scale < 0.f || c->decode_splits < 0 || c->decode_splits > kf::decode_max_splits()) return false;
   if (c->prefill_impl != KF_PREFILL_TENSOR && c->prefill_impl != KF_PREFILL_SIMT) return false;
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
   return true;
@@ -49,8 +49,7 @@ Layout make_layout(const kf_config* c) {
   const size_t units = (size_t)c->batch * c->n_heads;
   const size_t k = (size_t)c->budget_k, d = (size_t)c->head_dim, nl = (size_t)c->n_layers;
   L.units = (int)units;
-  L.max_splits = std::max(1, std::min(64, (tiles_of(c->budget_k) + 3) / 4));
-  if (c->decode_splits > 0) L.max_splits = std::max(L.max_splits, (int)c->decode_splits);
+  L.max_splits = kf::decode_max_splits();
   L.kv_layer = align_up(units * k * d * 2);
   L.sc_layer = align_up(units * k * 4);
   L.len_layer = align_up(units * 4);

@@ -19,6 +19,7 @@ namespace kf {
 namespace {
 
 constexpr int TILE_ROWS = 32;
+constexpr int MAX_SPLITS = 64;   // CTAs per unit (the closing CTA keeps one weight per split in shared memory)
 
 __device__ __forceinline__ void axpy8(float (&o)[8], float a, const uint4& vv) {
   const __half2* h = reinterpret_cast<const __half2*>(&vv);
@@ -47,6 +48,7 @@ __device__ __forceinline__ unsigned long long evict_key(float a, int pos) {
 template <int D, int NT>
 __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   __shared__ float sh_scalar[8];
+  __shared__ float sh_scale[MAX_SPLITS];   // 2^(m_s - m) of every split's attention partial (0 for an empty split)
   __shared__ unsigned long long sh_key[NT / 32];
   __shared__ int sh_victim;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -62,21 +64,30 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
     float s = 0.f;
     for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[c]), __half2float(kn[c]), s);
     s = warp_sum(s);
+    const float x_new = s * P.scale;  // bias(p, p) = 0
+    float y_new = 0.f;
+    if (lane == 0) y_new = (x_new + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
+    y_new = __shfl_sync(0xffffffffu, y_new, 0);
+    // merge the splits' (max, sum) pairs of both softmaxes, one split per lane
+    float mx = x_new, my = y_new;
+    for (int sp = lane; sp < P.splits; sp += 32) {
+      mx = fmaxf(mx, __ldcg(part + sp * PSTRIDE + 0));
+      my = fmaxf(my, __ldcg(part + sp * PSTRIDE + 2));
+    }
+    mx = warp_max(mx);
+    my = warp_max(my);
+    float lx = 0.f, ly = 0.f;
+    for (int sp = lane; sp < P.splits; sp += 32) {
+      const float m_s = __ldcg(part + sp * PSTRIDE + 0), l_s = __ldcg(part + sp * PSTRIDE + 1);
+      const float n_s = __ldcg(part + sp * PSTRIDE + 2), k_s = __ldcg(part + sp * PSTRIDE + 3);
+      const float w_s = l_s > 0.f ? fast_exp2((m_s - mx) * LOG2E) : 0.f;
+      sh_scale[sp] = w_s;
+      lx = fmaf(l_s, w_s, lx);
+      if (k_s > 0.f) ly = fmaf(k_s, fast_exp2((n_s - my) * LOG2E), ly);
+    }
+    lx = warp_sum(lx) + fast_exp2((x_new - mx) * LOG2E);
+    ly = warp_sum(ly) + fast_exp2((y_new - my) * LOG2E);
     if (lane == 0) {
-      const float x_new = s * P.scale;  // bias(p, p) = 0
-      const float y_new = (x_new + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
-      float mx = x_new, my = y_new;
-      for (int sp = 0; sp < P.splits; ++sp) {
-        mx = fmaxf(mx, __ldcg(part + sp * PSTRIDE + 0));
-        my = fmaxf(my, __ldcg(part + sp * PSTRIDE + 2));
-      }
-      float lx = fast_exp2((x_new - mx) * LOG2E), ly = fast_exp2((y_new - my) * LOG2E);
-      for (int sp = 0; sp < P.splits; ++sp) {
-        const float m_s = __ldcg(part + sp * PSTRIDE + 0), l_s = __ldcg(part + sp * PSTRIDE + 1);
-        const float n_s = __ldcg(part + sp * PSTRIDE + 2), k_s = __ldcg(part + sp * PSTRIDE + 3);
-        if (l_s > 0.f) lx = fmaf(l_s, fast_exp2((m_s - mx) * LOG2E), lx);
-        if (k_s > 0.f) ly = fmaf(k_s, fast_exp2((n_s - my) * LOG2E), ly);
-      }
       sh_scalar[0] = mx; sh_scalar[1] = 1.f / lx; sh_scalar[2] = my; sh_scalar[3] = 1.f / ly;
       sh_scalar[4] = x_new; sh_scalar[5] = y_new;
     }
@@ -88,10 +99,7 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   // attention output (Eq. 1): merged partial sums plus the new token's own value row
   for (int c = tid; c < D; c += NT) {
     float o = fast_exp2((x_new - mx) * LOG2E) * __half2float(vn[c]);
-    for (int sp = 0; sp < P.splits; ++sp) {
-      const float m_s = __ldcg(part + sp * PSTRIDE + 0), l_s = __ldcg(part + sp * PSTRIDE + 1);
-      if (l_s > 0.f) o = fmaf(__ldcg(part + sp * PSTRIDE + 4 + c), fast_exp2((m_s - mx) * LOG2E), o);
-    }
+    for (int sp = 0; sp < P.splits; ++sp) o = fmaf(__ldcg(part + sp * PSTRIDE + 4 + c), sh_scale[sp], o);
     P.out[(size_t)u * D + c] = __float2half_rn(o * inv_lx);
   }
 
@@ -421,8 +429,10 @@ cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
 }  // namespace
 
 int decode_tile_rows() { return TILE_ROWS; }
+int decode_max_splits() { return MAX_SPLITS; }
 
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
+  if (P.splits < 1 || P.splits > MAX_SPLITS) return cudaErrorInvalidValue;
   switch (head_dim) {
     case 64: return launch_one<64, 4, 4>(P, units, stream);
     case 128: return launch_one<128, 4, 2>(P, units, stream);   // 64 KB of ring per CTA: three CTAs per SM

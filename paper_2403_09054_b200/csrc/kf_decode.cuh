@@ -32,6 +32,7 @@ struct DecodeParams {
 constexpr size_t STATIC_SCRATCH_BYTES = (size_t)16 << 20;
 
 int decode_tile_rows();
+int decode_max_splits();
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 
 // Same launch with y_scratch / partials / counters carved out of the built-in scratch block
