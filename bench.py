@@ -2,9 +2,13 @@
 """Benchmark of the Keyformer generation-phase hot path (attend + score + evict).
 
 A "step" is one kf_decode_step for every layer of the workload (32 launches for the
-Cerebras-GPT-shaped configuration).  Prints one JSON line (see README/DESIGN for keys).
+Cerebras-GPT-shaped configuration).  Prints one JSON line: the metric (`value`, steps/s over all
+GPUs, inputs resident on the device), `roofline` (algorithmic bytes per launch / measured launch
+time against the measured HBM peak), `e2e` (the same step through kf_decode_step_host with host
+buffers), `cpu_baseline` (the CPU oracle on a bounded sample), `clocks`, `gpu_launches`.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+                    [--phase decode|prefill]
 """
 from __future__ import annotations
 
