@@ -99,7 +99,7 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
  * top-(k-w) of the others by f_theta (ties: lower position), and store the
  * kept K/V rows, positions and scores in ascending position order.  If
  * n_prompt <= k everything is kept.
- *   d_q, d_k, d_v : DEVICE fp16 [B][H][n_prompt][d], read only.
+ *   d_q, d_k, d_v : DEVICE fp16 [B][H][n_prompt][d], read only, 16-byte aligned (KF_EINVAL otherwise).
  *   d_score_opt   : DEVICE fp32 [B][H][n_prompt] or NULL; receives f_theta
  *                   before pruning.
  * Must be called once per layer before that layer's first kf_decode_step. */

@@ -137,6 +137,8 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
   const float* slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   const float inv_tau = (float)(1.0 / (double)c.tau_init);  // the prompt phase is iteration t = 0 of Eq. 12
   if (c.prefill_impl == KF_PREFILL_TENSOR) {
+    // TMA reads the prompt tensors: their base addresses must be 16-byte aligned
+    if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k)) & 15u) return KF_EINVAL;
     kf::PrefillTcArgs A{};
     A.Q = static_cast<const __half*>(d_q);
     A.K = static_cast<const __half*>(d_k);

@@ -79,6 +79,25 @@ def test_other_adjustments(noise, impl):
                           gpu_kwargs=dict(prefill_impl=impl))
 
 
+@pytest.mark.parametrize("seed", range(16))
+def test_random_small_configurations(seed):
+    """Seeded random shapes, budgets, temperatures, adjustments and biases, prompt phase plus a few steps."""
+    rng = np.random.default_rng(1000 + seed)
+    n = int(rng.integers(1, 420))
+    k = int(rng.integers(1, 300))
+    w = int(rng.integers(0, k + 1))
+    wl = W.Workload(name=f"fuzz{seed}", n_layers=int(rng.integers(1, 3)), batch=int(rng.integers(1, 4)),
+                    n_heads=int(rng.integers(1, 5)), head_dim=int(rng.choice([64, 128, 256])), prompt_len=n,
+                    budget_k=k, recent_w=w, gen_len_T=int(rng.integers(0, 9)),
+                    tau_init=float(rng.choice([0.5, 1.0, 1.5])), tau_end=float(rng.choice([1.0, 2.0, 3.0])),
+                    data_seed=seed, noise_seed=int(rng.integers(0, 2 ** 62)),
+                    positional=str(rng.choice(["none", "alibi", "rotary"])), rotary_dims=32)
+    noise = str(rng.choice(["gumbel", "gumbel", "none", "const", "gauss"]))
+    impl = kf.KF_PREFILL_TENSOR if seed % 4 else kf.KF_PREFILL_SIMT
+    steps = int(rng.integers(0, 7))          # may run past T: the temperature is clamped there
+    lockstep.run_workload(wl, steps=steps, noise=noise, gpu_kwargs=dict(prefill_impl=impl))
+
+
 def test_zero_noise_tau_one_scores_are_attention_weights():
     wl = _wl(head_dim=128, tau_init=1.0, tau_end=1.0, gen_len_T=3)
     gpu = lockstep.make_gpu(wl, noise_mode=kf.KF_NOISE_NONE)
