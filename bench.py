@@ -333,10 +333,15 @@ def run_ours(args, wl):
 
 
 # ----------------------------------------------------------------------------- prompt phase
-# Lane-instructions one causal logit needs per sweep when nothing is wasted: Philox4x32-10 shared by four
-# logits (10 rounds x 4 instructions / 4), the 23-bit uniform (3), two logarithms with the u -> 1 repair (6),
-# scale + adjustment (1), subtract + exponential (2), maximum or sum (2).
-PREFILL_LANE_INSTR_PER_LOGIT_SWEEP = 24
+# Issue slots one causal logit needs per sweep when nothing is wasted.  An SM has 128 FP32 lanes but 64 INT32
+# lanes, so a warp's integer / logic / compare instruction takes two dispatch cycles where an FP32 one takes one
+# (measured: the 40 integer instructions of one Philox4x32-10 call cost 84 cycles per warp on a scheduler).
+#   integer: Philox shared by four logits (10 rounds x (2 wide multiplies + 2 three-input xors) / 4 = 10),
+#            23-bit uniform (1 funnel shift), u -> 1 repair (compare + select = 2)                        -> 13
+#   FP32:    uniform and 1 - u (2), repair series (2), noise and logit FMAs (2), sum (1)                   ->  7
+#   MUFU:    two logarithms, one exponential (one issue slot each; 8 cycles each on the 16-lane XU)       ->  3
+PREFILL_INT_INSTR, PREFILL_FP_INSTR, PREFILL_MUFU_INSTR = 13, 7, 3
+PREFILL_LANE_INSTR_PER_LOGIT_SWEEP = 2 * PREFILL_INT_INSTR + PREFILL_FP_INSTR + PREFILL_MUFU_INSTR   # 36 FP32-lane slots
 ALU_LANES_PER_SM, N_SM = 128, 148
 
 
@@ -391,7 +396,7 @@ def run_prefill(args, wl):
                        "qk_tflops_both_sweeps": 2 * 2 * logits * wl.head_dim / (ms * 1e-3) / 1e12,
                        "l2": "Q, K, V of the call (%.0f MB) exceed L2" % (3 * units * n * wl.head_dim * 2 / 1e6)},
             "roofline": {"bound": "alu", "kernel": "prefill_tc (two sweeps)", "achieved": achieved, "peak": peak,
-                         "unit": "T lane-instr/s", "frac": achieved / peak, "traffic": None,
+                         "unit": "T FP32-lane issue slots/s (INT32 instructions count twice)", "frac": achieved / peak, "traffic": None,
                          "lane_instr_per_logit_sweep": PREFILL_LANE_INSTR_PER_LOGIT_SWEEP,
                          "peak_kind": "148 SMs x 128 lanes x 1965 MHz", "sm_mhz_seen": sm_mhz},
             "gpu_launches": int(launches), "clocks": clocks,
