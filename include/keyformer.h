@@ -126,9 +126,14 @@ int kf_decode_step(kf_ctx* ctx, int32_t layer, int32_t step,
                    const void* d_q, const void* d_knew, const void* d_vnew,
                    void* d_out, float* d_score_opt, void* stream);
 
-/* Same step with HOST buffers (pinned memory recommended): copies q, k_new,
- * v_new to the device, runs the step and copies `out` back, all on `stream`.
- * If `wait` is non-zero the call returns after the stream has drained. */
+/* Same step with HOST buffers (pinned memory recommended).  The three inputs are copied to the device on an
+ * internal copy stream, so that they overlap the kernel of the previous call; the step runs on `stream`; `out`
+ * is copied back on a second internal stream, overlapping the next call's kernel.
+ *   - h_q, h_knew, h_vnew must hold their values when the call is made (they are read without waiting for
+ *     work queued earlier on `stream`) and stay unchanged until the step has run.
+ *   - h_out is valid after a call with `wait` != 0 has returned (that call drains `stream` and the result
+ *     copies of all earlier calls), or after kf_poll_error.  With `wait` == 0 nothing is waited for.
+ * The first call creates two streams and six events (host resources; no device memory). */
 int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
                         const void* h_q, const void* h_knew, const void* h_vnew,
                         void* h_out, int32_t wait, void* stream);

@@ -66,7 +66,7 @@ Layout make_layout(const kf_config* c) {
   L.slopes = off; off += align_up((size_t)c->n_heads * 4);
   L.acc_full = off; off += align_up(units * (size_t)c->max_prompt_len * 4);
   L.idx = off; off += align_up(units * k * 4);
-  L.staging = off; off += 4 * align_up(units * d * 2);
+  L.staging = off; off += 8 * align_up(units * d * 2);   // two sets of (q, k_new, v_new, out)
   L.lse2 = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
   L.total = off;
   return L;
@@ -83,6 +83,10 @@ struct kf_ctx {
   std::vector<int32_t> n_prompt;   // per layer, -1 before prefill
   std::vector<int32_t> last_step;  // per layer
   int64_t launches;
+  // kf_decode_step_host: copy streams and events (created on first use), two staging sets used alternately
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t in_done[2] = {nullptr, nullptr}, kernel_done[2] = {nullptr, nullptr}, out_done[2] = {nullptr, nullptr};
+  int64_t host_calls = 0;
 };
 
 extern "C" {
@@ -273,20 +277,45 @@ int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
   if (rc != KF_OK) return rc;
   if (!h_q || !h_knew || !h_vnew || !h_out) return KF_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!ctx->copy_in) {   // host-side resources only: two streams and six events
+    bool ok = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < 2; ++i)
+      ok = cudaEventCreateWithFlags(&ctx->in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->kernel_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->out_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return KF_ECUDA;
+  }
   const Layout& L = ctx->lay;
   const size_t bytes = (size_t)L.units * ctx->cfg.head_dim * 2;
   const size_t stride = align_up(bytes);
-  unsigned char* sq = ctx->ws + L.staging;
+  const int set = (int)(ctx->host_calls & 1);
+  unsigned char* sq = ctx->ws + L.staging + (size_t)set * 4 * stride;
   unsigned char* sk = sq + stride;
   unsigned char* sv = sk + stride;
   unsigned char* so = sv + stride;
-  if (cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return KF_ECUDA;
-  if (cudaMemcpyAsync(sk, h_knew, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return KF_ECUDA;
-  if (cudaMemcpyAsync(sv, h_vnew, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return KF_ECUDA;
+  // Inputs travel on a copy stream so that they overlap the previous call's kernel; this staging set was last
+  // read by the kernel of two calls ago.  (Waiting on an event that was never recorded is a no-op.)
+  bool ok = cudaStreamWaitEvent(ctx->copy_in, ctx->kernel_done[set], 0) == cudaSuccess &&
+            cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
+            cudaMemcpyAsync(sk, h_knew, bytes, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
+            cudaMemcpyAsync(sv, h_vnew, bytes, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
+            cudaEventRecord(ctx->in_done[set], ctx->copy_in) == cudaSuccess &&
+            cudaStreamWaitEvent(st, ctx->in_done[set], 0) == cudaSuccess &&
+            cudaStreamWaitEvent(st, ctx->out_done[set], 0) == cudaSuccess;   // `out` of two calls ago has left
+  if (!ok) return KF_ECUDA;
   const int rc2 = decode_impl(ctx, layer, step, sq, sk, sv, so, nullptr, st);
   if (rc2 != KF_OK) return rc2;
-  if (cudaMemcpyAsync(h_out, so, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KF_ECUDA;
-  if (wait && cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
+  ctx->host_calls += 1;
+  // The result leaves on the other copy stream, overlapping the next call's kernel.
+  ok = cudaEventRecord(ctx->kernel_done[set], st) == cudaSuccess &&
+       cudaStreamWaitEvent(ctx->copy_out, ctx->kernel_done[set], 0) == cudaSuccess &&
+       cudaMemcpyAsync(h_out, so, bytes, cudaMemcpyDeviceToHost, ctx->copy_out) == cudaSuccess &&
+       cudaEventRecord(ctx->out_done[set], ctx->copy_out) == cudaSuccess;
+  if (!ok) return KF_ECUDA;
+  if (wait) {
+    if (cudaStreamSynchronize(ctx->copy_out) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
+  }
   return KF_OK;
 }
 
@@ -401,6 +430,7 @@ int kf_poll_error(kf_ctx* ctx, void* stream) {
   int word = 0;
   if (cudaMemcpyAsync(&word, ctx->ws + ctx->lay.err, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return KF_ECUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
+  if (ctx->copy_out && cudaStreamSynchronize(ctx->copy_out) != cudaSuccess) return KF_ECUDA;
   if (word != 0) {
     if (cudaMemsetAsync(ctx->ws + ctx->lay.err, 0, sizeof(int), st) != cudaSuccess) return KF_ECUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
@@ -412,6 +442,17 @@ int64_t kf_launch_count(const kf_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 int kf_destroy(kf_ctx* ctx) {
   if (!ctx) return KF_EINVAL;
+  if (ctx->copy_in) {   // drain and release the host-variant's streams and events
+    cudaStreamSynchronize(ctx->copy_in);
+    cudaStreamSynchronize(ctx->copy_out);
+    for (int i = 0; i < 2; ++i) {
+      if (ctx->in_done[i]) cudaEventDestroy(ctx->in_done[i]);
+      if (ctx->kernel_done[i]) cudaEventDestroy(ctx->kernel_done[i]);
+      if (ctx->out_done[i]) cudaEventDestroy(ctx->out_done[i]);
+    }
+    cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+  }
   delete ctx;
   return KF_OK;
 }

@@ -209,6 +209,20 @@ def test_host_buffer_variant_matches_device_variant():
         b.kf_decode_step_host(0, s, hq, hk, hv, out_b, wait=True)
         torch.cuda.synchronize()
         assert torch.equal(out_a.cpu(), out_b)
+    # several calls in flight (copies overlapping kernels), one wait at the end
+    outs_a, outs_b, keep = [], [], []
+    for s in range(4, 10):
+        q, kn, vn = W.make_step(wl, 0, s, DEV)
+        out_a = torch.empty_like(q)
+        a.kf_decode_step(0, s, q, kn, vn, out_a)
+        outs_a.append(out_a)
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, kn, vn))
+        keep.append((hq, hk, hv))            # host inputs must outlive the copies that read them
+        outs_b.append(torch.empty_like(hq).pin_memory())
+        b.kf_decode_step_host(0, s, hq, hk, hv, outs_b[-1], wait=(s == 9))
+    torch.cuda.synchronize()
+    for x, y in zip(outs_a, outs_b):
+        assert torch.equal(x.cpu(), y)
     sa, sb = a.kf_view_state(0), b.kf_view_state(0)
     torch.cuda.synchronize()
     for name, x, y in zip("K V pos acc len".split(), sa, sb):
