@@ -242,6 +242,25 @@ static void prefill_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t
   }
 }
 
+// Attention output of the prompt phase (Eq. 1 with the causal mask): row i attends to keys j <= i with the
+// plain softmax of x (no adjustment, temperature 1), exactly what the model's attention layer produces.
+static void prefill_attend_unit(const ko_params* P, int32_t h, int32_t n,
+                                const uint16_t* Q, const uint16_t* K, const uint16_t* V, double* out) {
+  const int d = P->head_dim;
+  std::vector<double> x(n), p(n);
+  for (int i = 0; i < n; ++i) {
+    const int m = i + 1;
+    for (int j = 0; j < m; ++j)
+      x[j] = P->logit_scale * dot_half(Q + (size_t)i * d, K + (size_t)j * d, d) + position_bias(P, h, i, j);
+    softmax_inplace(x.data(), p.data(), m);
+    for (int c = 0; c < d; ++c) {
+      double s = 0.0;
+      for (int j = 0; j < m; ++j) s += p[j] * h2d(V[(size_t)j * d + c]);
+      out[(size_t)i * d + c] = s;
+    }
+  }
+}
+
 // Prompt phase, pruning half: keep w recent + top-(k-w) of the rest, store the
 // kept rows in ascending position order.  keep_override (nullable, [n]) lets a
 // lock-step harness impose a kept set chosen inside the tolerance band.
@@ -350,6 +369,16 @@ void ko_prefill_score_units(const ko_params* P, int32_t U, const int32_t* lbh, i
   for (int u = 0; u < U; ++u) {
     prefill_score_unit(P, lbh[3 * u + 1], lbh[3 * u + 0], lbh[3 * u + 2], n,
                        Q + (size_t)u * n * d, K + (size_t)u * n * d, acc_full + (size_t)u * n);
+  }
+}
+
+void ko_prefill_attend_units(const ko_params* P, int32_t U, const int32_t* lbh, int32_t n,
+                             const uint16_t* Q, const uint16_t* K, const uint16_t* V, double* out /* [U][n][d] */) {
+  const size_t d = (size_t)P->head_dim;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int u = 0; u < U; ++u) {
+    prefill_attend_unit(P, lbh[3 * u + 2], n, Q + (size_t)u * n * d, K + (size_t)u * n * d, V + (size_t)u * n * d,
+                        out + (size_t)u * n * d);
   }
 }
 

@@ -69,6 +69,8 @@ def _load():
             lib.ko_select.argtypes = [vp, vp, i32, i32, i32, i32, vp]
             lib.ko_prefill_score_units.restype = None
             lib.ko_prefill_score_units.argtypes = [pp, i32, vp, i32, vp, vp, vp]
+            lib.ko_prefill_attend_units.restype = None
+            lib.ko_prefill_attend_units.argtypes = [pp, i32, vp, i32, vp, vp, vp, vp]
             lib.ko_prefill_prune_units.restype = None
             lib.ko_prefill_prune_units.argtypes = [pp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
             lib.ko_decode_score_units.restype = None
@@ -199,6 +201,16 @@ class State:
         cp = self.P.c()
         _load().ko_prefill_score_units(C.byref(cp), U, _ptr(self.lbh), n, _ptr(Qb), _ptr(Kb), _ptr(acc))
         return acc
+
+    def prefill_attend(self, Q, K, V) -> np.ndarray:
+        """Causal attention output of the prompt [U][n][d] (Eq. 1; plain softmax, no adjustment)."""
+        Qb, Kb, Vb = _half_bits(Q), _half_bits(K), _half_bits(V)
+        U, n, d = Kb.shape
+        assert U == self.U and d == self.P.head_dim and Qb.shape == Kb.shape == Vb.shape
+        out = np.zeros((U, n, d), dtype=np.float64)
+        cp = self.P.c()
+        _load().ko_prefill_attend_units(C.byref(cp), U, _ptr(self.lbh), n, _ptr(Qb), _ptr(Kb), _ptr(Vb), _ptr(out))
+        return out
 
     def prefill_prune(self, K, V, acc_full, keep_override=None) -> None:
         """Keep w recent + top-(k-w) of the rest (or the imposed set) and store the rows."""

@@ -291,6 +291,25 @@ def _step_inputs(seed, U, d):
     return mk(), mk(), mk()
 
 
+def test_prompt_attention_output_matches_library_causal_attention():
+    """Eq. 1 over the prompt with the causal mask, against torch's attention in fp64 (also with ALiBi as a mask)."""
+    U, n, d = 4, 37, 16
+    Q, K, V = _tiny_prompt(11, U, n, d)
+    t = lambda a: torch.from_numpy(a.astype(np.float64))
+    for slopes in (None, np.array([0.5, 0.125])):
+        P = _params(noise_seed=3, bias_mode=0 if slopes is None else 1, alibi_slopes=slopes)
+        lbh = _lbh(U, P.n_heads)
+        out = ko.State(P, lbh).prefill_attend(Q, K, V)
+        i, j = torch.arange(n)[:, None], torch.arange(n)[None, :]
+        mask = torch.zeros(U, n, n, dtype=torch.float64).masked_fill(j > i, float("-inf"))
+        if slopes is not None:
+            mask = mask - torch.from_numpy(slopes[lbh[:, 2]])[:, None, None] * (i - j).clamp(min=0).to(torch.float64)
+        ref = torch.nn.functional.scaled_dot_product_attention(t(Q), t(K), t(V), attn_mask=mask)
+        assert np.abs(out - ref.numpy()).max() < 1e-12
+    # a transposed operand or a dropped mask would show here: row 0 attends to itself only
+    assert np.abs(out[:, 0] - V[:, 0].astype(np.float64)).max() < 1e-12
+
+
 def test_decode_output_matches_library_attention():
     U, n, d = 3, 30, 16
     P = _params(budget_k=10, recent_w=3, noise_seed=8)
