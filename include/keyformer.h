@@ -107,6 +107,20 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
                            const void* d_q, const void* d_k, const void* d_v,
                            float* d_score_opt, void* stream);
 
+/* Attention output of the prompt phase (Eq. 1 under the causal mask): for every (batch row, head) and query
+ * position i, out_i = sum_{j <= i} softmax_j(x_ij) V_j with the plain softmax of x_ij = scale * Q_i.K_j
+ * (+ bias) -- no logit adjustment and temperature 1, i.e. what the model's attention layer produces, which
+ * section 3.4 leaves untouched.  Runs on the tensor cores; does not read or change the cache state.
+ *   d_q, d_k, d_v : DEVICE fp16 [B][H][n_prompt][d], read only, 16-byte aligned.
+ *   d_out         : DEVICE fp16 [B][H][n_prompt][d], 16-byte aligned.
+ * head_dim 64 and 128 only (KF_EINVAL for 256).
+ * kf_prefill_attend_score_prune is the two calls in one: attention output, then kf_prefill_score_prune. */
+int kf_prefill_attend(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void* d_k, const void* d_v,
+                      void* d_out, void* stream);
+int kf_prefill_attend_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
+                                  const void* d_q, const void* d_k, const void* d_v,
+                                  void* d_out, float* d_score_opt, void* stream);
+
 /* One generation step of Algorithm 1 (t = step >= 1; section 3.4) for every
  * (batch row, head) of `layer`.  The new token (original position
  * p = n_prompt + step - 1) joins the cached entries, so m = len + 1 logits:

@@ -21,7 +21,8 @@ KF_PREFILL_TENSOR, KF_PREFILL_SIMT = 0, 1
 
 EXPORTS = ("kf_workspace_bytes", "kf_create", "kf_prefill_score_prune", "kf_decode_step",
            "kf_decode_step_host", "kf_view_state", "kf_poll_error", "kf_launch_count",
-           "kf_destroy", "kf_strerror", "kf_decode_step_static", "kf_state_bytes", "kf_export_state", "kf_import_state")
+           "kf_destroy", "kf_strerror", "kf_decode_step_static", "kf_state_bytes", "kf_export_state", "kf_import_state",
+           "kf_prefill_attend", "kf_prefill_attend_score_prune")
 
 
 class kf_config(C.Structure):
@@ -62,6 +63,10 @@ def _load() -> C.CDLL:
     lib.kf_create.argtypes = [cfgp, vp, C.c_size_t, vp, C.POINTER(vp)]
     lib.kf_prefill_score_prune.restype = C.c_int
     lib.kf_prefill_score_prune.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.kf_prefill_attend.restype = C.c_int
+    lib.kf_prefill_attend.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.kf_prefill_attend_score_prune.restype = C.c_int
+    lib.kf_prefill_attend_score_prune.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.kf_decode_step.restype = C.c_int
     lib.kf_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.kf_decode_step_host.restype = C.c_int
@@ -200,6 +205,25 @@ class Keyformer:
             _dev_ptr(v, torch.float16, numel, "v"),
             _dev_ptr(score_out, torch.float32, B * H * n, "score_out"), _stream_ptr(stream)),
             "kf_prefill_score_prune")
+
+    def kf_prefill_attend(self, q, k, v, out, stream=None):
+        B, H, d = self.cfg.batch, self.cfg.n_heads, self.cfg.head_dim
+        n = q.shape[-2]
+        numel = B * H * n * d
+        _check(LIB.kf_prefill_attend(
+            self._h, n, _dev_ptr(q, torch.float16, numel, "q"), _dev_ptr(k, torch.float16, numel, "k"),
+            _dev_ptr(v, torch.float16, numel, "v"), _dev_ptr(out, torch.float16, numel, "out"), _stream_ptr(stream)),
+            "kf_prefill_attend")
+
+    def kf_prefill_attend_score_prune(self, layer, q, k, v, out, score_out=None, stream=None):
+        B, H, d = self.cfg.batch, self.cfg.n_heads, self.cfg.head_dim
+        n = q.shape[-2]
+        numel = B * H * n * d
+        _check(LIB.kf_prefill_attend_score_prune(
+            self._h, layer, n, _dev_ptr(q, torch.float16, numel, "q"), _dev_ptr(k, torch.float16, numel, "k"),
+            _dev_ptr(v, torch.float16, numel, "v"), _dev_ptr(out, torch.float16, numel, "out"),
+            _dev_ptr(score_out, torch.float32, B * H * n, "score_out"), _stream_ptr(stream)),
+            "kf_prefill_attend_score_prune")
 
     def kf_decode_step(self, layer, step, q, knew, vnew, out, score_out=None, stream=None):
         numel = self.units * self.cfg.head_dim

@@ -200,6 +200,39 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
   return KF_OK;
 }
 
+int kf_prefill_attend(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void* d_k, const void* d_v,
+                      void* d_out, void* stream) {
+  if (!ctx || !d_q || !d_k || !d_v || !d_out) return KF_EINVAL;
+  const kf_config& c = ctx->cfg;
+  if (n_prompt < 1) return KF_EINVAL;
+  if (c.head_dim != 64 && c.head_dim != 128) return KF_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) | reinterpret_cast<uintptr_t>(d_v) |
+       reinterpret_cast<uintptr_t>(d_out)) & 15u)
+    return KF_EINVAL;
+  const Layout& L = ctx->lay;
+  kf::PrefillAttendArgs A{};
+  A.Q = static_cast<const __half*>(d_q);
+  A.K = static_cast<const __half*>(d_k);
+  A.V = static_cast<const __half*>(d_v);
+  A.out = static_cast<__half*>(d_out);
+  A.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
+  A.err = reinterpret_cast<int*>(ctx->ws + L.err);
+  A.n = n_prompt; A.H = c.n_heads; A.bias_mode = c.bias_mode;
+  A.scale = ctx->scale;
+  if (kf::launch_prefill_attend(A, c.head_dim, L.units, static_cast<cudaStream_t>(stream)) != cudaSuccess) return KF_ECUDA;
+  ctx->launches += 1;
+  return KF_OK;
+}
+
+int kf_prefill_attend_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
+                                  const void* d_q, const void* d_k, const void* d_v,
+                                  void* d_out, float* d_score_opt, void* stream) {
+  if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers || n_prompt < 1 || n_prompt > ctx->cfg.max_prompt_len) return KF_EINVAL;
+  const int rc = kf_prefill_attend(ctx, n_prompt, d_q, d_k, d_v, d_out, stream);
+  if (rc != KF_OK) return rc;
+  return kf_prefill_score_prune(ctx, layer, n_prompt, d_q, d_k, d_v, d_score_opt, stream);
+}
+
 static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q, const void* d_knew,
                        const void* d_vnew, void* d_out, float* d_score_opt, cudaStream_t st) {
   const kf_config& c = ctx->cfg;

@@ -68,6 +68,19 @@ struct PrefillTcArgs {
   PhiloxKeys pk;
 };
 
+// Causal attention output of the prompt (see kf_prefill_attend.cu).
+struct PrefillAttendArgs {
+  const __half* Q;     // [units][n][d]
+  const __half* K;
+  const __half* V;
+  __half* out;         // [units][n][d]
+  const float* slopes; // [H] or null
+  int* err;
+  int32_t n, H, bias_mode;
+  float scale;
+};
+cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int units, cudaStream_t stream);
+
 size_t prefill_tc_lse_floats(int units, int n_max);
 cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int units, cudaStream_t stream);
 cudaError_t launch_prefill_score_simt(const PrefillParams& P, int head_dim, int units, cudaStream_t stream);

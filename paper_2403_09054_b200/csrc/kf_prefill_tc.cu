@@ -20,6 +20,7 @@
 // the 32 accumulator lanes selected by warp id mod 4).  Every wait is bounded; a wait that runs
 // out raises the error word and the CTA drains and frees tensor memory before it leaves.
 #include "kf_prefill.cuh"
+#include "kf_tc.cuh"
 
 #include <cuda.h>
 
@@ -39,90 +40,11 @@ constexpr int tc_threads(int ng) { return (2 + 4 * ng) * 32; }   // TMA warp + M
 constexpr int TC_NG = KF_TC_NG;               // compute groups for head_dim 64 / 128 (256 leaves room for 2)
 constexpr int TC_NACC = 4;                    // accumulator buffers: 4 x 128 columns = all of tensor memory
 constexpr uint32_t TC_TMEM_COLS = 512;
-constexpr uint32_t TC_WAIT_LIMIT = 1u << 21;
-constexpr int TC_BOX_BYTES = 128 * 128;       // one TMA box: 128 rows x 64 binary16
 constexpr int TC_XBUF_FLOATS = 4 * 32 * 4;    // per warp: 4 noise calls x 32 lanes x 4 words
 constexpr float LG2_LN2 = -0.5287663729448977f;  // log2(ln 2)
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
-      : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem] * B[smem]^T, binary16 operands, binary32 accumulation, issued by one thread.
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The barrier receives one arrival once every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// 32 lanes x 32 consecutive binary32 columns: thread t of the warp receives lane (base + t).
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-  tmem_wait_ld();
-#pragma unroll
-  for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
-}
-
-// Shared-memory matrix descriptor of a K-major operand stored as 128-byte swizzled rows
-// (what a TMA box with CU_TENSOR_MAP_SWIZZLE_128B writes): 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4)      // start address / 16
-         | (1ull << 16)                            // leading byte offset (unused with swizzle) = 1
-         | ((uint64_t)(1024 >> 4) << 32)           // stride byte offset between 8-row groups
-         | (1ull << 46)                            // descriptor version of sm_100
-         | (2ull << 61);                           // 128-byte swizzle
-}
-
 // Instruction descriptor: binary16 A and B, both K-major, binary32 accumulator, M = 128, N = 128.
 constexpr uint32_t UMMA_IDESC = (1u << 4) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
-
-// Bounded wait that also gives up when another role of the CTA has already given up.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < TC_WAIT_LIMIT; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if (it > 32) {
-      __nanosleep(40);
-      if ((it & 127u) == 0u && *abort_flag) return false;
-    }
-  }
-  return false;
-}
 
 // ------------------------------------------------------------------ the logit adjustment
 __device__ __forceinline__ float fast_lg2(float x) {   // arguments here are normal numbers: no subnormal handling
@@ -495,6 +417,9 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
 }
 
 // ------------------------------------------------------------------ host side
+}  // namespace
+
+namespace {
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -512,8 +437,8 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// fp16 [units][n][d] viewed as a 3-D tensor (d innermost); boxes of 64 columns x 128 rows, 128-byte swizzle.
-// Rows past n read as zeros, so a block never sees another unit's rows.
+}  // namespace
+
 bool make_operand_map(CUtensorMap* map, const __half* base, int units, int n, int d) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
@@ -525,6 +450,8 @@ bool make_operand_map(CUtensorMap* map, const __half* base, int units, int n, in
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+namespace {
 
 template <int D, int NST, int NG>
 constexpr size_t tc_smem_bytes() {

@@ -1,0 +1,74 @@
+"""GPU parity of the prompt-phase attention output (Eq. 1 under the causal mask) against the CPU oracle,
+through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2403_09054_b200 as kf
+import workloads as W
+from oracle import keyformer_oracle as ko
+from tests import lockstep
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _check(wl, units=None):
+    gpu = lockstep.make_gpu(wl)
+    q, k, v = W.make_prompt(wl, 0, DEV)
+    out = torch.empty_like(q)
+    gpu.kf_prefill_attend(q, k, v, out)
+    assert gpu.kf_poll_error() == 0
+    lbh = W.unit_list(wl, 0) if units is None else W.sample_units(wl, units, seed=3, layer=0)
+    flat = torch.as_tensor(lbh[:, 1] * wl.n_heads + lbh[:, 2], dtype=torch.long, device=DEV)
+    rows = lambda t: t.reshape(wl.batch * wl.n_heads, wl.prompt_len, wl.head_dim)[flat].cpu().numpy()
+    st = ko.State(lockstep.oracle_params(wl), lbh)
+    ref = st.prefill_attend(rows(q), rows(k), rows(v))
+    got = rows(out).astype(np.float64)
+    scale = np.abs(ref).max(axis=-1, keepdims=True)
+    err = np.abs(got - ref) / scale
+    assert err.max() <= lockstep.OUT_RTOL, f"attention output off by {err.max():.3e} of the row's largest value"
+    gpu.kf_destroy()
+    return float(err.max())
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n", [1, 57, 128, 129, 300, 641])
+def test_prompt_attention_small(n, d):
+    _check(W.Workload("attend", 1, 2, 3, d, n, max(1, n // 2), n // 8, 0, data_seed=n + d, noise_seed=1))
+
+
+@pytest.mark.parametrize("positional", ["alibi", "rotary"])
+def test_prompt_attention_with_positional_structure(positional):
+    _check(W.Workload("attend", 1, 2, 4, 128, 333, 100, 10, 0, data_seed=5, positional=positional, rotary_dims=32))
+
+
+def test_prompt_attention_heavy_hitters_sampled_units():
+    wl = W.get_config("c4_cerebras").scaled(n_layers=1, batch=2, n_heads=8, prompt_len=1500, budget_k=512, recent_w=128)
+    _check(wl, units=4)
+
+
+def test_attend_and_score_in_one_call_match_the_separate_calls():
+    wl = W.Workload("attend", 1, 2, 3, 128, 400, 150, 30, 4, data_seed=9, noise_seed=2)
+    q, k, v = W.make_prompt(wl, 0, DEV)
+    a, b = lockstep.make_gpu(wl), lockstep.make_gpu(wl)
+    out_a, out_b = torch.empty_like(q), torch.empty_like(q)
+    sc_a = torch.empty(wl.batch, wl.n_heads, wl.prompt_len, device=DEV)
+    sc_b = torch.empty_like(sc_a)
+    a.kf_prefill_attend_score_prune(0, q, k, v, out_a, score_out=sc_a)
+    b.kf_prefill_attend(q, k, v, out_b)
+    b.kf_prefill_score_prune(0, q, k, v, score_out=sc_b)
+    torch.cuda.synchronize()
+    assert torch.equal(out_a, out_b) and torch.equal(sc_a, sc_b)
+    for x, y in zip(a.kf_view_state(0), b.kf_view_state(0)):
+        assert torch.equal(x, y)
+    assert a.kf_poll_error() == 0 and b.kf_poll_error() == 0
+
+
+def test_attend_rejects_head_dim_256():
+    wl = W.Workload("attend", 1, 1, 2, 256, 64, 32, 8, 0)
+    gpu = lockstep.make_gpu(wl)
+    q, k, v = W.make_prompt(wl, 0, DEV)
+    with pytest.raises(kf.KeyformerError) as e:
+        gpu.kf_prefill_attend(q, k, v, torch.empty_like(q))
+    assert e.value.code == kf.KF_EINVAL
