@@ -362,8 +362,16 @@ def run_prefill(args, wl):
                        prefill_impl=kf.KF_PREFILL_SIMT if args.prefill_simt else kf.KF_PREFILL_TENSOR)
     q, k, v = W.make_prompt(wl, 0, dev)
     stream = torch.cuda.current_stream()
+    attn_out = torch.empty_like(q) if args.with_attention else None
+
+    def call():
+        if attn_out is None:
+            gpu.kf_prefill_score_prune(0, q, k, v, stream=stream)
+        else:
+            gpu.kf_prefill_attend_score_prune(0, q, k, v, attn_out, stream=stream)
+
     for _ in range(args.warmup):
-        gpu.kf_prefill_score_prune(0, q, k, v, stream=stream)
+        call()
     barrier(world)
     sampler = ClockSampler(local)
     sampler.start()
@@ -371,7 +379,7 @@ def run_prefill(args, wl):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        gpu.kf_prefill_score_prune(0, q, k, v, stream=stream)
+        call()
     e1.record(stream)
     barrier(world)
     clocks = sampler.stop()
@@ -390,7 +398,7 @@ def run_prefill(args, wl):
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16 operands, f32 accumulate and score arithmetic",
             "data": "synthetic",
-            "config": {"workload": wl.name, "phase": "prefill", "batch": wl.batch, "heads": wl.n_heads,
+            "config": {"workload": wl.name, "phase": "prefill", "with_attention_output": bool(args.with_attention), "batch": wl.batch, "heads": wl.n_heads,
                        "head_dim": wl.head_dim, "prompt": n, "budget_k": wl.budget_k, "recent_w": wl.recent_w,
                        "causal_logits": logits, "G_logits_per_s": logits / ms / 1e6,
                        "qk_tflops_both_sweeps": 2 * 2 * logits * wl.head_dim / (ms * 1e-3) / 1e12,
@@ -429,6 +437,8 @@ def main():
     ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
                     help="decode: the generation step (the headline metric); prefill: the prompt phase of one layer")
     ap.add_argument("--budget-frac", type=float, default=0.5, help="prefill phase: k as a fraction of the prompt")
+    ap.add_argument("--with-attention", action="store_true",
+                    help="prefill phase: kf_prefill_attend_score_prune (also produces the prompt's attention output)")
     ap.add_argument("--prefill-simt", action="store_true", help="prefill phase: CUDA-core scoring instead of tcgen05")
     args = ap.parse_args()
     wl = W.get_config(args.workload)
