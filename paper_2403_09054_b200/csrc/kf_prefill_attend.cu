@@ -9,8 +9,8 @@
 //            softmax weights, so no running rescale of the output is ever needed), round them to binary16
 //            and store them in shared memory in the 128-byte swizzled K-major operand layout; a second MMA
 //            accumulates O += P V_tile in tensor memory (V is the MN-major B operand, read as TMA wrote it).
-// Warp 0 issues the TMA loads (no multicast), warp 1 owns tensor memory and issues both MMAs, warps 2..9 are
-// two groups of four compute warps, each taking one half of a tile's 128 key columns.  Every wait is bounded;
+// Warp 0 issues the TMA loads (no multicast), warp 1 owns tensor memory and issues both MMAs, the other warps are
+// groups of four compute warps (four groups at head_dim 128), each taking an equal share of a tile's 128 key columns.  Every wait is bounded;
 // a wait that runs out raises the error word and the CTA drains and frees tensor memory before it leaves.
 #include "kf_prefill.cuh"
 #include "kf_tc.cuh"
@@ -21,7 +21,7 @@ namespace kf {
 
 namespace {
 
-constexpr int AT_THREADS = 10 * 32;
+constexpr int at_threads(int ng) { return (2 + 4 * ng) * 32; }   // TMA warp, MMA warp, NG groups of four compute warps
 constexpr uint32_t AT_TMEM_COLS = 512;   // S tiles at columns 0 and 128, O at 256 .. 256 + D
 constexpr uint32_t AT_O_COL = 256;
 
@@ -42,10 +42,14 @@ __device__ __forceinline__ uint64_t umma_smem_desc_mn(uint32_t saddr, uint32_t l
 }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-template <int D, int KST, int VST, bool ALIBI>
-__global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_constant__ AttendParams P) {
+template <int D, int KST, int VST, int NG, bool ALIBI>
+__global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid_constant__ AttendParams P) {
   constexpr int OP_BYTES = 128 * D * 2;
   constexpr int KCH = D / 64;
+  constexpr int NCW = 4 * NG;          // compute warps
+  constexpr int CPG = 4 / NG;          // 32-column chunks of a tile per group
+  static_assert(NG == 2 || NG == 4, "two or four compute groups");
+  static_assert(D / NG == 32, "each group writes one 32-column chunk of the output");
   constexpr uint32_t IDESC_QK = umma_idesc_kk(128);
   constexpr uint32_t IDESC_PV = (1u << 4) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   extern __shared__ unsigned char smem_raw[];
@@ -54,8 +58,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
   unsigned char* sK = sQ + OP_BYTES;
   unsigned char* sV = sK + (size_t)KST * OP_BYTES;
   unsigned char* sP = sV + (size_t)VST * OP_BYTES;            // 128 rows x 128 keys, binary16: two boxes of 16 KB
-  float* stats = reinterpret_cast<float*>(sP + 2 * TC_BOX_BYTES);   // [2 groups][ref, sum][128 rows]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stats + 2 * 2 * 128);
+  float* stats = reinterpret_cast<float*>(sP + 2 * TC_BOX_BYTES);   // [NG groups][ref, sum][128 rows]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stats + NG * 2 * 128);
   uint64_t* q_full = bars;
   uint64_t* k_full = q_full + 1;
   uint64_t* k_empty = k_full + KST;
@@ -82,11 +86,11 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
     mbar_init(q_full, 1);
     for (int s = 0; s < KST; ++s) { mbar_init(k_full + s, 1); mbar_init(k_empty + s, 1); }
     for (int s = 0; s < VST; ++s) { mbar_init(v_full + s, 1); mbar_init(v_empty + s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(s_full + b, 1); mbar_init(s_empty + b, 8); }
-    mbar_init(p_full, 8);
+    for (int b = 0; b < 2; ++b) { mbar_init(s_full + b, 1); mbar_init(s_empty + b, NCW); }
+    mbar_init(p_full, NCW);
     mbar_init(p_empty, 1);
     mbar_init(o_full, 1);
-    mbar_init(stats_bar, 8);
+    mbar_init(stats_bar, NCW);
     mbar_init(drain, 1);
     *abort_flag = 0;
     *issued_k = 0;
@@ -183,7 +187,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
   } else {
     // ------------------------------------------------------------ compute warps
     const int cw = warp - 2;
-    const int grp = cw >> 2;                 // key columns [64 grp, 64 grp + 64) of every tile
+    const int grp = cw >> 2;                 // key columns [128 / NG * grp, 128 / NG * (grp + 1)) of every tile
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int g_row = Rb * 128 + row;        // query position i
@@ -202,8 +206,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
       if (!ok) break;
       tc_fence_after();
 #pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        const int c = grp * 2 + cc;
+      for (int cc = 0; cc < CPG; ++cc) {
+        const int c = grp * CPG + cc;
         if (diag && c > quarter) continue;   // causally masked for the whole warp
         float v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * 128 + c * 32), v);
@@ -252,11 +256,15 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
     float lse = 0.f;
     if (ok) ok = __all_sync(0xffffffffu, wait_bar(stats_bar, 0, abort_flag));
     if (ok) {
-      const float m1 = stats[(grp ^ 1) * 256 + row], l1 = stats[(grp ^ 1) * 256 + 128 + row];
       float m = row_m, l = row_l;
-      if (l1 > 0.f) {
-        if (l > 0.f) { const float mm = fmaxf(m, m1); l = l * fast_exp2(m - mm) + l1 * fast_exp2(m1 - mm); m = mm; }
-        else { m = m1; l = l1; }
+#pragma unroll
+      for (int g = 1; g < NG; ++g) {   // the other groups' threads of this row (a sum of 0: no valid column)
+        const int og = (grp + g) % NG;
+        const float m1 = stats[og * 256 + row], l1 = stats[og * 256 + 128 + row];
+        if (l1 > 0.f) {
+          if (l > 0.f) { const float mm = fmaxf(m, m1); l = l * fast_exp2(m - mm) + l1 * fast_exp2(m1 - mm); m = mm; }
+          else { m = m1; l = l1; }
+        }
       }
       lse = m + log2f(l);
     }
@@ -271,8 +279,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
       if (!ok) break;
       tc_fence_after();
 #pragma unroll 1
-      for (int cc = 0; cc < 2; ++cc) {
-        const int c = grp * 2 + cc;
+      for (int cc = 0; cc < CPG; ++cc) {
+        const int c = grp * CPG + cc;
         uint32_t packed[16];
         if (diag && c > quarter) {
 #pragma unroll
@@ -313,9 +321,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
     if (ok) ok = __all_sync(0xffffffffu, wait_bar(o_full, 0, abort_flag));
     if (ok) {
       tc_fence_after();
-#pragma unroll 1
-      for (int c = 0; c < D / 64; ++c) {
-        const int col = grp * (D / 2) + c * 32;
+      {
+        const int col = grp * 32;
         float v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + AT_O_COL + (uint32_t)col, v);
         if (g_row < P.n) {
@@ -353,19 +360,19 @@ __global__ void __launch_bounds__(AT_THREADS, 1) prefill_attend(const __grid_con
   }
 }
 
-template <int D, int KST, int VST>
+template <int D, int KST, int VST, int NG>
 cudaError_t launch_attend(const AttendParams& P, int units, bool alibi, cudaStream_t st) {
-  constexpr size_t need = 1024 + (size_t)(1 + KST + VST) * 128 * D * 2 + 2 * TC_BOX_BYTES + 2 * 2 * 128 * 4 + 32 * 8 + 64;
+  constexpr size_t need = 1024 + (size_t)(1 + KST + VST) * 128 * D * 2 + 2 * TC_BOX_BYTES + NG * 2 * 128 * 4 + 32 * 8 + 64;
   constexpr size_t smem = need < 120 * 1024 ? 120 * 1024 : need;   // one CTA per SM: it takes all of tensor memory
   static_assert(smem <= 227 * 1024, "shared memory budget of one CTA");
   dim3 grid((unsigned)P.nblk, (unsigned)units);
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, AT_THREADS, smem, st>>>(P);
+    kern<<<grid, at_threads(NG), smem, st>>>(P);
     return cudaGetLastError();
   };
-  return alibi ? go(prefill_attend<D, KST, VST, true>) : go(prefill_attend<D, KST, VST, false>);
+  return alibi ? go(prefill_attend<D, KST, VST, NG, true>) : go(prefill_attend<D, KST, VST, NG, false>);
 }
 
 }  // namespace
@@ -385,8 +392,8 @@ cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int 
   P.a_scale = a.scale * LOG2E;
   const bool alibi = a.bias_mode == 1 && a.slopes != nullptr;
   switch (head_dim) {
-    case 64: return launch_attend<64, 3, 2>(P, units, alibi, stream);
-    case 128: return launch_attend<128, 2, 2>(P, units, alibi, stream);
+    case 64: return launch_attend<64, 3, 2, 2>(P, units, alibi, stream);
+    case 128: return launch_attend<128, 2, 2, 4>(P, units, alibi, stream);
     default: return cudaErrorInvalidValue;   // head_dim 256 does not fit this kernel's shared-memory plan
   }
 }
