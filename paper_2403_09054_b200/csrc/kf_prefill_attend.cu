@@ -7,8 +7,8 @@
 //            tile into the row's softmax reference and sum, giving lse2_i = log2 sum_j 2^(x2_ij).
 //   phase B  S again; the compute warps turn it into the normalised probabilities P = 2^(x2 - lse2) (exact
 //            softmax weights, so no running rescale of the output is ever needed), round them to binary16
-//            and store them in shared memory in the 128-byte swizzled K-major operand layout; a second MMA
-//            accumulates O += P V_tile in tensor memory (V is the MN-major B operand, read as TMA wrote it).
+//            and store them back into tensor memory (two buffers); a second MMA takes P from there as its A
+//            operand and accumulates O += P V_tile (V is the MN-major B operand, read as TMA wrote it).
 // Warp 0 issues the TMA loads (no multicast), warp 1 owns tensor memory and issues both MMAs, the other warps are
 // groups of four compute warps (four groups at head_dim 128), each taking an equal share of a tile's 128 key columns.  Every wait is bounded;
 // a wait that runs out raises the error word and the CTA drains and frees tensor memory before it leaves.
@@ -22,8 +22,9 @@ namespace kf {
 namespace {
 
 constexpr int at_threads(int ng) { return (2 + 4 * ng) * 32; }   // TMA warp, MMA warp, NG groups of four compute warps
-constexpr uint32_t AT_TMEM_COLS = 512;   // S tiles at columns 0 and 128, O at 256 .. 256 + D
+constexpr uint32_t AT_TMEM_COLS = 512;   // S tiles at columns 0 and 128, O at 256 .. 256 + D, P (binary16 pairs) at 384 and 448
 constexpr uint32_t AT_O_COL = 256;
+constexpr uint32_t AT_P_COL = 384;
 
 struct AttendParams {
   CUtensorMap tmQ, tmK, tmV;   // fp16 [units][n][d], 64 x 128 boxes, 128-byte swizzle
@@ -40,7 +41,6 @@ __device__ __forceinline__ uint64_t umma_smem_desc_mn(uint32_t saddr, uint32_t l
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46) |
          (2ull << 61);
 }
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 template <int D, int KST, int VST, int NG, bool ALIBI>
 __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid_constant__ AttendParams P) {
@@ -57,8 +57,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
   unsigned char* sQ = smem;
   unsigned char* sK = sQ + OP_BYTES;
   unsigned char* sV = sK + (size_t)KST * OP_BYTES;
-  unsigned char* sP = sV + (size_t)VST * OP_BYTES;            // 128 rows x 128 keys, binary16: two boxes of 16 KB
-  float* stats = reinterpret_cast<float*>(sP + 2 * TC_BOX_BYTES);   // [NG groups][ref, sum][128 rows]
+  float* stats = reinterpret_cast<float*>(sV + (size_t)VST * OP_BYTES);   // [NG groups][ref, sum][128 rows]
   uint64_t* bars = reinterpret_cast<uint64_t*>(stats + NG * 2 * 128);
   uint64_t* q_full = bars;
   uint64_t* k_full = q_full + 1;
@@ -68,8 +67,8 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
   uint64_t* s_full = v_empty + VST;
   uint64_t* s_empty = s_full + 2;
   uint64_t* p_full = s_empty + 2;
-  uint64_t* p_empty = p_full + 1;
-  uint64_t* o_full = p_empty + 1;
+  uint64_t* p_empty = p_full + 2;
+  uint64_t* o_full = p_empty + 2;
   uint64_t* stats_bar = o_full + 1;
   uint64_t* drain = stats_bar + 1;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
@@ -87,8 +86,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
     for (int s = 0; s < KST; ++s) { mbar_init(k_full + s, 1); mbar_init(k_empty + s, 1); }
     for (int s = 0; s < VST; ++s) { mbar_init(v_full + s, 1); mbar_init(v_empty + s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(s_full + b, 1); mbar_init(s_empty + b, NCW); }
-    mbar_init(p_full, NCW);
-    mbar_init(p_empty, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(p_full + b, NCW); mbar_init(p_empty + b, 1); }
     mbar_init(o_full, 1);
     mbar_init(stats_bar, NCW);
     mbar_init(drain, 1);
@@ -165,18 +163,18 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
         if (t + 1 < T) mma_qk();                            // S of the next tile while P of this one is being written
         if (!ok) break;
         const int sv = t % VST;
-        ok = wait_bar(p_full, (uint32_t)(t & 1), abort_flag);
+        ok = wait_bar(p_full + (t & 1), (uint32_t)((t >> 1) & 1), abort_flag);
         if (ok) ok = wait_bar(v_full + sv, (uint32_t)((t / VST) & 1), abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t p_addr = smem_u32(sP), v_addr = smem_u32(sV + (size_t)sv * OP_BYTES);
+        const uint32_t p_tmem = tmem_base + AT_P_COL + (uint32_t)((t & 1) * 64);
+        const uint32_t v_addr = smem_u32(sV + (size_t)sv * OP_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {                    // 128 keys = 8 x 16
-          const uint64_t da = umma_smem_desc(p_addr + (uint32_t)((kk >> 2) * TC_BOX_BYTES + (kk & 3) * 32));
+        for (int kk = 0; kk < 8; ++kk) {                    // 128 keys = 8 x 16; 16 binary16 = 8 columns of P
           const uint64_t db = umma_smem_desc_mn(v_addr + (uint32_t)(kk * 16 * 128), TC_BOX_BYTES, 1024);
-          umma_f16(tmem_base + AT_O_COL, da, db, IDESC_PV, (t > 0 || kk > 0) ? 1u : 0u);
+          umma_f16_ts(tmem_base + AT_O_COL, p_tmem + (uint32_t)(kk * 8), db, IDESC_PV, (t > 0 || kk > 0) ? 1u : 0u);
         }
-        umma_commit(p_empty);
+        umma_commit(p_empty + (t & 1));
         umma_commit(v_empty + sv);
       }
       if (ok) umma_commit(o_full);
@@ -274,7 +272,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
       const int sit = T + t, b = sit % 2;
       const bool diag = (t == Rb);
       ok = wait_bar(s_full + b, (uint32_t)((sit / 2) & 1), abort_flag);
-      if (ok && t >= 1) ok = wait_bar(p_empty, (uint32_t)((t - 1) & 1), abort_flag);
+      if (ok && t >= 2) ok = wait_bar(p_empty + (t & 1), (uint32_t)(((t >> 1) - 1) & 1), abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -302,19 +300,13 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
             packed[e >> 1] = *reinterpret_cast<const uint32_t*>(&h);
           }
         }
-        // row `row`, keys 32 c .. 32 c + 31: four 16-byte chunks of the 128-byte swizzled row
-        unsigned char* prow = sP + (c >> 1) * TC_BOX_BYTES + row * 128;
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const int chunk = ((c & 1) * 4 + q4) ^ (row & 7);
-          *reinterpret_cast<uint4*>(prow + chunk * 16) =
-              make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
-        }
+        // keys 32 c .. 32 c + 31 of this row: 16 columns of binary16 pairs
+        tmem_st_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + AT_P_COL + (uint32_t)((t & 1) * 64 + c * 16), packed);
       }
-      fence_proxy_async_smem();   // the MMA reads P through the async proxy
+      tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(p_full); mbar_arrive(s_empty + b); }
+      if (lane == 0) { mbar_arrive(p_full + (t & 1)); mbar_arrive(s_empty + b); }
     }
 
     // ---- output: this group's half of the row
@@ -362,7 +354,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
 
 template <int D, int KST, int VST, int NG>
 cudaError_t launch_attend(const AttendParams& P, int units, bool alibi, cudaStream_t st) {
-  constexpr size_t need = 1024 + (size_t)(1 + KST + VST) * 128 * D * 2 + 2 * TC_BOX_BYTES + NG * 2 * 128 * 4 + 32 * 8 + 64;
+  constexpr size_t need = 1024 + (size_t)(1 + KST + VST) * 128 * D * 2 + NG * 2 * 128 * 4 + 32 * 8 + 64;
   constexpr size_t smem = need < 120 * 1024 ? 120 * 1024 : need;   // one CTA per SM: it takes all of tensor memory
   static_assert(smem <= 227 * 1024, "shared memory budget of one CTA");
   dim3 grid((unsigned)P.nblk, (unsigned)units);
@@ -393,7 +385,7 @@ cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int 
   const bool alibi = a.bias_mode == 1 && a.slopes != nullptr;
   switch (head_dim) {
     case 64: return launch_attend<64, 3, 2, 2>(P, units, alibi, stream);
-    case 128: return launch_attend<128, 2, 2, 4>(P, units, alibi, stream);
+    case 128: return launch_attend<128, 3, 2, 4>(P, units, alibi, stream);
     default: return cudaErrorInvalidValue;   // head_dim 256 does not fit this kernel's shared-memory plan
   }
 }
