@@ -21,13 +21,19 @@ namespace {
 constexpr int TILE_ROWS = 32;
 constexpr int MAX_SPLITS = 64;   // CTAs per unit (the closing CTA keeps one weight per split in shared memory)
 
-__device__ __forceinline__ void axpy8(float (&o)[8], float a, const uint4& vv) {
-  const __half2* h = reinterpret_cast<const __half2*>(&vv);
+// o[0..8) += p * v[0..8) for one 16-byte chunk of a value row.  `pp` holds the softmax weight p twice, as a
+// binary16 pair: the products p * v are then exact in binary32 and each mixed-precision fma rounds once, with
+// no conversion instructions (p <= 1 carries a relative rounding error of 2^-11, far inside the output tolerance).
+__device__ __forceinline__ void axpy8(float (&o)[8], uint32_t pp, const uint4& vv) {
+  const uint32_t vw[4] = {vv.x, vv.y, vv.z, vv.w};
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
-    const float2 f = __half22float2(h[c]);
-    o[2 * c] = fmaf(a, f.x, o[2 * c]);
-    o[2 * c + 1] = fmaf(a, f.y, o[2 * c + 1]);
+    asm("{\n\t.reg .b16 pl, ph, vl, vh;\n\t"
+        "mov.b32 {pl, ph}, %2;\n\t"
+        "mov.b32 {vl, vh}, %3;\n\t"
+        "fma.rn.f32.f16 %0, pl, vl, %0;\n\t"
+        "fma.rn.f32.f16 %1, ph, vh, %1;\n\t}"
+        : "+f"(o[2 * c]), "+f"(o[2 * c + 1]) : "r"(pp), "r"(vw[c]));
   }
 }
 
@@ -323,6 +329,8 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
     const float corr_y = fast_exp2((m_y - my_new) * LOG2E);
     const float pr = valid ? fast_exp2((x - mx_new) * LOG2E) : 0.f;
     const float ey = valid ? fast_exp2((y - my_new) * LOG2E) : 0.f;
+    const __half2 pr_h2 = __float2half2_rn(pr);
+    const uint32_t pr_pair = *reinterpret_cast<const uint32_t*>(&pr_h2);   // (p, p) as binary16, for the value phase
     l_x = fmaf(l_x, corr_x, pr);
     l_y = fmaf(l_y, corr_y, ey);
     m_x = mx_new; m_y = my_new;
@@ -339,11 +347,11 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
 #pragma unroll
       for (int i0 = 0; i0 < NLD; i0 += CH) {
         uint4 vv[CH];
-        float a[CH];
+        uint32_t a[CH];
 #pragma unroll
         for (int i = 0; i < CH; ++i) {
           const int r = grp * LPR + i0 + i;
-          a[i] = __shfl_sync(0xffffffffu, pr, r);
+          a[i] = __shfl_sync(0xffffffffu, pr_pair, r);
           vv[i] = r < rows ? *reinterpret_cast<const uint4*>(slot + (size_t)r * D * 2) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
