@@ -113,7 +113,6 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
  * section 3.4 leaves untouched.  Runs on the tensor cores; does not read or change the cache state.
  *   d_q, d_k, d_v : DEVICE fp16 [B][H][n_prompt][d], read only, 16-byte aligned.
  *   d_out         : DEVICE fp16 [B][H][n_prompt][d], 16-byte aligned.
- * head_dim 64 and 128 only (KF_EINVAL for 256).
  * kf_prefill_attend_score_prune is the two calls in one: attention output, then kf_prefill_score_prune. */
 int kf_prefill_attend(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void* d_k, const void* d_v,
                       void* d_out, void* stream);

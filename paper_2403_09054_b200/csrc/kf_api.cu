@@ -205,7 +205,6 @@ int kf_prefill_attend(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void
   if (!ctx || !d_q || !d_k || !d_v || !d_out) return KF_EINVAL;
   const kf_config& c = ctx->cfg;
   if (n_prompt < 1) return KF_EINVAL;
-  if (c.head_dim != 64 && c.head_dim != 128) return KF_EINVAL;
   if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) | reinterpret_cast<uintptr_t>(d_v) |
        reinterpret_cast<uintptr_t>(d_out)) & 15u)
     return KF_EINVAL;

@@ -22,12 +22,10 @@ namespace kf {
 namespace {
 
 constexpr int at_threads(int ng) { return (2 + 4 * ng) * 32; }   // TMA warp, MMA warp, NG groups of four compute warps
-constexpr uint32_t AT_TMEM_COLS = 512;   // S tiles at columns 0 and 128, O at 256 .. 256 + D, P (binary16 pairs) at 384 and 448
-constexpr uint32_t AT_O_COL = 256;
-constexpr uint32_t AT_P_COL = 384;
+constexpr uint32_t AT_TMEM_COLS = 512;   // two S tiles (BN columns each), then O (D columns), then two P buffers (BN / 2 columns of binary16 pairs each)
 
 struct AttendParams {
-  CUtensorMap tmQ, tmK, tmV;   // fp16 [units][n][d], 64 x 128 boxes, 128-byte swizzle
+  CUtensorMap tmQ, tmK, tmV;   // fp16 [units][n][d], boxes of 64 columns x 128 rows (Q) or BN rows (K, V), 128-byte swizzle
   __half* out;                 // [units][n][d]
   const float* slopes;         // [H] or null
   int* err;
@@ -42,22 +40,26 @@ __device__ __forceinline__ uint64_t umma_smem_desc_mn(uint32_t saddr, uint32_t l
          (2ull << 61);
 }
 
-template <int D, int KST, int VST, int NG, bool ALIBI>
+template <int D, int BN, int KST, int VST, int NG, bool ALIBI>
 __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid_constant__ AttendParams P) {
-  constexpr int OP_BYTES = 128 * D * 2;
+  constexpr int OP_BYTES = 128 * D * 2;   // the query block
+  constexpr int KOP_BYTES = BN * D * 2;   // one key / value tile of BN rows
+  constexpr int KBOX = BN * 128;          // one TMA box of a key / value tile: BN rows x 64 binary16
+  constexpr uint32_t AT_O_COL = 2 * BN, AT_P_COL = 2 * BN + D;
+  static_assert(2 * BN + D + BN <= 512, "tensor memory plan");
   constexpr int KCH = D / 64;
   constexpr int NCW = 4 * NG;          // compute warps
-  constexpr int CPG = 4 / NG;          // 32-column chunks of a tile per group
-  static_assert(NG == 2 || NG == 4, "two or four compute groups");
-  static_assert(D / NG == 32, "each group writes one 32-column chunk of the output");
-  constexpr uint32_t IDESC_QK = umma_idesc_kk(128);
+  constexpr int CPG = BN / 32 / NG;    // 32-column chunks of a tile per group
+  constexpr int OCH = D / NG / 32;     // 32-column chunks of the output per group
+  static_assert(CPG >= 1 && CPG * NG * 32 == BN && OCH >= 1 && OCH * NG * 32 == D, "column split over the compute groups");
+  constexpr uint32_t IDESC_QK = umma_idesc_kk(BN);
   constexpr uint32_t IDESC_PV = (1u << 4) | (1u << 16) | ((uint32_t)(D >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   unsigned char* sQ = smem;
   unsigned char* sK = sQ + OP_BYTES;
-  unsigned char* sV = sK + (size_t)KST * OP_BYTES;
-  float* stats = reinterpret_cast<float*>(sV + (size_t)VST * OP_BYTES);   // [NG groups][ref, sum][128 rows]
+  unsigned char* sV = sK + (size_t)KST * KOP_BYTES;
+  float* stats = reinterpret_cast<float*>(sV + (size_t)VST * KOP_BYTES);   // [NG groups][ref, sum][128 rows]
   uint64_t* bars = reinterpret_cast<uint64_t*>(stats + NG * 2 * 128);
   uint64_t* q_full = bars;
   uint64_t* k_full = q_full + 1;
@@ -79,7 +81,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.y;
   const int Rb = P.nblk - 1 - (int)blockIdx.x;   // the longest CTAs of a unit start first
-  const int T = Rb + 1;                          // key tiles 0 .. Rb
+  const int T = (Rb + 1) * (128 / BN);           // key tiles of BN rows up to the end of this query block
 
   if (tid == 0) {
     mbar_init(q_full, 1);
@@ -116,15 +118,15 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
           const int s = kit % KST;
           if (kit >= KST) ok = wait_bar(k_empty + s, (uint32_t)((kit / KST - 1) & 1), abort_flag);
           if (!ok) break;
-          mbar_expect_tx(k_full + s, OP_BYTES);
-          for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sK + (size_t)s * OP_BYTES + kc * TC_BOX_BYTES, &P.tmK, kc * 64, t * 128, u, k_full + s);
+          mbar_expect_tx(k_full + s, KOP_BYTES);
+          for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sK + (size_t)s * KOP_BYTES + kc * KBOX, &P.tmK, kc * 64, t * BN, u, k_full + s);
           ++kit;
           if (pass == 1) {
             const int sv = vit % VST;
             if (vit >= VST) ok = wait_bar(v_empty + sv, (uint32_t)((vit / VST - 1) & 1), abort_flag);
             if (!ok) break;
-            mbar_expect_tx(v_full + sv, OP_BYTES);
-            for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sV + (size_t)sv * OP_BYTES + kc * TC_BOX_BYTES, &P.tmV, kc * 64, t * 128, u, v_full + sv);
+            mbar_expect_tx(v_full + sv, KOP_BYTES);
+            for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sV + (size_t)sv * KOP_BYTES + kc * KBOX, &P.tmV, kc * 64, t * BN, u, v_full + sv);
             ++vit;
           }
         }
@@ -145,11 +147,12 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
         if (ok && sit >= 2) ok = wait_bar(s_empty + b, (uint32_t)((sit / 2 - 1) & 1), abort_flag);
         if (!ok) return;
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(sK + (size_t)s * OP_BYTES);
+        const uint32_t k_addr = smem_u32(sK + (size_t)s * KOP_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (uint32_t)((kk >> 2) * TC_BOX_BYTES + (kk & 3) * 32);
-          umma_f16(tmem_base + (uint32_t)(b * 128), umma_smem_desc(q_addr + off), umma_smem_desc(k_addr + off), IDESC_QK,
+        for (int kk = 0; kk < D / 16; ++kk) {   // 64-column box, then 16 columns = 32 bytes inside it
+          const uint32_t qoff = (uint32_t)((kk >> 2) * TC_BOX_BYTES + (kk & 3) * 32);
+          const uint32_t koff = (uint32_t)((kk >> 2) * KBOX + (kk & 3) * 32);
+          umma_f16(tmem_base + (uint32_t)(b * BN), umma_smem_desc(q_addr + qoff), umma_smem_desc(k_addr + koff), IDESC_QK,
                    kk > 0 ? 1u : 0u);
         }
         umma_commit(k_empty + s);
@@ -167,11 +170,11 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
         if (ok) ok = wait_bar(v_full + sv, (uint32_t)((t / VST) & 1), abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t p_tmem = tmem_base + AT_P_COL + (uint32_t)((t & 1) * 64);
-        const uint32_t v_addr = smem_u32(sV + (size_t)sv * OP_BYTES);
+        const uint32_t p_tmem = tmem_base + AT_P_COL + (uint32_t)((t & 1) * (BN / 2));
+        const uint32_t v_addr = smem_u32(sV + (size_t)sv * KOP_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {                    // 128 keys = 8 x 16; 16 binary16 = 8 columns of P
-          const uint64_t db = umma_smem_desc_mn(v_addr + (uint32_t)(kk * 16 * 128), TC_BOX_BYTES, 1024);
+        for (int kk = 0; kk < BN / 16; ++kk) {              // 16 keys per MMA; 16 binary16 = 8 columns of P
+          const uint64_t db = umma_smem_desc_mn(v_addr + (uint32_t)(kk * 16 * 128), KBOX, 1024);
           umma_f16_ts(tmem_base + AT_O_COL, p_tmem + (uint32_t)(kk * 8), db, IDESC_PV, (t > 0 || kk > 0) ? 1u : 0u);
         }
         umma_commit(p_empty + (t & 1));
@@ -199,22 +202,22 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
     // ---- phase A: softmax statistics of this row over this group's columns
     for (int it = 0; it < T; ++it) {
       const int b = it % 2;
-      const bool diag = (it == Rb);
+      const int dj = it * BN - Rb * 128;   // first key of the tile relative to the first query of the block
       ok = __all_sync(0xffffffffu, wait_bar(s_full + b, (uint32_t)((it / 2) & 1), abort_flag));
       if (!ok) break;
       tc_fence_after();
 #pragma unroll 1
       for (int cc = 0; cc < CPG; ++cc) {
         const int c = grp * CPG + cc;
-        if (diag && c > quarter) continue;   // causally masked for the whole warp
+        if (dj + c * 32 > quarter * 32) continue;   // causally masked for the whole warp
         float v[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * 128 + c * 32), v);
-        if (diag && c == quarter) {
+        tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * BN + c * 32), v);
+        if (dj + c * 32 == quarter * 32) {          // the chunk that holds the diagonal of these 32 rows
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = e <= lane ? v[e] : -INFINITY;
         }
         float bias0 = 0.f;
-        if (ALIBI) bias0 = sb * (float)(it * 128 + c * 32 - g_row);
+        if (ALIBI) bias0 = sb * (float)(it * BN + c * 32 - g_row);
         if (!started) { row_m = fmaf(v[0], A, bias0); started = true; }
         auto fold = [&](float ref, auto mode) -> float {
           constexpr bool WANT_MAX = decltype(mode)::value;
@@ -270,7 +273,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
     // ---- phase B: normalised probabilities of this group's 64 columns into the P operand
     for (int t = 0; ok && t < T; ++t) {
       const int sit = T + t, b = sit % 2;
-      const bool diag = (t == Rb);
+      const int dj = t * BN - Rb * 128;
       ok = wait_bar(s_full + b, (uint32_t)((sit / 2) & 1), abort_flag);
       if (ok && t >= 2) ok = wait_bar(p_empty + (t & 1), (uint32_t)(((t >> 1) - 1) & 1), abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -280,18 +283,18 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
       for (int cc = 0; cc < CPG; ++cc) {
         const int c = grp * CPG + cc;
         uint32_t packed[16];
-        if (diag && c > quarter) {
+        if (dj + c * 32 > quarter * 32) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) packed[e] = 0u;
         } else {
           float v[32];
-          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * 128 + c * 32), v);
-          if (diag && c == quarter) {
+          tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * BN + c * 32), v);
+          if (dj + c * 32 == quarter * 32) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) v[e] = e <= lane ? v[e] : -INFINITY;
           }
           float off = -lse;
-          if (ALIBI) off += sb * (float)(t * 128 + c * 32 - g_row);
+          if (ALIBI) off += sb * (float)(t * BN + c * 32 - g_row);
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             float a0 = fmaf(v[e], A, off), a1 = fmaf(v[e + 1], A, off);
@@ -301,7 +304,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
           }
         }
         // keys 32 c .. 32 c + 31 of this row: 16 columns of binary16 pairs
-        tmem_st_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + AT_P_COL + (uint32_t)((t & 1) * 64 + c * 16), packed);
+        tmem_st_32x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + AT_P_COL + (uint32_t)((t & 1) * (BN / 2) + c * 16), packed);
       }
       tmem_wait_st();
       tc_fence_before();
@@ -313,8 +316,9 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
     if (ok) ok = __all_sync(0xffffffffu, wait_bar(o_full, 0, abort_flag));
     if (ok) {
       tc_fence_after();
-      {
-        const int col = grp * 32;
+#pragma unroll 1
+      for (int oc = 0; oc < OCH; ++oc) {
+        const int col = (grp * OCH + oc) * 32;
         float v[32];
         tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + AT_O_COL + (uint32_t)col, v);
         if (g_row < P.n) {
@@ -352,9 +356,9 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
   }
 }
 
-template <int D, int KST, int VST, int NG>
+template <int D, int BN, int KST, int VST, int NG>
 cudaError_t launch_attend(const AttendParams& P, int units, bool alibi, cudaStream_t st) {
-  constexpr size_t need = 1024 + (size_t)(1 + KST + VST) * 128 * D * 2 + NG * 2 * 128 * 4 + 32 * 8 + 64;
+  constexpr size_t need = 1024 + (size_t)128 * D * 2 + (size_t)(KST + VST) * BN * D * 2 + NG * 2 * 128 * 4 + 32 * 8 + 64;
   constexpr size_t smem = need < 120 * 1024 ? 120 * 1024 : need;   // one CTA per SM: it takes all of tensor memory
   static_assert(smem <= 227 * 1024, "shared memory budget of one CTA");
   dim3 grid((unsigned)P.nblk, (unsigned)units);
@@ -364,7 +368,7 @@ cudaError_t launch_attend(const AttendParams& P, int units, bool alibi, cudaStre
     kern<<<grid, at_threads(NG), smem, st>>>(P);
     return cudaGetLastError();
   };
-  return alibi ? go(prefill_attend<D, KST, VST, NG, true>) : go(prefill_attend<D, KST, VST, NG, false>);
+  return alibi ? go(prefill_attend<D, BN, KST, VST, NG, true>) : go(prefill_attend<D, BN, KST, VST, NG, false>);
 }
 
 }  // namespace
@@ -372,9 +376,10 @@ cudaError_t launch_attend(const AttendParams& P, int units, bool alibi, cudaStre
 cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int units, cudaStream_t stream) {
   if (a.n < 1 || units < 1 || units > 65535) return cudaErrorInvalidValue;
   AttendParams P{};
-  if (!make_operand_map(&P.tmQ, a.Q, units, a.n, head_dim)) return cudaErrorNotSupported;
-  if (!make_operand_map(&P.tmK, a.K, units, a.n, head_dim)) return cudaErrorNotSupported;
-  if (!make_operand_map(&P.tmV, a.V, units, a.n, head_dim)) return cudaErrorNotSupported;
+  const int bn = head_dim == 256 ? 64 : 128;   // key / value rows per tile
+  if (!make_operand_map(&P.tmQ, a.Q, units, a.n, head_dim, 128)) return cudaErrorNotSupported;
+  if (!make_operand_map(&P.tmK, a.K, units, a.n, head_dim, bn)) return cudaErrorNotSupported;
+  if (!make_operand_map(&P.tmV, a.V, units, a.n, head_dim, bn)) return cudaErrorNotSupported;
   P.out = a.out;
   P.slopes = a.slopes;
   P.err = a.err;
@@ -384,9 +389,10 @@ cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int 
   P.a_scale = a.scale * LOG2E;
   const bool alibi = a.bias_mode == 1 && a.slopes != nullptr;
   switch (head_dim) {
-    case 64: return launch_attend<64, 3, 2, 2>(P, units, alibi, stream);
-    case 128: return launch_attend<128, 3, 2, 4>(P, units, alibi, stream);
-    default: return cudaErrorInvalidValue;   // head_dim 256 does not fit this kernel's shared-memory plan
+    case 64: return launch_attend<64, 128, 3, 2, 2>(P, units, alibi, stream);
+    case 128: return launch_attend<128, 128, 3, 2, 4>(P, units, alibi, stream);
+    case 256: return launch_attend<256, 64, 2, 2, 2>(P, units, alibi, stream);   // 64-row key tiles: the 64 KB query block leaves room for no more
+    default: return cudaErrorInvalidValue;
   }
 }
 

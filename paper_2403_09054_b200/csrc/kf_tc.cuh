@@ -110,8 +110,8 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
 // K-major binary16 operands, binary32 accumulator, M = 128, N = n.
 __host__ __device__ constexpr uint32_t umma_idesc_kk(int n) { return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24); }
 
-// fp16 [units][n][d] viewed as a 3-D tensor (d innermost); boxes of 64 columns x 128 rows, 128-byte swizzle.
+// fp16 [units][n][d] viewed as a 3-D tensor (d innermost); boxes of 64 columns x `box_rows` rows, 128-byte swizzle.
 // Rows past n read as zeros, so a block never sees another unit's rows.  False if the driver refuses.
-bool make_operand_map(CUtensorMap* map, const __half* base, int units, int n, int d);
+bool make_operand_map(CUtensorMap* map, const __half* base, int units, int n, int d, int box_rows = 128);
 
 }  // namespace kf
