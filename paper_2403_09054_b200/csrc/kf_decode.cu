@@ -66,6 +66,23 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   constexpr int PSTRIDE = 4 + D;
   const float* part = P.partials + (size_t)u * P.splits * PSTRIDE;
 
+  // Every thread's first batch of entries is requested before the split merge below, so that these loads are
+  // in flight while warp 0 does the merge (the values are only needed after it).
+  float* __restrict__ acc = P.acc + (size_t)u * P.k;
+  int32_t* __restrict__ pos = P.pos + (size_t)u * P.k;
+  const float* __restrict__ ys = P.y_scratch + (size_t)u * (P.k + 1);
+  constexpr int BATCH = 8;
+  float yv[BATCH], av[BATCH];
+  int pv[BATCH];
+#pragma unroll
+  for (int i = 0; i < BATCH; ++i) {
+    const int j = tid + i * NT;
+    const bool in = j < len;
+    yv[i] = in ? __ldcg(ys + j) : 0.f;
+    av[i] = in ? acc[j] : 0.f;
+    pv[i] = in ? pos[j] : 0x7fffffff;
+  }
+
   if (warp == 0) {
     float s = 0.f;
     for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[c]), __half2float(kn[c]), s);
@@ -111,24 +128,20 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
 
   // score (Eq. 11), accumulation and the eviction candidate.  Loads are issued in batches so
   // that a thread has several cache lines in flight instead of one round trip per entry.
-  float* __restrict__ acc = P.acc + (size_t)u * P.k;
-  int32_t* __restrict__ pos = P.pos + (size_t)u * P.k;
-  const float* __restrict__ ys = P.y_scratch + (size_t)u * (P.k + 1);
   float* __restrict__ sc = P.score_opt ? P.score_opt + (size_t)u * (P.k + 1) : nullptr;
   unsigned long long best = ~0ull;
   int best_j = -1;
   const int cutoff = P.p - P.w;  // entries with pos <= cutoff are outside the recent window
-  constexpr int BATCH = 8;
   for (int j0 = tid; j0 < len; j0 += NT * BATCH) {
-    float yv[BATCH], av[BATCH];
-    int pv[BATCH];
+    if (j0 != tid) {   // the first batch was loaded above
 #pragma unroll
-    for (int i = 0; i < BATCH; ++i) {
-      const int j = j0 + i * NT;
-      const bool in = j < len;
-      yv[i] = in ? __ldcg(ys + j) : 0.f;
-      av[i] = in ? acc[j] : 0.f;
-      pv[i] = in ? pos[j] : 0x7fffffff;
+      for (int i = 0; i < BATCH; ++i) {
+        const int j = j0 + i * NT;
+        const bool in = j < len;
+        yv[i] = in ? __ldcg(ys + j) : 0.f;
+        av[i] = in ? acc[j] : 0.f;
+        pv[i] = in ? pos[j] : 0x7fffffff;
+      }
     }
 #pragma unroll
     for (int i = 0; i < BATCH; ++i) {
