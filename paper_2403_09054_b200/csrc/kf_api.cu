@@ -280,7 +280,7 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.noise_mu = c.noise_mu; P.noise_sigma = c.noise_sigma;
   P.pk = ctx->pk;
   if (kf::launch_decode(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
-  ctx->launches += 1;
+  ctx->launches += 2;   // streaming kernel + closing kernel
   ctx->last_step[layer] = step;
   return KF_OK;
 }

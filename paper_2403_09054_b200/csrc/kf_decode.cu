@@ -1,15 +1,18 @@
-// Generation-phase kernel (Algorithm 1, t >= 1): one launch per layer call does
-//   logits -> attention output + Gumbel-softmax score -> accumulate -> evict -> replace.
+// Generation-phase kernels (Algorithm 1, t >= 1): one layer call does
+//   logits -> attention output + Gumbel-softmax score -> accumulate -> evict -> replace
+// in two launches.
 //
-// Grid = (splits, units); a unit is one (batch row, head).  Each CTA streams a
+// decode_kernel, grid = (splits, units); a unit is one (batch row, head).  Each CTA streams a
 // contiguous range of cache slots exactly once: every warp owns 32-row tiles,
 // fetched into a private shared-memory ring by 1-D bulk async copies
 // (cp.async.bulk + mbarrier, no multicast), computes the logits x_j = q.K_j
 // once and uses them twice -- for the value-weighted output (Eq. 1) and for
-// the score softmax of (x_j + zeta_j) / tau (Eq. 4, 11).  The CTA that
-// finishes a unit last (ticket counter, no waiting) merges the split partials,
-// normalises the scores, adds them into f_theta, picks the entry to evict and
-// writes the new token's row into the freed slot.
+// the score softmax of (x_j + zeta_j) / tau (Eq. 4, 11) -- and leaves one partial per split.
+//
+// decode_close_kernel, one CTA per unit, launched as the streaming kernel's programmatic dependent
+// (its CTAs become resident during the streaming kernel's last wave, request what does not depend
+// on it, then pass griddepcontrol.wait): merges the split partials, normalises the scores, adds
+// them into f_theta, picks the entry to evict and writes the new token's row into the freed slot.
 #include "kf_decode.cuh"
 
 #include <mutex>
@@ -50,13 +53,13 @@ __device__ __forceinline__ unsigned long long evict_key(float a, int pos) {
   return ((unsigned long long)__float_as_uint(a) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)pos);
 }
 
-// Work of the CTA that closes a unit: merge splits, normalise, accumulate, evict, replace.
+// Closing a unit: merge splits, normalise, accumulate, evict, replace.  Everything that does not depend on the
+// streaming kernel (scores and positions of the entries, the new token's own logit) is requested before
+// `griddepcontrol.wait`, i.e. while the streaming kernel's last CTAs are still running.
 template <int D, int NT>
 __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
-  __shared__ float sh_scalar[8];
-  __shared__ float sh_scale[MAX_SPLITS];   // 2^(m_s - m) of every split's attention partial (0 for an empty split)
   __shared__ unsigned long long sh_key[NT / 32];
-  __shared__ int sh_victim;
+  __shared__ int sh_j[NT / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = P.H;
   const uint32_t b = (uint32_t)(u / H), h = (uint32_t)(u % H), lh = (uint32_t)P.layer * H + h;
@@ -64,70 +67,86 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   const __half* kn = P.knew + (size_t)u * D;
   const __half* vn = P.vnew + (size_t)u * D;
   constexpr int PSTRIDE = 4 + D;
+  constexpr int CPT = (D + NT - 1) / NT;   // output columns per thread
   const float* part = P.partials + (size_t)u * P.splits * PSTRIDE;
-
-  // Every thread's first batch of entries is requested before the split merge below, so that these loads are
-  // in flight while warp 0 does the merge (the values are only needed after it).
   float* __restrict__ acc = P.acc + (size_t)u * P.k;
   int32_t* __restrict__ pos = P.pos + (size_t)u * P.k;
   const float* __restrict__ ys = P.y_scratch + (size_t)u * (P.k + 1);
-  constexpr int BATCH = 8;
+
+  // ---- independent of the streaming kernel: scores and positions of the first batch of entries, the new
+  //      token's row, its own logit and adjusted logit (every warp computes these for itself: no hand-over)
+  constexpr int BATCH = 8;   // 64 registers per thread keep all closing CTAs of 1024 units resident at once
   float yv[BATCH], av[BATCH];
   int pv[BATCH];
 #pragma unroll
   for (int i = 0; i < BATCH; ++i) {
     const int j = tid + i * NT;
     const bool in = j < len;
-    yv[i] = in ? __ldcg(ys + j) : 0.f;
     av[i] = in ? acc[j] : 0.f;
     pv[i] = in ? pos[j] : 0x7fffffff;
   }
+  // entries beyond the first batch: pull their scores and positions into L2 (one request per 128-byte line)
+  for (int line = tid + (NT * BATCH) / 32; line * 32 < len; line += NT) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(acc + line * 32));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(pos + line * 32));
+  }
+  __half kn_r[CPT], vn_r[CPT];
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    const int c = tid + i * NT;
+    kn_r[i] = c < D ? kn[c] : __float2half(0.f);
+    vn_r[i] = c < D ? vn[c] : __float2half(0.f);
+  }
+  float s = 0.f;
+  for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[c]), __half2float(kn[c]), s);
+  const float x_new = warp_sum(s) * P.scale;  // bias(p, p) = 0
+  float y_new = 0.f;
+  if (lane == 0) y_new = (x_new + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
+  y_new = __shfl_sync(0xffffffffu, y_new, 0);
 
-  if (warp == 0) {
-    float s = 0.f;
-    for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[c]), __half2float(kn[c]), s);
-    s = warp_sum(s);
-    const float x_new = s * P.scale;  // bias(p, p) = 0
-    float y_new = 0.f;
-    if (lane == 0) y_new = (x_new + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
-    y_new = __shfl_sync(0xffffffffu, y_new, 0);
-    // merge the splits' (max, sum) pairs of both softmaxes, one split per lane
-    float mx = x_new, my = y_new;
-    for (int sp = lane; sp < P.splits; sp += 32) {
-      mx = fmaxf(mx, __ldcg(part + sp * PSTRIDE + 0));
-      my = fmaxf(my, __ldcg(part + sp * PSTRIDE + 2));
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the streaming kernel has finished; its writes are visible
+
+  // ---- everything the streaming kernel produced is requested at once
+#pragma unroll
+  for (int i = 0; i < BATCH; ++i) {
+    const int j = tid + i * NT;
+    yv[i] = j < len ? __ldcg(ys + j) : 0.f;
+  }
+  // (max, sum) pairs of both softmaxes: split `lane` and split `lane + 32`
+  float4 ps0 = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), ps1 = ps0;
+  if (lane < P.splits) ps0 = __ldcg(reinterpret_cast<const float4*>(part + (size_t)lane * PSTRIDE));
+  if (lane + 32 < P.splits) ps1 = __ldcg(reinterpret_cast<const float4*>(part + (size_t)(lane + 32) * PSTRIDE));
+  const float mx = warp_max(fmaxf(x_new, fmaxf(ps0.y > 0.f ? ps0.x : -INFINITY, ps1.y > 0.f ? ps1.x : -INFINITY)));
+  const float my = warp_max(fmaxf(y_new, fmaxf(ps0.w > 0.f ? ps0.z : -INFINITY, ps1.w > 0.f ? ps1.z : -INFINITY)));
+  const float w0 = ps0.y > 0.f ? fast_exp2((ps0.x - mx) * LOG2E) : 0.f;   // weight of split `lane` in the output
+  const float w1 = ps1.y > 0.f ? fast_exp2((ps1.x - mx) * LOG2E) : 0.f;
+  float lx = fmaf(ps0.y, w0, ps1.y * w1);
+  float ly = (ps0.w > 0.f ? ps0.w * fast_exp2((ps0.z - my) * LOG2E) : 0.f) + (ps1.w > 0.f ? ps1.w * fast_exp2((ps1.z - my) * LOG2E) : 0.f);
+  const float inv_lx = 1.f / (warp_sum(lx) + fast_exp2((x_new - mx) * LOG2E));
+  const float inv_ly = 1.f / (warp_sum(ly) + fast_exp2((y_new - my) * LOG2E));
+
+  // ---- attention output (Eq. 1): merged partial sums plus the new token's own value row
+  {
+    float o[CPT];
+#pragma unroll
+    for (int i = 0; i < CPT; ++i) o[i] = fast_exp2((x_new - mx) * LOG2E) * __half2float(vn_r[i]);
+#pragma unroll 4
+    for (int sp = 0; sp < P.splits; ++sp) {
+      const float w = __shfl_sync(0xffffffffu, sp < 32 ? w0 : w1, sp & 31);
+#pragma unroll
+      for (int i = 0; i < CPT; ++i) {
+        const int c = tid + i * NT;
+        if (c < D) o[i] = fmaf(__ldcg(part + (size_t)sp * PSTRIDE + 4 + c), w, o[i]);
+      }
     }
-    mx = warp_max(mx);
-    my = warp_max(my);
-    float lx = 0.f, ly = 0.f;
-    for (int sp = lane; sp < P.splits; sp += 32) {
-      const float m_s = __ldcg(part + sp * PSTRIDE + 0), l_s = __ldcg(part + sp * PSTRIDE + 1);
-      const float n_s = __ldcg(part + sp * PSTRIDE + 2), k_s = __ldcg(part + sp * PSTRIDE + 3);
-      const float w_s = l_s > 0.f ? fast_exp2((m_s - mx) * LOG2E) : 0.f;
-      sh_scale[sp] = w_s;
-      lx = fmaf(l_s, w_s, lx);
-      if (k_s > 0.f) ly = fmaf(k_s, fast_exp2((n_s - my) * LOG2E), ly);
-    }
-    lx = warp_sum(lx) + fast_exp2((x_new - mx) * LOG2E);
-    ly = warp_sum(ly) + fast_exp2((y_new - my) * LOG2E);
-    if (lane == 0) {
-      sh_scalar[0] = mx; sh_scalar[1] = 1.f / lx; sh_scalar[2] = my; sh_scalar[3] = 1.f / ly;
-      sh_scalar[4] = x_new; sh_scalar[5] = y_new;
+#pragma unroll
+    for (int i = 0; i < CPT; ++i) {
+      const int c = tid + i * NT;
+      if (c < D) P.out[(size_t)u * D + c] = __float2half_rn(o[i] * inv_lx);
     }
   }
-  __syncthreads();
-  const float mx = sh_scalar[0], inv_lx = sh_scalar[1], my = sh_scalar[2], inv_ly = sh_scalar[3];
-  const float x_new = sh_scalar[4], y_new = sh_scalar[5];
 
-  // attention output (Eq. 1): merged partial sums plus the new token's own value row
-  for (int c = tid; c < D; c += NT) {
-    float o = fast_exp2((x_new - mx) * LOG2E) * __half2float(vn[c]);
-    for (int sp = 0; sp < P.splits; ++sp) o = fmaf(__ldcg(part + sp * PSTRIDE + 4 + c), sh_scale[sp], o);
-    P.out[(size_t)u * D + c] = __float2half_rn(o * inv_lx);
-  }
-
-  // score (Eq. 11), accumulation and the eviction candidate.  Loads are issued in batches so
-  // that a thread has several cache lines in flight instead of one round trip per entry.
+  // ---- score (Eq. 11), accumulation and the eviction candidate
   float* __restrict__ sc = P.score_opt ? P.score_opt + (size_t)u * (P.k + 1) : nullptr;
   unsigned long long best = ~0ull;
   int best_j = -1;
@@ -162,43 +181,39 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   if (sc && tid == 0) sc[len] = z_new;
   const unsigned long long key_new = evict_key(z_new, P.p);
 
+  int slot;   // where the new token's row goes
   if (len < P.k) {  // cache not full yet: append
-    if (tid == 0) { pos[len] = P.p; acc[len] = z_new; P.len[u] = len + 1; }
-    __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + len) * D;
-    __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + len) * D;
-    for (int c = tid; c < D; c += NT) { Kr[c] = kn[c]; Vr[c] = vn[c]; }
-    return;
-  }
-
-  const unsigned long long mine = best;
-  if (P.w == 0) best = key_new < best ? key_new : best;
+    slot = len;
+    if (tid == 0) P.len[u] = len + 1;
+  } else {
+    // smallest key over the CTA: warp minimum by shuffles, the owning lane publishes it with its slot
+    const unsigned long long mine = best;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-    best = other < best ? other : best;
-  }
-  if (lane == 0) sh_key[warp] = best;
-  if (tid == 0) sh_victim = -1;
-  __syncthreads();
-  best = sh_key[0];
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other < best ? other : best;
+    }
+    if (best == ~0ull ? lane == 0 : mine == best) { sh_key[warp] = best; sh_j[warp] = best_j; }   // keys are unique
+    __syncthreads();
+    best = sh_key[0];
+    slot = sh_j[0];
 #pragma unroll
-  for (int wi = 1; wi < NT / 32; ++wi) best = sh_key[wi] < best ? sh_key[wi] : best;
-  if (best == ~0ull) {  // cannot happen for 0 <= w <= k; flag it instead of guessing
-    if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
-    return;
+    for (int wi = 1; wi < NT / 32; ++wi)
+      if (sh_key[wi] < best) { best = sh_key[wi]; slot = sh_j[wi]; }
+    if (P.w == 0 && key_new < best) return;  // the new token itself has the lowest score: it is not stored
+    if (best == ~0ull || slot < 0 || slot >= len) {  // cannot happen for 0 <= w <= k; flag it instead of guessing
+      if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
+      return;
+    }
   }
-  if (best == key_new && P.w == 0) return;  // the new token itself has the lowest score: it is not stored
-  if (mine == best) sh_victim = best_j;      // keys are unique (positions are), so exactly one thread owns it
-  __syncthreads();
-  const int jv = sh_victim;
-  if (jv < 0 || jv >= len) {
-    if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
-    return;
+  if (tid == 0) { pos[slot] = P.p; acc[slot] = z_new; }
+  __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + slot) * D;
+  __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + slot) * D;
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    const int c = tid + i * NT;
+    if (c < D) { Kr[c] = kn_r[i]; Vr[c] = vn_r[i]; }
   }
-  if (tid == 0) { pos[jv] = P.p; acc[jv] = z_new; }
-  __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + jv) * D;
-  __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + jv) * D;
-  for (int c = tid; c < D; c += NT) { Kr[c] = kn[c]; Vr[c] = vn[c]; }
 }
 
 // Warp-wide maximum in one instruction (f32 redux is an sm_100a feature).
@@ -237,8 +252,10 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   __shared__ float sh_m[NW], sh_l[NW], sh_my[NW], sh_ly[NW];
   __shared__ float sh_o[NW][D];
   __shared__ __align__(16) __half sh_q[D];
-  __shared__ unsigned int sh_ticket;
 
+  // the closing kernel may be scheduled as soon as every CTA of this grid has started: it only prefetches until
+  // this grid has completed
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int s = blockIdx.x, u = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane % LPR, grp = lane / LPR;
@@ -423,15 +440,13 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
     }
   }
 
-  // ---- the CTA that arrives last closes the unit (no CTA ever waits for another)
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) sh_ticket = atomicAdd(P.counters + u, 1u);
-  __syncthreads();
-  if (sh_ticket != (unsigned)(P.splits - 1)) return;
-  __threadfence();
-  if (tid == 0) P.counters[u] = 0u;  // ready for the next launch
-  combine_and_evict<D, NT>(P, u, len);
+}
+
+// One CTA per unit, launched behind the streaming kernel as its programmatic dependent.
+template <int D>
+__global__ void __launch_bounds__(128, 8) decode_close_kernel(const __grid_constant__ DecodeParams P) {
+  const int u = blockIdx.x;
+  combine_and_evict<D, 128>(P, u, P.len[u]);
 }
 
 template <int D, int NW, int NSTAGE>
@@ -444,7 +459,21 @@ cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   }
   dim3 grid((unsigned)P.splits, (unsigned)units);
   kern<<<grid, NW * 32, smem, stream>>>(P);
-  return cudaGetLastError();
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  // the closing kernel: programmatic stream serialization lets its CTAs become resident during the streaming
+  // kernel's last wave and run their prologue; griddepcontrol.wait inside orders everything else
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)units);
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_close_kernel<D>, P);
 }
 
 }  // namespace

@@ -150,7 +150,7 @@ def test_call_order_and_argument_errors():
     assert e.value.code == kf.KF_EINVAL
     gpu.kf_decode_step(0, 1, q, kn, vn, out)
     assert gpu.kf_poll_error() == 0
-    assert gpu.kf_launch_count() == 5   # prompt phase: 2 scoring sweeps + select + gather; then 1 decode kernel
+    assert gpu.kf_launch_count() == 6   # prompt phase: 2 scoring sweeps + select + gather; then the decode step's 2 kernels
 
 
 def test_export_import_state_resumes_bit_exactly():
