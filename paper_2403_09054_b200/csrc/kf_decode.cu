@@ -253,8 +253,11 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   __shared__ float sh_o[NW][D];
   __shared__ __align__(16) __half sh_q[D];
 
-  // the closing kernel may be scheduled as soon as every CTA of this grid has started: it only prefetches until
-  // this grid has completed
+  // Both kernels of a step are launched with programmatic stream serialization: this grid's CTAs may become
+  // resident while the kernel before it in the stream is draining, and wait here until that kernel has
+  // completed (so nothing is read or written early); the closing kernel in turn may be scheduled as soon as
+  // every CTA of this grid has started, and only prefetches until this grid has completed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int s = blockIdx.x, u = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -445,6 +448,7 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
 // One CTA per unit, launched behind the streaming kernel as its programmatic dependent.
 template <int D>
 __global__ void __launch_bounds__(128, 8) decode_close_kernel(const __grid_constant__ DecodeParams P) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // lets the next kernel's CTAs queue up behind this grid
   const int u = blockIdx.x;
   combine_and_evict<D, 128>(P, u, P.len[u]);
 }
@@ -457,22 +461,23 @@ cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  dim3 grid((unsigned)P.splits, (unsigned)units);
-  kern<<<grid, NW * 32, smem, stream>>>(P);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  // the closing kernel: programmatic stream serialization lets its CTAs become resident during the streaming
-  // kernel's last wave and run their prologue; griddepcontrol.wait inside orders everything else
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)units);
-  cfg.blockDim = dim3(128);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = stream;
+  // Programmatic stream serialization on both launches: a kernel's CTAs may become resident while its
+  // predecessor in the stream drains; griddepcontrol.wait inside each kernel keeps the ordering.
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)P.splits, (unsigned)units);
+  cfg.blockDim = dim3(NW * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, P);
+  if (e != cudaSuccess) return e;
+  cfg.gridDim = dim3((unsigned)units);
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = 0;
   return cudaLaunchKernelEx(&cfg, decode_close_kernel<D>, P);
 }
 
