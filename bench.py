@@ -42,9 +42,9 @@ def algorithmic_bytes_per_launch(wl: W.Workload) -> int:
     return wl.batch * wl.n_heads * per_unit
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_kernel<128,4,2> launch on a c4_cerebras layer
-# (1024 units, k = 2048, d = 128), from the ncu capture summarised in profiles/decode_kernel_c4_cerebras.md.
-C4_DECODE_TRAFFIC_BYTES = 1.126e9
+# dram__bytes_read.sum + dram__bytes_write.sum of one layer call (decode_kernel<128,4,2> + decode_close_kernel<128>) on a
+# c4_cerebras layer (1024 units, k = 2048, d = 128), from the ncu capture summarised in profiles/decode_kernel_c4_cerebras.md.
+C4_DECODE_TRAFFIC_BYTES = 1.124e9
 
 
 def measured_peaks():
