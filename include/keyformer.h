@@ -176,7 +176,7 @@ typedef struct kf_static_step {
  * being captured or replayed and must not allocate, under a framework that owns every byte of
  * the GPU through its own pool, or in a process whose memory budget is fixed up front.  Such a
  * caller keeps the cache tensors itself and passes them in; the per-launch scratch (adjusted
- * logits, split partials, arrival tickets) lives in a block of KF_STATIC_SCRATCH_BYTES of device
+ * logits, split partials) lives in a block of KF_STATIC_SCRATCH_BYTES of device
  * memory that is part of the library image.  Every GPU that loads the library holds that block
  * until the process exits.  The call itself calls no cudaMalloc, cudaFree or other allocating
  * routine.
@@ -192,8 +192,9 @@ typedef struct kf_static_step {
  *     block the call returns KF_ENOSPC and enqueues nothing.
  *   - The first call on a device looks up the block's device address (with that device current);
  *     make that first call outside any stream capture.
- *   - All calls on a device share the one block, which keeps the previous call's contents; the
- *     call clears what must start at zero.  Two calls whose kernels overlap on the GPU (different
+ *   - All calls on a device share the one block, which keeps the previous call's contents; no
+ *     part of it has to start at zero (the step's first kernel writes every word its second
+ *     kernel reads), so nothing is cleared.  Two calls whose kernels overlap on the GPU (different
  *     streams, no ordering between them) would race on it: keep them on one stream or order them.
  *   - Device-side self-checks have nowhere to report to in this variant (there is no context to
  *     poll); arguments are validated on the host as far as possible. */

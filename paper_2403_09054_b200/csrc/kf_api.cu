@@ -18,7 +18,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
   size_t K, V, acc, pos, len;          // per-layer strides are kv_layer / sc_layer / len_layer
-  size_t y_scratch, partials, counters, err, slopes;
+  size_t y_scratch, partials, err, slopes;
   size_t acc_full, idx, staging, lse2;
   size_t total;
   size_t kv_layer, sc_layer, len_layer; // bytes per layer
@@ -61,7 +61,6 @@ Layout make_layout(const kf_config* c) {
   L.len = off; off += nl * L.len_layer;
   L.y_scratch = off; off += align_up(units * (k + 1) * 4);
   L.partials = off; off += align_up(units * (size_t)L.max_splits * (4 + d) * 4);
-  L.counters = off; off += align_up(units * 4);
   L.err = off; off += ALIGN;
   L.slopes = off; off += align_up((size_t)c->n_heads * 4);
   L.acc_full = off; off += align_up(units * (size_t)c->max_prompt_len * 4);
@@ -118,7 +117,7 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
   ctx->launches = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(ctx->ws + lay.acc, 0, lay.y_scratch - lay.acc, st);  // acc, pos, len
-  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + lay.counters, 0, lay.slopes - lay.counters, st);  // counters, err
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + lay.err, 0, lay.slopes - lay.err, st);  // error word
   if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI)
     e = cudaMemcpyAsync(ctx->ws + lay.slopes, cfg->h_alibi_slopes, (size_t)cfg->n_heads * 4, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI) e = cudaStreamSynchronize(st);  // host array may go away
@@ -249,7 +248,6 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.score_opt = d_score_opt;
   P.y_scratch = reinterpret_cast<float*>(ctx->ws + L.y_scratch);
   P.partials = reinterpret_cast<float*>(ctx->ws + L.partials);
-  P.counters = reinterpret_cast<unsigned int*>(ctx->ws + L.counters);
   P.err = reinterpret_cast<int*>(ctx->ws + L.err);
   P.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   P.k = c.budget_k; P.w = c.recent_w;
@@ -369,8 +367,7 @@ int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t
   splits = (tiles + tps - 1) / tps;
   const size_t y_bytes = align_up((size_t)units * ((size_t)a->budget_k + 1) * 4);
   const size_t partial_bytes = align_up((size_t)units * splits * (4 + (size_t)a->head_dim) * 4);
-  const size_t counter_bytes = align_up((size_t)units * 4);
-  if (y_bytes + partial_bytes + counter_bytes + 256 > kf::STATIC_SCRATCH_BYTES) return KF_ENOSPC;  // before any CUDA call
+  if (y_bytes + partial_bytes + 256 > kf::STATIC_SCRATCH_BYTES) return KF_ENOSPC;  // before any CUDA call
 
   kf::DecodeParams P{};
   P.K = static_cast<const __half*>(d_K);
@@ -390,7 +387,7 @@ int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t
   P.inv_tau = (float)(1.0 / a->tau);
   P.noise_const = a->noise_const;
   P.pk = kf::philox_expand_key(a->noise_seed);
-  const cudaError_t e = kf::launch_decode_static(P, a->head_dim, units, y_bytes, partial_bytes, counter_bytes,
+  const cudaError_t e = kf::launch_decode_static(P, a->head_dim, units, y_bytes, partial_bytes,
                                                  static_cast<cudaStream_t>(stream));
   if (e == cudaErrorMemoryAllocation) return KF_ENOSPC;
   return e == cudaSuccess ? KF_OK : KF_ECUDA;

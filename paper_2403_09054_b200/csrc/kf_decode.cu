@@ -509,8 +509,8 @@ void* g_static_addr[64] = {};
 }  // namespace
 
 cudaError_t launch_decode_static(DecodeParams P, int head_dim, int units, size_t y_bytes, size_t partial_bytes,
-                                 size_t counter_bytes, cudaStream_t stream) {
-  if (y_bytes + partial_bytes + counter_bytes + 256 > STATIC_SCRATCH_BYTES) return cudaErrorMemoryAllocation;
+                                 cudaStream_t stream) {
+  if (y_bytes + partial_bytes + 256 > STATIC_SCRATCH_BYTES) return cudaErrorMemoryAllocation;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -529,11 +529,9 @@ cudaError_t launch_decode_static(DecodeParams P, int head_dim, int units, size_t
   unsigned char* b = static_cast<unsigned char*>(base);
   P.y_scratch = reinterpret_cast<float*>(b);
   P.partials = reinterpret_cast<float*>(b + y_bytes);
-  P.counters = reinterpret_cast<unsigned int*>(b + y_bytes + partial_bytes);
   P.err = reinterpret_cast<int*>(b + STATIC_SCRATCH_BYTES - 256);  // error word of the kernel's self-checks
-  // the arrival tickets must start at zero; everything else is written before it is read
-  e = cudaMemsetAsync(P.counters, 0, counter_bytes, stream);
-  if (e != cudaSuccess) return e;
+  // nothing in the block has to start at zero: every word the closing kernel reads was written by this call's
+  // streaming kernel first
   return launch_decode(P, head_dim, units, stream);
 }
 

@@ -18,7 +18,6 @@ struct DecodeParams {
   float* score_opt;       // [units][k+1] or null
   float* y_scratch;       // [units][k+1] adjusted logits (x + zeta) / tau
   float* partials;        // [units][splits][4 + d]
-  unsigned int* counters; // [units] arrival tickets, zero between launches
   int* err;               // device error word
   const float* slopes;    // [H] ALiBi slopes or null
   int32_t k, w, p;        // budget, recent window, position of the query token
@@ -35,9 +34,9 @@ int decode_tile_rows();
 int decode_max_splits();
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 
-// Same launch with y_scratch / partials / counters carved out of the built-in scratch block
-// (the three sizes are in bytes, each a multiple of 256).  Allocates nothing.
+// Same launch with y_scratch / partials carved out of the built-in scratch block
+// (the sizes are in bytes, each a multiple of 256).  Allocates nothing.
 cudaError_t launch_decode_static(DecodeParams P, int head_dim, int units, size_t y_bytes, size_t partial_bytes,
-                                 size_t counter_bytes, cudaStream_t stream);
+                                 cudaStream_t stream);
 
 }  // namespace kf
