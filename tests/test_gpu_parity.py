@@ -72,6 +72,12 @@ def test_split_counts(splits):
     lockstep.run_workload(wl, gpu_kwargs=dict(decode_splits=splits))
 
 
+def test_large_budget_many_splits():
+    """k = 6200 slots streamed by 48 CTAs per unit: the closing kernel merges more than 32 split partials."""
+    wl = _wl(batch=1, n_heads=2, head_dim=64, prompt_len=6500, budget_k=6200, recent_w=100, gen_len_T=3)
+    lockstep.run_workload(wl, gpu_kwargs=dict(decode_splits=48))
+
+
 @pytest.mark.parametrize("impl", [kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_SIMT])
 @pytest.mark.parametrize("noise", ["none", "const", "gauss"])
 def test_other_adjustments(noise, impl):
