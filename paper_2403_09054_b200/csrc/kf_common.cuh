@@ -133,7 +133,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   return false;
 }
 // 1-D bulk copy global -> shared of `bytes` (multiple of 16, both addresses
-// 16-byte aligned), completion counted on `bar`.  No multicast.
+// 16-byte aligned), completion counted on `bar`.  Each CTA fetches its own copy.
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

@@ -5,7 +5,7 @@
 // decode_kernel, grid = (splits, units); a unit is one (batch row, head).  Each CTA streams a
 // contiguous range of cache slots exactly once: every warp owns 32-row tiles,
 // fetched into a private shared-memory ring by 1-D bulk async copies
-// (cp.async.bulk + mbarrier, no multicast), computes the logits x_j = q.K_j
+// (cp.async.bulk + mbarrier, one copy per CTA), computes the logits x_j = q.K_j
 // once and uses them twice -- for the value-weighted output (Eq. 1) and for
 // the score softmax of (x_j + zeta_j) / tau (Eq. 4, 11) -- and leaves one partial per split.
 //

@@ -9,7 +9,7 @@
 //            softmax weights, so no running rescale of the output is ever needed), round them to binary16
 //            and store them back into tensor memory (two buffers); a second MMA takes P from there as its A
 //            operand and accumulates O += P V_tile (V is the MN-major B operand, read as TMA wrote it).
-// Warp 0 issues the TMA loads (no multicast), warp 1 owns tensor memory and issues both MMAs, the other warps are
+// Warp 0 issues the TMA loads (one copy per CTA), warp 1 owns tensor memory and issues both MMAs, the other warps are
 // groups of four compute warps (four groups at head_dim 128), each taking an equal share of a tile's 128 key columns.  Every wait is bounded;
 // a wait that runs out raises the error word and the CTA drains and frees tensor memory before it leaves.
 #include "kf_prefill.cuh"

@@ -15,7 +15,7 @@
 //
 // One CTA owns a block of 128 rows of the resident operand and streams 128-row tiles of the
 // other one through a ring of shared-memory stages.  Warp 0 issues the TMA loads (128-byte
-// swizzled boxes, no multicast), warp 1 owns tensor memory and issues the MMAs, the other warps are
+// swizzled boxes, one copy per CTA), warp 1 owns tensor memory and issues the MMAs, the other warps are
 // groups of four compute warps that take accumulator tiles in turn (a warp can read
 // the 32 accumulator lanes selected by warp id mod 4).  Every wait is bounded; a wait that runs
 // out raises the error word and the CTA drains and frees tensor memory before it leaves.
