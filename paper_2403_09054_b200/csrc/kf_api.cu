@@ -19,7 +19,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 struct Layout {
   size_t K, V, acc, pos, len;          // per-layer strides are kv_layer / sc_layer / len_layer
   size_t y_scratch, partials, err, slopes;
-  size_t acc_full, idx, staging, lse2;
+  size_t acc_full, idx, staging, lse2, lse_x;
   size_t total;
   size_t kv_layer, sc_layer, len_layer; // bytes per layer
   int units, max_splits;
@@ -67,6 +67,7 @@ Layout make_layout(const kf_config* c) {
   L.idx = off; off += align_up(units * k * 4);
   L.staging = off; off += 8 * align_up(units * d * 2);   // two sets of (q, k_new, v_new, out)
   L.lse2 = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
+  L.lse_x = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
   L.total = off;
   return L;
 }
@@ -126,9 +127,11 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
   return KF_OK;
 }
 
-int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
-                           const void* d_q, const void* d_k, const void* d_v,
-                           float* d_score_opt, void* stream) {
+// `want_x`: the scoring sweep also leaves the plain softmax statistics of the prompt rows in the workspace
+// (tensor-core scoring only), for the attention output kernel.
+static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
+                                    const void* d_q, const void* d_k, const void* d_v,
+                                    float* d_score_opt, bool want_x, void* stream) {
   if (!ctx || !d_q || !d_k || !d_v) return KF_EINVAL;
   const kf_config& c = ctx->cfg;
   if (layer < 0 || layer >= c.n_layers) return KF_EINVAL;
@@ -146,6 +149,7 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
     A.Q = static_cast<const __half*>(d_q);
     A.K = static_cast<const __half*>(d_k);
     A.lse2 = reinterpret_cast<float*>(ctx->ws + L.lse2);
+    A.lse_x = want_x ? reinterpret_cast<float*>(ctx->ws + L.lse_x) : nullptr;
     A.acc_full = acc_full;
     A.slopes = slopes;
     A.err = err;
@@ -199,8 +203,14 @@ int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
   return KF_OK;
 }
 
-int kf_prefill_attend(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void* d_k, const void* d_v,
-                      void* d_out, void* stream) {
+int kf_prefill_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
+                           const void* d_q, const void* d_k, const void* d_v,
+                           float* d_score_opt, void* stream) {
+  return prefill_score_prune_impl(ctx, layer, n_prompt, d_q, d_k, d_v, d_score_opt, false, stream);
+}
+
+static int prefill_attend_impl(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void* d_k, const void* d_v,
+                               void* d_out, bool have_lse_x, void* stream) {
   if (!ctx || !d_q || !d_k || !d_v || !d_out) return KF_EINVAL;
   const kf_config& c = ctx->cfg;
   if (n_prompt < 1) return KF_EINVAL;
@@ -213,6 +223,7 @@ int kf_prefill_attend(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void
   A.K = static_cast<const __half*>(d_k);
   A.V = static_cast<const __half*>(d_v);
   A.out = static_cast<__half*>(d_out);
+  A.lse_x = have_lse_x ? reinterpret_cast<const float*>(ctx->ws + L.lse_x) : nullptr;
   A.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   A.err = reinterpret_cast<int*>(ctx->ws + L.err);
   A.n = n_prompt; A.H = c.n_heads; A.bias_mode = c.bias_mode;
@@ -226,9 +237,18 @@ int kf_prefill_attend_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
                                   const void* d_q, const void* d_k, const void* d_v,
                                   void* d_out, float* d_score_opt, void* stream) {
   if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers || n_prompt < 1 || n_prompt > ctx->cfg.max_prompt_len) return KF_EINVAL;
-  const int rc = kf_prefill_attend(ctx, n_prompt, d_q, d_k, d_v, d_out, stream);
+  if (!d_out) return KF_EINVAL;
+  // with tensor-core scoring the first sweep also produces the rows' plain softmax statistics, so the attention
+  // kernel skips its own statistics pass (one Q K^T pass fewer)
+  const bool share = ctx->cfg.prefill_impl == KF_PREFILL_TENSOR;
+  const int rc = prefill_score_prune_impl(ctx, layer, n_prompt, d_q, d_k, d_v, d_score_opt, share, stream);
   if (rc != KF_OK) return rc;
-  return kf_prefill_score_prune(ctx, layer, n_prompt, d_q, d_k, d_v, d_score_opt, stream);
+  return prefill_attend_impl(ctx, n_prompt, d_q, d_k, d_v, d_out, share, stream);
+}
+
+int kf_prefill_attend(kf_ctx* ctx, int32_t n_prompt, const void* d_q, const void* d_k, const void* d_v,
+                      void* d_out, void* stream) {
+  return prefill_attend_impl(ctx, n_prompt, d_q, d_k, d_v, d_out, false, stream);
 }
 
 static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q, const void* d_knew,

@@ -43,11 +43,13 @@ struct PrefillTcParams {
   CUtensorMap tmQ;     // fp16 [units][n][d], 64 x 128 boxes, 128-byte swizzle
   CUtensorMap tmK;
   float* lse2;         // [units][nblk * 128] log2-domain log-sum-exp of every query row (+inf past n)
+  float* lse_x;        // same for the plain logits x (sweep 1 fills it when non-null), or null
   float* acc_full;     // [units][n] f_theta before pruning
   const float* slopes; // [H] or null
   int* err;
   int32_t n, nblk, H, layer;
   float a_scale;       // logit scale * log2(e) / tau
+  float ax;            // logit scale * log2(e)
   float c1;            // log2(e) / tau
   float inv_tau;
   float const_term;    // constant logit adjustment in the scaled log2 domain (0 without one)
@@ -60,6 +62,7 @@ struct PrefillTcArgs {
   const __half* Q;     // [units][n][d]
   const __half* K;
   float* lse2;         // scratch, prefill_tc_lse_floats(units, n) floats
+  float* lse_x;        // null, or a second such array: receives the plain softmax statistics of the prompt rows
   float* acc_full;     // [units][n], fully overwritten
   const float* slopes;
   int* err;
@@ -74,6 +77,7 @@ struct PrefillAttendArgs {
   const __half* K;
   const __half* V;
   __half* out;         // [units][n][d]
+  const float* lse_x;  // null, or the rows' log2-domain log-sum-exp from the scoring sweep (skips the statistics phase)
   const float* slopes; // [H] or null
   int* err;
   int32_t n, H, bias_mode;

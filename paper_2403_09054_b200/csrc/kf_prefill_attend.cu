@@ -27,6 +27,7 @@ constexpr uint32_t AT_TMEM_COLS = 512;   // two S tiles (BN columns each), then 
 struct AttendParams {
   CUtensorMap tmQ, tmK, tmV;   // fp16 [units][n][d], boxes of 64 columns x 128 rows (Q) or BN rows (K, V), 128-byte swizzle
   __half* out;                 // [units][n][d]
+  const float* lse_in;         // null, or [units][nblk * 128] log2-domain log-sum-exp of the rows: phase A is skipped
   const float* slopes;         // [H] or null
   int* err;
   int32_t n, nblk, H;
@@ -82,6 +83,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
   const int u = blockIdx.y;
   const int Rb = P.nblk - 1 - (int)blockIdx.x;   // the longest CTAs of a unit start first
   const int T = (Rb + 1) * (128 / BN);           // key tiles of BN rows up to the end of this query block
+  const int TA = P.lse_in ? 0 : T;               // tiles of the statistics phase
 
   if (tid == 0) {
     mbar_init(q_full, 1);
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
       for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sQ + kc * TC_BOX_BYTES, &P.tmQ, kc * 64, Rb * 128, u, q_full);
       bool ok = true;
       int kit = 0, vit = 0;
-      for (int pass = 0; ok && pass < 2; ++pass) {
+      for (int pass = (TA == 0 ? 1 : 0); ok && pass < 2; ++pass) {
         for (int t = 0; ok && t < T; ++t) {
           const int s = kit % KST;
           if (kit >= KST) ok = wait_bar(k_empty + s, (uint32_t)((kit / KST - 1) & 1), abort_flag);
@@ -160,7 +162,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
         ++kit;
         ++sit;
       };
-      for (int t = 0; ok && t < T; ++t) mma_qk();          // phase A
+      for (int t = 0; ok && t < TA; ++t) mma_qk();         // phase A
       if (ok) mma_qk();                                     // phase B, tile 0
       for (int t = 0; ok && t < T; ++t) {
         if (t + 1 < T) mma_qk();                            // S of the next tile while P of this one is being written
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
     bool started = false;
 
     // ---- phase A: softmax statistics of this row over this group's columns
-    for (int it = 0; it < T; ++it) {
+    for (int it = 0; it < TA; ++it) {
       const int b = it % 2;
       const int dj = it * BN - Rb * 128;   // first key of the tile relative to the first query of the block
       ok = __all_sync(0xffffffffu, wait_bar(s_full + b, (uint32_t)((it / 2) & 1), abort_flag));
@@ -255,8 +257,9 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
     __syncwarp();
     if (lane == 0) mbar_arrive(stats_bar);
     float lse = 0.f;
-    if (ok) ok = __all_sync(0xffffffffu, wait_bar(stats_bar, 0, abort_flag));
-    if (ok) {
+    if (TA == 0) lse = P.lse_in[(size_t)u * P.nblk * 128 + g_row];   // +inf past the prompt: those rows get P = 0
+    if (ok && TA > 0) ok = __all_sync(0xffffffffu, wait_bar(stats_bar, 0, abort_flag));
+    if (ok && TA > 0) {
       float m = row_m, l = row_l;
 #pragma unroll
       for (int g = 1; g < NG; ++g) {   // the other groups' threads of this row (a sum of 0: no valid column)
@@ -272,7 +275,7 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
 
     // ---- phase B: normalised probabilities of this group's 64 columns into the P operand
     for (int t = 0; ok && t < T; ++t) {
-      const int sit = T + t, b = sit % 2;
+      const int sit = TA + t, b = sit % 2;
       const int dj = t * BN - Rb * 128;
       ok = wait_bar(s_full + b, (uint32_t)((sit / 2) & 1), abort_flag);
       if (ok && t >= 2) ok = wait_bar(p_empty + (t & 1), (uint32_t)(((t >> 1) - 1) & 1), abort_flag);
@@ -381,6 +384,7 @@ cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int 
   if (!make_operand_map(&P.tmK, a.K, units, a.n, head_dim, bn)) return cudaErrorNotSupported;
   if (!make_operand_map(&P.tmV, a.V, units, a.n, head_dim, bn)) return cudaErrorNotSupported;
   P.out = a.out;
+  P.lse_in = a.lse_x;
   P.slopes = a.slopes;
   P.err = a.err;
   P.n = a.n;

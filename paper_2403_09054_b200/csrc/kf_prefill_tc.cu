@@ -94,7 +94,7 @@ __device__ __forceinline__ float4 noise_terms(const PhiloxKeys& pk, uint32_t jgr
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int D, int NST, int NG, bool SWEEP2, int NOISE, bool ALIBI>
+template <int D, int NST, int NG, bool SWEEP2, int NOISE, bool ALIBI, bool WANT_X>
 __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_constant__ PrefillTcParams P) {
   constexpr int OP_BYTES = TC_BM * D * 2;  // one operand block: D / 64 boxes
   constexpr int KCH = D / 64;              // 64-column boxes per operand row
@@ -105,8 +105,8 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
   constexpr int NCW = 4 * NG;                                // compute warps
   float* xbuf = reinterpret_cast<float*>(sS + (size_t)NST * OP_BYTES);  // [NCW][TC_XBUF_FLOATS] noise exchange
   float* lse_s = xbuf + NCW * TC_XBUF_FLOATS;                // [NCW][128] lse2 of the current query tile
-  float* comb = lse_s + NCW * 128;                           // [NG - 1][2][128] hand-over between the compute groups
-  uint64_t* bars = reinterpret_cast<uint64_t*>(comb + (NG - 1) * 2 * 128);
+  float* comb = lse_s + NCW * 128;                           // [NG - 1][4][128] hand-over between the compute groups
+  uint64_t* bars = reinterpret_cast<uint64_t*>(comb + (NG - 1) * 4 * 128);
   uint64_t* r_full = bars;
   uint64_t* s_full = bars + 1;
   uint64_t* s_empty = s_full + NST;
@@ -147,6 +147,9 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
   // per-thread results of the compute warps
   float row_m = 0.f, row_l = 0.f;         // sweep 1: reference exponent and sum_j 2^(y2_j - row_m) of this query row
   bool started = false;
+  // sweep 1, when the caller also wants the attention layer's own statistics: the same for the plain logits
+  float rowx_m = 0.f, rowx_l = 0.f;
+  bool started_x = false;
   float col_sum = 0.f;                    // sweep 2: f_theta partial of this key
 
   if (warp == 0) {
@@ -302,6 +305,38 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
             row_l *= 5.4210109e-20f;     // 2^-64
             row_m += 64.f;
           }
+          if (WANT_X) {
+            // plain softmax of x (no adjustment, temperature 1): log-sum-exp for the attention output kernel
+            const float Ax = P.ax;
+            float bias0x = 0.f, sbx = 0.f;
+            if (ALIBI) { sbx = P.slopes[h] * LOG2E; bias0x = sbx * (float)(col0 - g_row); }
+            if (!started_x) { rowx_m = fmaf(v[0], Ax, bias0x); started_x = true; }
+            auto fold_x = [&](float rx, auto mode) -> float {
+              constexpr bool WANT_MAX = decltype(mode)::value;
+              float r0 = WANT_MAX ? -INFINITY : 0.f, r1 = r0, r2 = r0, r3 = r0;
+#pragma unroll
+              for (int e = 0; e < 32; e += 4) {
+                float a4[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  a4[q] = fmaf(v[e + q], Ax, bias0x - rx);
+                  if (ALIBI) a4[q] = fmaf(sbx, (float)(e + q), a4[q]);
+                }
+                if (WANT_MAX) { r0 = fmaxf(r0, a4[0]); r1 = fmaxf(r1, a4[1]); r2 = fmaxf(r2, a4[2]); r3 = fmaxf(r3, a4[3]); }
+                else { r0 += fast_exp2(a4[0]); r1 += fast_exp2(a4[1]); r2 += fast_exp2(a4[2]); r3 += fast_exp2(a4[3]); }
+              }
+              return WANT_MAX ? fmaxf(fmaxf(r0, r1), fmaxf(r2, r3)) : (r0 + r1) + (r2 + r3);
+            };
+            float rx = rowx_m;
+            float sx = fold_x(rx, std::false_type{});
+            if (!(sx < 1e30f)) {
+              const float cm = fold_x(rx, std::true_type{});
+              if (cm < INFINITY) { rx += cm; sx = fold_x(rx, std::false_type{}); }
+            }
+            if (rx != rowx_m) { rowx_l *= fast_exp2(rowx_m - rx); rowx_m = rx; }
+            rowx_l += sx;
+            if (rowx_l > 1.8446744e19f) { rowx_l *= 5.4210109e-20f; rowx_m += 64.f; }
+          }
         } else {
           // ---- thread = key j: add z_ij = 2^(y2_ij - lse2_i) over 32 queries to col_sum
           float bias0 = 0.f;
@@ -365,9 +400,11 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
       atomicExch(P.err, ERR_TIMEOUT);
     }
     if (grp > 0) {
-      float* mine = comb + (grp - 1) * 256;
+      float* mine = comb + (grp - 1) * 512;
       mine[row] = SWEEP2 ? col_sum : row_m;
       mine[128 + row] = row_l;
+      mine[256 + row] = rowx_m;
+      mine[384 + row] = rowx_l;
     }
   }
 
@@ -377,26 +414,29 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
     const int g_row = Rb * TC_BM + row;
     if (!SWEEP2) {
       // merge the groups' (reference, sum) pairs; a sum of 0 marks a group that had no tile
-      float m = row_m, l = row_l;
+      auto merged = [&](float m, float l, int off) -> float {
 #pragma unroll
-      for (int g = 1; g < NG; ++g) {
-        const float m1 = comb[(g - 1) * 256 + row], l1 = comb[(g - 1) * 256 + 128 + row];
-        if (l1 > 0.f) {
-          if (l > 0.f) {
-            const float mm = fmaxf(m, m1);
-            l = l * fast_exp2(m - mm) + l1 * fast_exp2(m1 - mm);
-            m = mm;
-          } else {
-            m = m1; l = l1;
+        for (int g = 1; g < NG; ++g) {
+          const float m1 = comb[(g - 1) * 512 + off + row], l1 = comb[(g - 1) * 512 + off + 128 + row];
+          if (l1 > 0.f) {
+            if (l > 0.f) {
+              const float mm = fmaxf(m, m1);
+              l = l * fast_exp2(m - mm) + l1 * fast_exp2(m1 - mm);
+              m = mm;
+            } else {
+              m = m1; l = l1;
+            }
           }
         }
-      }
-      // rows past the prompt get +inf: their scores vanish in sweep 2
-      P.lse2[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? m + log2f(l) : INFINITY;
+        return m + log2f(l);
+      };
+      // rows past the prompt get +inf: their scores vanish in sweep 2 (and their attention weights likewise)
+      P.lse2[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? merged(row_m, row_l, 0) : INFINITY;
+      if (WANT_X) P.lse_x[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? merged(rowx_m, rowx_l, 256) : INFINITY;
     } else if (g_row < P.n) {
       float total = col_sum;
 #pragma unroll
-      for (int g = 1; g < NG; ++g) total += comb[(g - 1) * 256 + row];
+      for (int g = 1; g < NG; ++g) total += comb[(g - 1) * 512 + row];
       P.acc_full[(size_t)u * P.n + g_row] = total;
     }
   }
@@ -456,7 +496,7 @@ namespace {
 template <int D, int NST, int NG>
 constexpr size_t tc_smem_bytes() {
   size_t b = 1024 + (size_t)(1 + NST) * TC_BM * D * 2 + (size_t)4 * NG * TC_XBUF_FLOATS * 4 + (size_t)4 * NG * 128 * 4 +
-             (size_t)(NG - 1) * 2 * 128 * 4 + 32 * 8 + 64;
+             (size_t)(NG - 1) * 4 * 128 * 4 + 32 * 8 + 64;
   return b < 120 * 1024 ? 120 * 1024 : b;   // one CTA per SM: each takes all of tensor memory
 }
 
@@ -471,11 +511,22 @@ cudaError_t launch_variant(const PrefillTcParams& P, int units, int noise, bool 
     kern<<<grid, tc_threads(NG), smem, st>>>(P);
     return cudaGetLastError();
   };
+  // the plain-softmax statistics are an extra of sweep 1 only
+  const bool want_x = !SWEEP2 && P.lse_x != nullptr;
+  auto pick = [&](auto noise_c, auto alibi_c) -> cudaError_t {
+    constexpr int NZ = decltype(noise_c)::value;
+    constexpr bool AL = decltype(alibi_c)::value;
+    if constexpr (!SWEEP2) {
+      if (want_x) return go(prefill_tc<D, NST, NG, false, NZ, AL, true>);
+    }
+    return go(prefill_tc<D, NST, NG, SWEEP2, NZ, AL, false>);
+  };
+  using std::integral_constant;
   if (noise == NOISE_GUMBEL_T)
-    return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GUMBEL_T, true>) : go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GUMBEL_T, false>);
+    return alibi ? pick(integral_constant<int, NOISE_GUMBEL_T>{}, std::true_type{}) : pick(integral_constant<int, NOISE_GUMBEL_T>{}, std::false_type{});
   if (noise == NOISE_GAUSS_T)
-    return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GAUSS_T, true>) : go(prefill_tc<D, NST, NG, SWEEP2, NOISE_GAUSS_T, false>);
-  return alibi ? go(prefill_tc<D, NST, NG, SWEEP2, NOISE_OFF, true>) : go(prefill_tc<D, NST, NG, SWEEP2, NOISE_OFF, false>);
+    return alibi ? pick(integral_constant<int, NOISE_GAUSS_T>{}, std::true_type{}) : pick(integral_constant<int, NOISE_GAUSS_T>{}, std::false_type{});
+  return alibi ? pick(integral_constant<int, NOISE_OFF>{}, std::true_type{}) : pick(integral_constant<int, NOISE_OFF>{}, std::false_type{});
 }
 
 }  // namespace
@@ -486,6 +537,8 @@ cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int un
   if (!make_operand_map(&P.tmQ, a.Q, units, a.n, head_dim)) return cudaErrorNotSupported;
   if (!make_operand_map(&P.tmK, a.K, units, a.n, head_dim)) return cudaErrorNotSupported;
   P.lse2 = a.lse2;
+  P.lse_x = a.lse_x;
+  P.ax = a.scale * LOG2E;
   P.acc_full = a.acc_full;
   P.slopes = a.slopes;
   P.err = a.err;

@@ -48,8 +48,9 @@ def test_prompt_attention_heavy_hitters_sampled_units():
     _check(wl, units=4)
 
 
-def test_attend_and_score_in_one_call_match_the_separate_calls():
-    wl = W.Workload("attend", 1, 2, 3, 128, 400, 150, 30, 4, data_seed=9, noise_seed=2)
+@pytest.mark.parametrize("d,positional", [(128, "none"), (64, "alibi"), (256, "rotary")])
+def test_attend_and_score_in_one_call_match_the_separate_calls(d, positional):
+    wl = W.Workload("attend", 1, 2, 3, d, 400, 150, 30, 4, data_seed=9, noise_seed=2, positional=positional, rotary_dims=32)
     q, k, v = W.make_prompt(wl, 0, DEV)
     a, b = lockstep.make_gpu(wl), lockstep.make_gpu(wl)
     out_a, out_b = torch.empty_like(q), torch.empty_like(q)
@@ -59,7 +60,10 @@ def test_attend_and_score_in_one_call_match_the_separate_calls():
     b.kf_prefill_attend(q, k, v, out_b)
     b.kf_prefill_score_prune(0, q, k, v, score_out=sc_b)
     torch.cuda.synchronize()
-    assert torch.equal(out_a, out_b) and torch.equal(sc_a, sc_b)
+    # the one-call form takes the rows' softmax statistics from the scoring sweep (another summation order)
+    scale = out_b.float().abs().amax(dim=-1, keepdim=True)
+    assert ((out_a.float() - out_b.float()).abs() <= 1e-3 * scale).all()
+    assert torch.equal(sc_a, sc_b)
     for x, y in zip(a.kf_view_state(0), b.kf_view_state(0)):
         assert torch.equal(x, y)
     assert a.kf_poll_error() == 0 and b.kf_poll_error() == 0
