@@ -430,6 +430,7 @@ def main():
                     help="DRAM bytes per launch of the decode kernel from an ncu capture (default: the committed "
                          "capture of the current kernel on the Cerebras-shaped layer, see profiles/)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling a small case)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (a scaled copy of the workload)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (profiling a small case)")
     ap.add_argument("--graph", action="store_true",
                     help="decode phase: record the timed steps into one CUDA graph and replay it once (takes the host's "
@@ -444,6 +445,8 @@ def main():
     wl = W.get_config(args.workload)
     if args.layers > 0:
         wl = wl.scaled(n_layers=args.layers, name=f"{wl.name}[layers={args.layers}]")
+    if args.batch > 0:
+        wl = wl.scaled(batch=args.batch, name=f"{wl.name}[batch={args.batch}]")
     if args.phase == "prefill" and args.impl == "ours":
         run_prefill(args, wl)
     elif args.impl == "reference":
