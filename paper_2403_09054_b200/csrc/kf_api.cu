@@ -237,7 +237,11 @@ int kf_prefill_attend_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
                                   const void* d_q, const void* d_k, const void* d_v,
                                   void* d_out, float* d_score_opt, void* stream) {
   if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers || n_prompt < 1 || n_prompt > ctx->cfg.max_prompt_len) return KF_EINVAL;
-  if (!d_out) return KF_EINVAL;
+  // everything the second half would reject is rejected here, before anything is enqueued
+  if (!d_q || !d_k || !d_v || !d_out) return KF_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) | reinterpret_cast<uintptr_t>(d_v) |
+       reinterpret_cast<uintptr_t>(d_out)) & 15u)
+    return KF_EINVAL;
   // with tensor-core scoring the first sweep also produces the rows' plain softmax statistics, so the attention
   // kernel skips its own statistics pass (one Q K^T pass fewer)
   const bool share = ctx->cfg.prefill_impl == KF_PREFILL_TENSOR;
