@@ -76,7 +76,7 @@ typedef struct kf_config {
   const float* h_alibi_slopes; /* HOST [H], read during kf_create when bias_mode == KF_BIAS_ALIBI */
   float   logit_scale;     /* 0 => 1/sqrt(d) (Eq. 1 / Eq. 4)                      */
   float   noise_const;     /* c of KF_NOISE_CONST                                 */
-  int32_t decode_splits;   /* 0 = choose automatically; else CTAs per unit in the decode kernel */
+  int32_t decode_splits;   /* 0 = choose automatically; else CTAs per unit in the decode kernel (at most 64) */
   int32_t prefill_impl;    /* KF_PREFILL_*                                        */
   float   noise_mu;        /* mean of KF_NOISE_GAUSS (the paper matches Gumbel's 0.5772)          */
   float   noise_sigma;     /* standard deviation of KF_NOISE_GAUSS (1.2825 in the paper)         */
