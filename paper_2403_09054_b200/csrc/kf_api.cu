@@ -281,7 +281,7 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   const int tiles = tiles_of(c.budget_k);
   int splits = c.decode_splits;
   if (splits <= 0) {
-    const int target_ctas = 148 * 8;
+    const int target_ctas = 148 * 20;   // about ten waves of the two resident CTAs per SM
     splits = (target_ctas + L.units - 1) / L.units;
   }
   splits = std::max(1, std::min(splits, std::min(L.max_splits, (tiles + 3) / 4)));
@@ -386,7 +386,7 @@ int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t
   if (a->bias_mode == KF_BIAS_ALIBI && !a->d_alibi_slopes) return KF_EINVAL;
   const int units = a->batch * a->n_heads;
   const int tiles = tiles_of(a->budget_k);
-  int splits = std::max(1, std::min((148 * 8 + units - 1) / units, std::min(64, (tiles + 3) / 4)));
+  int splits = std::max(1, std::min((148 * 20 + units - 1) / units, std::min(64, (tiles + 3) / 4)));
   int tps = ((tiles + splits - 1) / splits + 3) / 4 * 4;
   splits = (tiles + tps - 1) / tps;
   const size_t y_bytes = align_up((size_t)units * ((size_t)a->budget_k + 1) * 4);

@@ -490,7 +490,10 @@ cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaSt
   if (P.splits < 1 || P.splits > MAX_SPLITS) return cudaErrorInvalidValue;
   switch (head_dim) {
     case 64: return launch_one<64, 4, 4>(P, units, stream);
-    case 128: return launch_one<128, 4, 2>(P, units, stream);   // 64 KB of ring per CTA: three CTAs per SM
+    case 128:
+      // long items (bandwidth-bound workloads): five warps and 80 KB of ring per CTA, two CTAs per SM, measured best;
+      // short items (few units, latency-bound): four warps, three CTAs per SM
+      return P.tiles_per_split >= 16 ? launch_one<128, 5, 2>(P, units, stream) : launch_one<128, 4, 2>(P, units, stream);
     case 256: return launch_one<256, 4, 2>(P, units, stream);
     default: return cudaErrorInvalidValue;
   }
