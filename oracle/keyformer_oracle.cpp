@@ -40,7 +40,7 @@ struct ko_params {
   int32_t gen_len_T;     // T
   int32_t noise_mode;    // 0 Gumbel (Eq. 7), 1 none, 2 constant c, 3 Gaussian(mu, sigma)
   int32_t bias_mode;     // 0 none, 1 ALiBi: bias(i,j) = -slope_h * (i - j)
-  int32_t reserved;
+  int32_t pos_mode;      // 0 original token positions in the bias, 1 positions within the reduced cache (section 4.4.2)
   double tau_init;       // Eq. 12
   double tau_end;        // Eq. 12
   double logit_scale;    // 1/sqrt(d_k) of Eq. 1 / Eq. 4
@@ -313,7 +313,10 @@ static void decode_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t 
   const double tau = ko_tau(P, step);
   std::vector<double> x(m), y(m), a(m);
   for (int j = 0; j < m; ++j) {
-    x[j] = P->logit_scale * dot_half(q, st_K + (size_t)j * d, d) + position_bias(P, h, p, st_pos[j]);
+    // "New Pos" (section 4.4.2): the bias sees the entries' places in the reduced cache, which this list
+    // keeps in position order, so entry j sits at place j and the current token at place m - 1.
+    const double bias = P->pos_mode == 1 ? position_bias(P, h, m - 1, j) : position_bias(P, h, p, st_pos[j]);
+    x[j] = P->logit_scale * dot_half(q, st_K + (size_t)j * d, d) + bias;
     y[j] = (x[j] + ko_noise(P, b, l, h, p, st_pos[j])) / tau;
   }
   softmax_inplace(x.data(), a.data(), m);

@@ -38,7 +38,7 @@ class _Params(C.Structure):
     _fields_ = [
         ("head_dim", C.c_int32), ("n_heads", C.c_int32), ("budget_k", C.c_int32),
         ("recent_w", C.c_int32), ("gen_len_T", C.c_int32), ("noise_mode", C.c_int32),
-        ("bias_mode", C.c_int32), ("reserved", C.c_int32),
+        ("bias_mode", C.c_int32), ("pos_mode", C.c_int32),
         ("tau_init", C.c_double), ("tau_end", C.c_double), ("logit_scale", C.c_double),
         ("noise_const", C.c_double), ("noise_mu", C.c_double), ("noise_sigma", C.c_double),
         ("noise_seed", C.c_uint64), ("alibi_slopes", C.POINTER(C.c_double)),
@@ -115,6 +115,7 @@ class Params:
     noise_const: float = 0.5772
     noise_mu: float = 0.5772
     noise_sigma: float = 1.2825
+    pos_mode: int = 0                 # 0 original positions in the bias, 1 places within the reduced cache
     _keep: list = field(default_factory=list, repr=False)
 
     def c(self) -> _Params:
@@ -122,7 +123,7 @@ class Params:
         p = _Params()
         p.head_dim, p.n_heads, p.budget_k = self.head_dim, self.n_heads, self.budget_k
         p.recent_w, p.gen_len_T, p.noise_mode = self.recent_w, self.gen_len_T, self.noise_mode
-        p.bias_mode = self.bias_mode
+        p.bias_mode, p.pos_mode = self.bias_mode, self.pos_mode
         p.tau_init, p.tau_end, p.logit_scale = self.tau_init, self.tau_end, scale
         p.noise_const, p.noise_mu, p.noise_sigma = self.noise_const, self.noise_mu, self.noise_sigma
         p.noise_seed = self.noise_seed & 0xFFFFFFFFFFFFFFFF

@@ -463,3 +463,59 @@ def test_forced_eviction_and_forced_keep_are_applied():
     st.decode_score(1, q, kn, vn)
     ev = st.decode_evict(1, force_evict_pos=np.array([3], np.int32))
     assert ev[0] == 3 and st.pos[0, :8].tolist() == [0, 1, 2, 4, 5, 18, 19, 20]
+
+
+# ---------------------------------------------------------------- position variants (section 4.4.2)
+def test_decode_new_positions_bias_follows_the_place_in_the_reduced_cache():
+    """"New Pos": the ALiBi distance is counted in places of the reduced cache.  The reference is library
+    attention with an additive mask built here from the kept positions; with original positions the same
+    construction uses the position gaps, so the two variants must differ once tokens have been evicted."""
+    U, n, d, H = 2, 40, 16, 2
+    slopes = W.alibi_slopes(H)
+    outs = {}
+    for mode in (0, 1):
+        P = _params(budget_k=10, recent_w=3, noise_mode=ko.NOISE_NONE, tau_init=1.0, tau_end=1.0, bias_mode=1,
+                    alibi_slopes=slopes, n_heads=H, pos_mode=mode)
+        st = _prefilled(P, U, n, d, 21)
+        for s in (1, 2, 3):
+            q, kn, vn = _step_inputs(40 + s, U, d)
+            out, z = st.decode_score(s, q, kn, vn)
+            m = 11
+            p = n + s - 1
+            pos = st.pos[:, :m].astype(np.float64)
+            assert (np.diff(pos, axis=1) > 0).all() and (pos[:, -1] == p).all()
+            sl = np.array([slopes[st.lbh[u][2]] for u in range(U)])[:, None]
+            dist = (m - 1 - np.arange(m, dtype=np.float64))[None, :] if mode == 1 else p - pos
+            assert mode == 1 or (dist[:, 0] > m - 1).all()      # something was evicted: gaps exceed places
+            mask = torch.from_numpy(-sl * dist)[:, None, :]
+            Kc = torch.from_numpy(st.K[:, :m].view(np.float16).astype(np.float64))
+            Vc = torch.from_numpy(st.V[:, :m].view(np.float16).astype(np.float64))
+            ref = torch.nn.functional.scaled_dot_product_attention(
+                torch.from_numpy(q.astype(np.float64))[:, None, :], Kc, Vc, attn_mask=mask)[:, 0]
+            assert np.abs(out - ref.numpy()).max() < 1e-12
+            # zero noise, temperature 1: the score is the attention weight under the same bias
+            x = np.einsum("ud,umd->um", q.astype(np.float64), Kc.numpy()) / math.sqrt(d) - sl * dist
+            assert np.abs(z[:, :m] - torch.softmax(torch.from_numpy(x), -1).numpy()).max() < 1e-12
+            st.decode_evict(s)
+            outs[(mode, s)] = out
+    assert np.abs(outs[(0, 1)] - outs[(1, 1)]).max() > 1e-4
+
+
+def test_new_positions_equal_original_positions_until_something_is_evicted():
+    U, n, d, H = 2, 6, 16, 2
+    slopes = W.alibi_slopes(H)
+    res = []
+    for mode in (0, 1):
+        P = _params(budget_k=12, recent_w=3, noise_seed=4, bias_mode=1, alibi_slopes=slopes, n_heads=H, pos_mode=mode)
+        st = _prefilled(P, U, n, d, 22)
+        steps = []
+        for s in range(1, 9):
+            q, kn, vn = _step_inputs(60 + s, U, d)
+            out, z = st.decode_score(s, q, kn, vn)
+            st.decode_evict(s)
+            steps.append(out.copy())
+        res.append(steps)
+    for s in range(8):
+        if n + s <= 12:                # nothing evicted before this step's scoring: places are positions
+            assert np.array_equal(res[0][s], res[1][s])
+    assert not np.array_equal(res[0][7], res[1][7])
