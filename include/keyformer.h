@@ -53,7 +53,14 @@ extern "C" {
 #define KF_PREFILL_SIMT   1 /* CUDA cores; scores are summed with floating-point atomics     */
 
 #define KF_BIAS_NONE  0
-#define KF_BIAS_ALIBI 1     /* x_ij += -slope_h * (i - j) on ORIGINAL token positions (section 4.4.2) */
+#define KF_BIAS_ALIBI 1     /* x_ij += -slope_h * (i - j); which i and j is chosen by pos_mode */
+
+/* Positional information seen by the bias once the cache has been reduced (section 4.4.2). */
+#define KF_POS_ORIGINAL 0   /* i, j = positions of the tokens in the text ("Org Pos", the method's default) */
+#define KF_POS_NEW      1   /* i, j = places within the reduced cache, counted in position order ("New Pos"):
+                               the oldest kept entry is 0, the current token is the last.  Only the generation
+                               phase differs (nothing has been dropped while the prompt is scored); the noise
+                               is keyed by the original positions in both modes.                              */
 
 typedef struct kf_ctx kf_ctx;
 
@@ -80,6 +87,7 @@ typedef struct kf_config {
   int32_t prefill_impl;    /* KF_PREFILL_*                                        */
   float   noise_mu;        /* mean of KF_NOISE_GAUSS (the paper matches Gumbel's 0.5772)          */
   float   noise_sigma;     /* standard deviation of KF_NOISE_GAUSS (1.2825 in the paper)         */
+  int32_t pos_mode;        /* KF_POS_*; KF_POS_NEW keeps one more int32 per cache slot            */
 } kf_config;
 
 /* Bytes of device workspace kf_create needs for this configuration
@@ -208,6 +216,10 @@ int kf_decode_step_static(const kf_static_step* args,
  *   acc fp32 [B][H][k] (f_theta); len int32 [B][H] (entries in use).  Any may be NULL. */
 int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V,
                   const int32_t** d_pos, const float** d_acc, const int32_t** d_len);
+
+/* KF_POS_NEW only: borrowed DEVICE pointer to the places, int32 [B][H][k]; entry j of a unit holds the
+ * number of entries of that unit with a smaller position.  KF_EINVAL in the other mode. */
+int kf_view_place(kf_ctx* ctx, int32_t layer, const int32_t** d_place);
 
 /* Checkpoint of one layer's cache (section 3.3: the reduced KV cache and f_theta are the whole state the
  * method carries from step to step).  kf_state_bytes gives the size of one layer's image: K, V, f_theta,

@@ -18,11 +18,12 @@ KF_OK, KF_EINVAL, KF_ENOSPC, KF_ESTATE, KF_ECUDA, KF_ETIMEOUT, KF_EBOUNDS = 0, -
 KF_NOISE_GUMBEL, KF_NOISE_NONE, KF_NOISE_CONST, KF_NOISE_GAUSS = 0, 1, 2, 3
 KF_BIAS_NONE, KF_BIAS_ALIBI = 0, 1
 KF_PREFILL_TENSOR, KF_PREFILL_SIMT = 0, 1
+KF_POS_ORIGINAL, KF_POS_NEW = 0, 1
 
 EXPORTS = ("kf_workspace_bytes", "kf_create", "kf_prefill_score_prune", "kf_decode_step",
            "kf_decode_step_host", "kf_view_state", "kf_poll_error", "kf_launch_count",
            "kf_destroy", "kf_strerror", "kf_decode_step_static", "kf_state_bytes", "kf_export_state", "kf_import_state",
-           "kf_prefill_attend", "kf_prefill_attend_score_prune")
+           "kf_prefill_attend", "kf_prefill_attend_score_prune", "kf_view_place")
 
 
 class kf_config(C.Structure):
@@ -33,7 +34,7 @@ class kf_config(C.Structure):
         ("noise_mode", C.c_int32), ("bias_mode", C.c_int32), ("h_alibi_slopes", C.POINTER(C.c_float)),
         ("logit_scale", C.c_float), ("noise_const", C.c_float),
         ("decode_splits", C.c_int32), ("prefill_impl", C.c_int32),
-        ("noise_mu", C.c_float), ("noise_sigma", C.c_float),
+        ("noise_mu", C.c_float), ("noise_sigma", C.c_float), ("pos_mode", C.c_int32),
     ]
 
 
@@ -79,6 +80,8 @@ def _load() -> C.CDLL:
     lib.kf_export_state.argtypes = [vp, i32, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32), vp]
     lib.kf_import_state.restype = C.c_int
     lib.kf_import_state.argtypes = [vp, i32, vp, C.c_size_t, i32, i32, vp]
+    lib.kf_view_place.restype = C.c_int
+    lib.kf_view_place.argtypes = [vp, i32, C.POINTER(vp)]
     lib.kf_view_state.restype = C.c_int
     lib.kf_view_state.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
     lib.kf_poll_error.restype = C.c_int
@@ -114,7 +117,7 @@ def kf_strerror(code: int) -> str:
 def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_prompt_len, gen_len_T,
                 tau_init=1.0, tau_end=2.0, noise_seed=0, noise_mode=KF_NOISE_GUMBEL, bias_mode=KF_BIAS_NONE,
                 alibi_slopes=None, logit_scale=0.0, noise_const=0.5772, decode_splits=0,
-                prefill_impl=KF_PREFILL_TENSOR, noise_mu=0.5772, noise_sigma=1.2825):
+                prefill_impl=KF_PREFILL_TENSOR, noise_mu=0.5772, noise_sigma=1.2825, pos_mode=KF_POS_ORIGINAL):
     """Fill a kf_config; returns (config, keepalive) where keepalive holds the slopes array."""
     cfg = kf_config()
     cfg.n_layers, cfg.batch, cfg.n_heads, cfg.head_dim = n_layers, batch, n_heads, head_dim
@@ -129,6 +132,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
     cfg.logit_scale, cfg.noise_const = logit_scale, noise_const
     cfg.decode_splits, cfg.prefill_impl = decode_splits, prefill_impl
     cfg.noise_mu, cfg.noise_sigma = noise_mu, noise_sigma
+    cfg.pos_mode = pos_mode
     return cfg, keep
 
 
@@ -258,6 +262,14 @@ class Keyformer:
         acc = view(ptrs[3], B * H * k * 4, torch.float32, (B, H, k))
         ln = view(ptrs[4], B * H * 4, torch.int32, (B, H))
         return K, V, pos, acc, ln
+
+    def kf_view_place(self, layer):
+        """Zero-copy torch view of one layer's places (KF_POS_NEW only), int32 [B, H, k]."""
+        ptr = C.c_void_p()
+        _check(LIB.kf_view_place(self._h, layer, C.byref(ptr)), "kf_view_place")
+        B, H, k = self.cfg.batch, self.cfg.n_heads, self.cfg.budget_k
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + B * H * k * 4].view(torch.int32).view(B, H, k)
 
     def kf_state_bytes(self) -> int:
         return int(LIB.kf_state_bytes(self._h))

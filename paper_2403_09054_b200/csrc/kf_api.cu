@@ -18,6 +18,7 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
   size_t K, V, acc, pos, len;          // per-layer strides are kv_layer / sc_layer / len_layer
+  size_t place;                        // KF_POS_NEW only (sc_layer per layer)
   size_t y_scratch, partials, err, slopes;
   size_t acc_full, idx, staging, lse2, lse_x;
   size_t total;
@@ -38,6 +39,7 @@ bool config_ok(const kf_config* c) {
   if (c->bias_mode == KF_BIAS_ALIBI && !c->h_alibi_slopes) return false;
   if (c->logit_scale < 0.f || c->decode_splits < 0 || c->decode_splits > kf::decode_max_splits()) return false;
   if (c->prefill_impl != KF_PREFILL_TENSOR && c->prefill_impl != KF_PREFILL_SIMT) return false;
+  if (c->pos_mode != KF_POS_ORIGINAL && c->pos_mode != KF_POS_NEW) return false;
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
   return true;
 }
@@ -68,6 +70,7 @@ Layout make_layout(const kf_config* c) {
   L.staging = off; off += 8 * align_up(units * d * 2);   // two sets of (q, k_new, v_new, out)
   L.lse2 = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
   L.lse_x = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
+  L.place = off; if (c->pos_mode == KF_POS_NEW) off += nl * L.sc_layer;
   L.total = off;
   return L;
 }
@@ -194,6 +197,7 @@ static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt
   G.Vc = reinterpret_cast<__half*>(ctx->ws + L.V + (size_t)layer * L.kv_layer);
   G.pos = reinterpret_cast<int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer);
   G.acc = reinterpret_cast<float*>(ctx->ws + L.acc + (size_t)layer * L.sc_layer);
+  G.place = c.pos_mode == KF_POS_NEW ? reinterpret_cast<int32_t*>(ctx->ws + L.place + (size_t)layer * L.sc_layer) : nullptr;
   G.n = n_prompt; G.k = c.budget_k;
   if (kf::launch_prefill_gather(G, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
 
@@ -265,6 +269,7 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.acc = reinterpret_cast<float*>(ctx->ws + L.acc + (size_t)layer * L.sc_layer);
   P.pos = reinterpret_cast<int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer);
   P.len = reinterpret_cast<int32_t*>(ctx->ws + L.len + (size_t)layer * L.len_layer);
+  P.place = c.pos_mode == KF_POS_NEW ? reinterpret_cast<int32_t*>(ctx->ws + L.place + (size_t)layer * L.sc_layer) : nullptr;
   P.q = static_cast<const __half*>(d_q);
   P.knew = static_cast<const __half*>(d_knew);
   P.vnew = static_cast<const __half*>(d_vnew);
@@ -429,6 +434,12 @@ int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V
   return KF_OK;
 }
 
+int kf_view_place(kf_ctx* ctx, int32_t layer, const int32_t** d_place) {
+  if (!ctx || !d_place || layer < 0 || layer >= ctx->cfg.n_layers || ctx->cfg.pos_mode != KF_POS_NEW) return KF_EINVAL;
+  *d_place = reinterpret_cast<const int32_t*>(ctx->ws + ctx->lay.place + (size_t)layer * ctx->lay.sc_layer);
+  return KF_OK;
+}
+
 size_t kf_state_bytes(const kf_ctx* ctx) {
   if (!ctx) return 0;
   const Layout& L = ctx->lay;
@@ -472,6 +483,16 @@ int kf_import_state(kf_ctx* ctx, int32_t layer, const void* d_src, size_t bytes,
   const int rc = copy_state(ctx, layer, const_cast<unsigned char*>(static_cast<const unsigned char*>(d_src)), false,
                             static_cast<cudaStream_t>(stream));
   if (rc != KF_OK) return rc;
+  if (ctx->cfg.pos_mode == KF_POS_NEW) {
+    // the image carries positions only: the places follow from them
+    const Layout& L = ctx->lay;
+    if (kf::launch_rebuild_place(reinterpret_cast<const int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer),
+                                 reinterpret_cast<const int32_t*>(ctx->ws + L.len + (size_t)layer * L.len_layer),
+                                 reinterpret_cast<int32_t*>(ctx->ws + L.place + (size_t)layer * L.sc_layer),
+                                 ctx->cfg.budget_k, L.units, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+      return KF_ECUDA;
+    ctx->launches += 1;
+  }
   ctx->n_prompt[layer] = n_prompt;
   ctx->last_step[layer] = last_step;
   return KF_OK;

@@ -206,6 +206,16 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
       return;
     }
   }
+  if (P.place) {
+    // the entries behind the one that leaves move up one place; the new token takes the last place
+    int32_t* __restrict__ place = P.place + (size_t)u * P.k;
+    if (len >= P.k) {
+      const int pos_out = (int)(0xffffffffu - (uint32_t)best);   // the key's low word is 2^32 - 1 - position
+      for (int j = tid; j < len; j += NT)
+        if (j != slot && pos[j] > pos_out) place[j] -= 1;
+    }
+    if (tid == 0) place[slot] = len < P.k ? len : P.k - 1;
+  }
   if (tid == 0) { pos[slot] = P.p; acc[slot] = z_new; }
   __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + slot) * D;
   __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + slot) * D;
@@ -239,7 +249,7 @@ __device__ __forceinline__ void dot8_mixed(float& acc, const uint4& kv, const ui
   }
 }
 
-template <int D, int NW, int NSTAGE>
+template <int D, int NW, int NSTAGE, bool NEWPOS>
 __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__ DecodeParams P) {
   constexpr int CPR = D / 8;          // 16-byte chunks per row
   constexpr int LPR = CPR;            // lanes that share one row in the value phase
@@ -305,9 +315,13 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
 #pragma unroll
   for (int c = 0; c < 8; ++c) o[c] = 0.f;
   int pos_next = 0;
+  // "New Pos": the bias counts places within the cache; the current token stands at place len
+  const int32_t* place_u = NEWPOS ? P.place + (size_t)u * P.k : nullptr;
+  int place_next = 0;
   if (my_tiles > 0) {
     const int tb = tile_base_of(0);
     pos_next = (tb + lane < row_end) ? pos_u[tb + lane] : 0;
+    if (NEWPOS) place_next = (tb + lane < row_end) ? place_u[tb + lane] : 0;
   }
 
   int consumed = 0;  // ring items whose slot has been released
@@ -315,9 +329,11 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
     const int tile_base = tile_base_of(ti);
     const int rows = min(TILE_ROWS, row_end - tile_base);
     const int pj = pos_next;
+    const int dist = NEWPOS ? len - place_next : P.p - pj;   // distance between the query and this key in the bias
     if (ti + 1 < my_tiles) {
       const int tb = tile_base_of(ti + 1);
       pos_next = (tb + lane < row_end) ? pos_u[tb + lane] : 0;
+      if (NEWPOS) place_next = (tb + lane < row_end) ? place_u[tb + lane] : 0;
     }
 
     // ---- logits: lane r computes x of row tile_base + r.  Chunks are visited in a rotated
@@ -352,7 +368,7 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
     const bool valid = lane < rows;
     float x = -INFINITY, y = -INFINITY;
     if (valid) {
-      x = fmaf(x_mine, P.scale, -slope * (float)(P.p - pj));
+      x = fmaf(x_mine, P.scale, -slope * (float)dist);
       y = (x + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)pj)) * P.inv_tau;
       P.y_scratch[(size_t)u * (P.k + 1) + tile_base + lane] = y;
     }
@@ -456,7 +472,7 @@ __global__ void __launch_bounds__(128, 8) decode_close_kernel(const __grid_const
 template <int D, int NW, int NSTAGE>
 cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   constexpr size_t smem = (size_t)NW * NSTAGE * (TILE_ROWS * D * 2) + (size_t)NW * NSTAGE * 8;
-  auto kern = decode_kernel<D, NW, NSTAGE>;
+  auto kern = P.place ? decode_kernel<D, NW, NSTAGE, true> : decode_kernel<D, NW, NSTAGE, false>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -481,7 +497,27 @@ cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   return cudaLaunchKernelEx(&cfg, decode_close_kernel<D>, P);
 }
 
+// One CTA per unit: place[j] = #{i : pos[i] < pos[j]} (positions of a unit are distinct).
+__global__ void __launch_bounds__(256) rebuild_place_kernel(const int32_t* __restrict__ pos, const int32_t* __restrict__ len,
+                                                            int32_t* __restrict__ place, int k) {
+  const int u = blockIdx.x;
+  const int n = min(len[u], k);
+  const int32_t* pu = pos + (size_t)u * k;
+  for (int j = threadIdx.x; j < n; j += blockDim.x) {
+    const int pj = pu[j];
+    int c = 0;
+    for (int i = 0; i < n; ++i) c += pu[i] < pj ? 1 : 0;
+    place[(size_t)u * k + j] = c;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_rebuild_place(const int32_t* pos, const int32_t* len, int32_t* place, int k, int units,
+                                 cudaStream_t stream) {
+  rebuild_place_kernel<<<units, 256, 0, stream>>>(pos, len, place, k);
+  return cudaGetLastError();
+}
 
 int decode_tile_rows() { return TILE_ROWS; }
 int decode_max_splits() { return MAX_SPLITS; }

@@ -11,6 +11,8 @@ struct DecodeParams {
   float* acc;             // [units][k]  accumulated score f_theta
   int32_t* pos;           // [units][k]  original token positions
   int32_t* len;           // [units]     entries in use
+  int32_t* place;         // [units][k]  place of each entry within the cache in position order, or null when the
+                          //             bias uses the original positions (section 4.4.2)
   const __half* q;        // [units][d]
   const __half* knew;     // [units][d]
   const __half* vnew;     // [units][d]
@@ -33,6 +35,10 @@ constexpr size_t STATIC_SCRATCH_BYTES = (size_t)16 << 20;
 int decode_tile_rows();
 int decode_max_splits();
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
+
+// place[j] = number of entries of the unit with a smaller position, for every unit of a layer (after a state import).
+cudaError_t launch_rebuild_place(const int32_t* pos, const int32_t* len, int32_t* place, int k, int units,
+                                 cudaStream_t stream);
 
 // Same launch with y_scratch / partials carved out of the built-in scratch block
 // (the sizes are in bytes, each a multiple of 256).  Allocates nothing.

@@ -35,6 +35,7 @@ struct GatherParams {
   __half* Vc;
   int32_t* pos;          // [units][k]
   float* acc;            // [units][k]
+  int32_t* place;        // [units][k] or null: place within the cache (= slot, the rows are stored in position order)
   int32_t n, k;
 };
 

@@ -232,6 +232,7 @@ __global__ void __launch_bounds__(128) prefill_gather(const __grid_constant__ Ga
   const int lane = threadIdx.x & 31;
   if (slot >= P.k) return;
   const int j = P.idx[(size_t)u * P.k + slot];
+  if (P.place && lane == 0) P.place[(size_t)u * P.k + slot] = slot;
   uint4* Kd = reinterpret_cast<uint4*>(P.Kc + ((size_t)u * P.k + slot) * D);
   uint4* Vd = reinterpret_cast<uint4*>(P.Vc + ((size_t)u * P.k + slot) * D);
   if (j < 0 || j >= P.n) {

@@ -26,10 +26,10 @@ SCORE_ATOL = 1e-7
 BAND = 1e-3
 
 
-def oracle_params(wl: W.Workload, noise_mode=ko.NOISE_GUMBEL, logit_scale=0.0) -> ko.Params:
+def oracle_params(wl: W.Workload, noise_mode=ko.NOISE_GUMBEL, logit_scale=0.0, pos_mode=0) -> ko.Params:
     return ko.Params(head_dim=wl.head_dim, n_heads=wl.n_heads, budget_k=wl.budget_k, recent_w=wl.recent_w,
                      gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end,
-                     noise_seed=wl.noise_seed, noise_mode=noise_mode, logit_scale=logit_scale,
+                     noise_seed=wl.noise_seed, noise_mode=noise_mode, logit_scale=logit_scale, pos_mode=pos_mode,
                      bias_mode=1 if wl.positional == "alibi" else 0,
                      alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None)
 
@@ -64,12 +64,13 @@ class LockStep:
     """One layer of a workload on the GPU next to the oracle on a sample of its units."""
 
     def __init__(self, wl: W.Workload, gpu: kf.Keyformer, layer: int, units: np.ndarray,
-                 noise_mode=ko.NOISE_GUMBEL, logit_scale=0.0):
+                 noise_mode=ko.NOISE_GUMBEL, logit_scale=0.0, pos_mode=0):
         self.wl, self.gpu, self.layer = wl, gpu, layer
+        self.pos_mode = pos_mode
         self.units = np.ascontiguousarray(units, dtype=np.int32).reshape(-1, 3)
         assert (self.units[:, 0] == layer).all()
         self.flat = torch.as_tensor(self.units[:, 1] * wl.n_heads + self.units[:, 2], dtype=torch.long)
-        self.P = oracle_params(wl, noise_mode, logit_scale)
+        self.P = oracle_params(wl, noise_mode, logit_scale, pos_mode)
         self.st = ko.State(self.P, self.units)
         self.adoptions = 0
         self.n = None
@@ -184,6 +185,12 @@ class LockStep:
                 own[u] = int(ref_pos[~keep][0])
         self.adoptions += int((forced != own).sum())
         self.st.decode_evict(step, force_evict_pos=forced if (forced >= 0).any() else None)
+        if check_state and self.pos_mode == 1:
+            # the places the bias will use next step: rank of each entry's position within its unit
+            place = self._rows(self.gpu.kf_view_place(self.layer))
+            for u in range(U):
+                La = int(len_after[u])
+                assert (place[u, :La] == np.argsort(np.argsort(pos_after[u, :La]))).all(), f"step {step}: places out of order"
         if check_state:
             for u in range(U):
                 La = int(len_after[u])
@@ -199,18 +206,18 @@ class LockStep:
 
 
 def run_workload(wl: W.Workload, units_per_layer=None, steps=None, layers=None, device="cuda:0",
-                 sample_seed=0, check_state_every=1, gpu_kwargs=None, noise="gumbel", logit_scale=0.0):
+                 sample_seed=0, check_state_every=1, gpu_kwargs=None, noise="gumbel", logit_scale=0.0, pos_mode=0):
     """Prefill + `steps` decode steps of `wl` on the GPU in lock step with the oracle.
     Returns a dict of summary numbers."""
     nm_gpu = {"gumbel": kf.KF_NOISE_GUMBEL, "none": kf.KF_NOISE_NONE, "const": kf.KF_NOISE_CONST, "gauss": kf.KF_NOISE_GAUSS}[noise]
     nm_ref = {"gumbel": ko.NOISE_GUMBEL, "none": ko.NOISE_NONE, "const": ko.NOISE_CONST, "gauss": ko.NOISE_GAUSS}[noise]
-    gpu = make_gpu(wl, noise_mode=nm_gpu, logit_scale=logit_scale, **(gpu_kwargs or {}))
+    gpu = make_gpu(wl, noise_mode=nm_gpu, logit_scale=logit_scale, pos_mode=pos_mode, **(gpu_kwargs or {}))
     layers = list(range(wl.n_layers)) if layers is None else layers
     steps = wl.gen_len_T if steps is None else steps
     drivers = []
     for l in layers:
         units = W.unit_list(wl, l) if units_per_layer is None else W.sample_units(wl, units_per_layer, sample_seed + l, l)
-        ls = LockStep(wl, gpu, l, units, noise_mode=nm_ref, logit_scale=logit_scale)
+        ls = LockStep(wl, gpu, l, units, noise_mode=nm_ref, logit_scale=logit_scale, pos_mode=pos_mode)
         q, k, v = W.make_prompt(wl, l, device)
         ls.prefill(q, k, v)
         del q, k, v

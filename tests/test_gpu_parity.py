@@ -127,6 +127,51 @@ def test_alibi_and_rotary_workloads_scaled_down():
     lockstep.run_workload(W.get_config("c2_gptj").scaled(n_heads=2, prompt_len=300, budget_k=150, recent_w=37, gen_len_T=10))
 
 
+@pytest.mark.parametrize("d,n,k,w", [(128, 600, 300, 75), (64, 200, 96, 0), (256, 150, 40, 40), (128, 40, 64, 16)])
+def test_new_positions_in_the_bias(d, n, k, w):
+    """"New Pos" (section 4.4.2) with ALiBi: the bias distance is the place within the reduced cache.  Covers
+    several splits, no recent window, window = budget, and a cache that only fills up during generation."""
+    wl = W.get_config("c3_mpt").scaled(n_heads=4, head_dim=d, prompt_len=n, budget_k=k, recent_w=w, gen_len_T=30)
+    r = lockstep.run_workload(wl, pos_mode=1)
+    assert r["steps"] == 30
+
+
+def test_new_positions_differ_from_original_positions_and_survive_import():
+    wl = W.get_config("c3_mpt").scaled(n_heads=4, batch=2, prompt_len=300, budget_k=128, recent_w=32, gen_len_T=12)
+    q, k, v = W.make_prompt(wl, 0, DEV)
+
+    def run(gpu, first, last):
+        outs = []
+        for s in range(first, last + 1):
+            qs, kn, vn = W.make_step(wl, 0, s, DEV)
+            out = torch.empty_like(qs)
+            gpu.kf_decode_step(0, s, qs, kn, vn, out)
+            outs.append(out)
+        return outs
+
+    org = lockstep.make_gpu(wl)
+    org.kf_prefill_score_prune(0, q, k, v)
+    with pytest.raises(kf.KeyformerError) as e:
+        org.kf_view_place(0)
+    assert e.value.code == kf.KF_EINVAL
+    new = lockstep.make_gpu(wl, pos_mode=kf.KF_POS_NEW)
+    new.kf_prefill_score_prune(0, q, k, v)
+    o_org, o_new = run(org, 1, 6), run(new, 1, 6)
+    assert not torch.equal(o_org[0], o_new[0])          # 172 prompt tokens are gone: distances shrink
+    img = torch.empty(new.kf_state_bytes(), dtype=torch.uint8, device=DEV)
+    n_prompt, last_step = new.kf_export_state(0, img)
+    rest = run(new, 7, 12)
+    again = lockstep.make_gpu(wl, pos_mode=kf.KF_POS_NEW)
+    again.kf_import_state(0, img, n_prompt, last_step)     # the places are rebuilt from the positions
+    for x, y in zip(run(again, 7, 12), rest):
+        assert torch.equal(x, y)
+    torch.cuda.synchronize()
+    assert torch.equal(again.kf_view_place(0), new.kf_view_place(0))
+    pos = new.kf_view_state(0)[2]
+    assert torch.equal(new.kf_view_place(0).long(), pos.argsort(-1).argsort(-1))
+    assert org.kf_poll_error() == 0 and new.kf_poll_error() == 0 and again.kf_poll_error() == 0
+
+
 def test_heavy_hitter_multi_layer_scaled_down():
     wl = W.get_config("c4_cerebras").scaled(n_layers=3, batch=2, n_heads=4, prompt_len=400, budget_k=200, recent_w=50, gen_len_T=8)
     lockstep.run_workload(wl)
