@@ -210,7 +210,8 @@ def run_ours(args, wl):
                        gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
                        bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
                        alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None,
-                       decode_splits=args.splits)
+                       decode_splits=args.splits,
+                       pos_mode=kf.KF_POS_NEW if args.new_pos else kf.KF_POS_ORIGINAL)
     t_pre = time.perf_counter()
     for l in range(wl.n_layers):
         q, k, v = W.make_prompt(wl_r, l, dev)
@@ -311,6 +312,7 @@ def run_ours(args, wl):
                        "l2": ("inputs larger than L2 (KV state %.1f GB per GPU)" if kv_bytes > 126e6 else
                               "KV state of this workload (%.3f GB) fits L2: cache-resident by nature, no flush") % (kv_bytes / 1e9),
                        "prefill_s": t_pre, "decode_splits": args.splits,
+                       "positions_in_bias": "places within the reduced cache" if args.new_pos else "original",
                        "launch_mode": "one CUDA graph of the timed steps" if args.graph else "stream launches"},
             "roofline": {"bound": "hbm", "kernel": "decode_kernel (+ decode_close_kernel: the duration is one layer call)", "achieved": achieved, "peak": peaks["hbm_gbs"],
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
@@ -440,6 +442,8 @@ def main():
     ap.add_argument("--budget-frac", type=float, default=0.5, help="prefill phase: k as a fraction of the prompt")
     ap.add_argument("--with-attention", action="store_true",
                     help="prefill phase: kf_prefill_attend_score_prune (also produces the prompt's attention output)")
+    ap.add_argument("--new-pos", action="store_true",
+                    help="decode phase: the bias counts places within the reduced cache (only matters with ALiBi workloads)")
     ap.add_argument("--prefill-simt", action="store_true", help="prefill phase: CUDA-core scoring instead of tcgen05")
     args = ap.parse_args()
     wl = W.get_config(args.workload)

@@ -211,8 +211,20 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
     int32_t* __restrict__ place = P.place + (size_t)u * P.k;
     if (len >= P.k) {
       const int pos_out = (int)(0xffffffffu - (uint32_t)best);   // the key's low word is 2^32 - 1 - position
-      for (int j = tid; j < len; j += NT)
-        if (j != slot && pos[j] > pos_out) place[j] -= 1;
+      for (int j0 = tid; j0 < len; j0 += NT * BATCH) {   // loads of a batch first, so that they overlap
+        int pp[BATCH], pl[BATCH];
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+          const int j = j0 + i * NT;
+          pp[i] = j < len ? pos[j] : -1;
+          pl[i] = j < len ? place[j] : 0;
+        }
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+          const int j = j0 + i * NT;
+          if (j != slot && pp[i] > pos_out) place[j] = pl[i] - 1;   // pp = -1 beyond the end never passes
+        }
+      }
     }
     if (tid == 0) place[slot] = len < P.k ? len : P.k - 1;
   }
