@@ -39,9 +39,15 @@ def test_workspace_size_covers_the_cache():
     assert nbytes >= kv and nbytes % 256 == 0
 
 
+def test_new_positions_cost_one_int32_per_slot():
+    base, new = kf.kf_workspace_bytes(_cfg()), kf.kf_workspace_bytes(_cfg(pos_mode=kf.KF_POS_NEW))
+    assert new - base == 2 * 2 * 4 * 64 * 4          # layers x batch x heads x k x sizeof(int32), already 256-aligned
+
+
 @pytest.mark.parametrize("bad", [dict(head_dim=96), dict(budget_k=0), dict(recent_w=65), dict(recent_w=-1),
                                  dict(tau_init=0.0), dict(tau_end=-1.0), dict(n_layers=0), dict(gen_len_T=-1),
-                                 dict(noise_mode=7), dict(bias_mode=1), dict(max_prompt_len=0)])
+                                 dict(noise_mode=7), dict(bias_mode=1), dict(max_prompt_len=0), dict(pos_mode=2),
+                                 dict(pos_mode=-1)])
 def test_invalid_configurations_are_rejected(bad):
     assert kf.kf_workspace_bytes(_cfg(**bad)) == 0
 
