@@ -25,6 +25,13 @@ def test_config3_mpt_sampled_units():
     print("c3", r)
 
 
+def test_config3_mpt_new_positions_sampled_units():
+    """The ALiBi workload at full size with the bias counted in places of the reduced cache (section 4.4.2)."""
+    wl = W.get_config("c3_mpt")
+    r = lockstep.run_workload(wl, units_per_layer=4, steps=8, check_state_every=4, pos_mode=1)
+    print("c3 new positions", r)
+
+
 def test_config4_cerebras_first_and_last_layer_sampled_units():
     wl = W.get_config("c4_cerebras")
     r = lockstep.run_workload(wl, units_per_layer=8, steps=6, layers=[0, wl.n_layers - 1], check_state_every=3)
