@@ -49,6 +49,7 @@ struct PrefillTcParams {
   const float* slopes; // [H] or null
   int* err;
   int32_t n, nblk, H, layer;
+  int32_t units;       // (batch row, head) pairs of the call
   float a_scale;       // logit scale * log2(e) / tau
   float ax;            // logit scale * log2(e)
   float c1;            // log2(e) / tau

@@ -13,12 +13,17 @@
 //            thread sums z_ij = 2^(y2_ij - lse2[i]) over the queries i >= j in a register and
 //            stores f_theta(j) directly: no atomics, a reproducible summation order.
 //
-// One CTA owns a block of 128 rows of the resident operand and streams 128-row tiles of the
-// other one through a ring of shared-memory stages.  Warp 0 issues the TMA loads (128-byte
-// swizzled boxes, one copy per CTA), warp 1 owns tensor memory and issues the MMAs, the other warps are
-// groups of four compute warps that take accumulator tiles in turn (a warp can read
-// the 32 accumulator lanes selected by warp id mod 4).  Every wait is bounded; a wait that runs
-// out raises the error word and the CTA drains and frees tensor memory before it leaves.
+// A work item is a block of 128 rows of the resident operand together with the 128-row tiles of the
+// other operand it meets under the causal mask, streamed through a ring of shared-memory stages.
+// The grid is persistent (one CTA per SM): every CTA walks a fixed list of items, long and short
+// ones paired so that all lists weigh the same, and its pipeline keeps running across the items --
+// the loads and MMAs of the next item are issued while the compute warps still work on the
+// accumulator tiles of the current one, so no SM idles through a prologue per item.
+// Warp 0 issues the TMA loads (128-byte swizzled boxes, one copy per CTA), warp 1 owns tensor
+// memory and issues the MMAs, the other warps are groups of four compute warps that take
+// accumulator tiles in turn (a warp can read the 32 accumulator lanes selected by warp id mod 4).
+// Every wait is bounded; a wait that runs out raises the error word and the CTA drains and frees
+// tensor memory before it leaves.
 #include "kf_prefill.cuh"
 #include "kf_tc.cuh"
 
@@ -41,6 +46,7 @@ constexpr int TC_NG = KF_TC_NG;               // compute groups for head_dim 64 
 constexpr int TC_NACC = 4;                    // accumulator buffers: 4 x 128 columns = all of tensor memory
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr int TC_XBUF_FLOATS = 4 * 32 * 4;    // per warp: 4 noise calls x 32 lanes x 4 words
+__host__ __device__ constexpr int tc_comb_buffers(int d) { return d == 256 ? 2 : 4; }   // what the shared memory left over allows
 constexpr float LG2_LN2 = -0.5287663729448977f;  // log2(ln 2)
 
 // Instruction descriptor: binary16 A and B, both K-major, binary32 accumulator, M = 128, N = 128.
@@ -105,34 +111,54 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
   constexpr int NCW = 4 * NG;                                // compute warps
   float* xbuf = reinterpret_cast<float*>(sS + (size_t)NST * OP_BYTES);  // [NCW][TC_XBUF_FLOATS] noise exchange
   float* lse_s = xbuf + NCW * TC_XBUF_FLOATS;                // [NCW][128] lse2 of the current query tile
-  float* comb = lse_s + NCW * 128;                           // [NG - 1][4][128] hand-over between the compute groups
-  uint64_t* bars = reinterpret_cast<uint64_t*>(comb + (NG - 1) * 4 * 128);
+  constexpr int COMB_FLOATS = NG * 4 * 128;
+  constexpr int NCB = tc_comb_buffers(D);                    // items whose hand-over may be pending at one time
+  float* comb = lse_s + NCW * 128;                           // [NCB][NG][4][128] hand-over between the compute groups
+  uint64_t* bars = reinterpret_cast<uint64_t*>(comb + NCB * COMB_FLOATS);
   uint64_t* r_full = bars;
-  uint64_t* s_full = bars + 1;
+  uint64_t* r_empty = bars + 1;
+  uint64_t* s_full = bars + 2;
   uint64_t* s_empty = s_full + NST;
   uint64_t* t_full = s_empty + NST;
   uint64_t* t_empty = t_full + TC_NACC;
   uint64_t* drain = t_empty + TC_NACC;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  uint64_t* c_full = drain + 1;
+  uint64_t* c_empty = c_full + NCB;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(c_empty + NCB);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* issued_slot = const_cast<int*>(abort_flag) + 1;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int u = blockIdx.y;
   const int nblk = P.nblk;
-  const int Rb = SWEEP2 ? (int)blockIdx.x : nblk - 1 - (int)blockIdx.x;   // the longest CTAs of a unit start first
-  const int t_begin = SWEEP2 ? Rb : 0;
-  const int n_tiles = SWEEP2 ? nblk - Rb : Rb + 1;
   const CUtensorMap* mapR = SWEEP2 ? &P.tmK : &P.tmQ;
   const CUtensorMap* mapS = SWEEP2 ? &P.tmQ : &P.tmK;
 
+  // The items of this CTA.  All (unit, block) pairs are listed unit by unit, the blocks of a unit in the
+  // order longest, shortest, second longest, second shortest, ...; the list is cut into chunks of two
+  // (together nblk + 1 tiles, whatever the pair) and chunk q belongs to CTA q mod gridDim.x.  Consecutive
+  // chunks belong to the same few units, so the CTAs running at one time share their operands in L2.
+  const long long n_items = (long long)P.units * nblk;
+  auto item_at = [&](int k, int& u, int& Rb) -> bool {
+    const long long e = 2 * ((long long)blockIdx.x + (long long)(k >> 1) * gridDim.x) + (k & 1);
+    if (e >= n_items) return false;
+    u = (int)(e / nblk);
+    const int z = (int)(e % nblk);
+    const int r = (z & 1) ? nblk - 1 - (z >> 1) : (z >> 1);   // rank by length, 0 = longest
+    Rb = SWEEP2 ? r : nblk - 1 - r;
+    return true;
+  };
+  auto tiles_of = [&](int Rb) { return SWEEP2 ? nblk - Rb : Rb + 1; };
+
   if (tid == 0) {
     mbar_init(r_full, 1);
+    mbar_init(r_empty, 1);
     for (int s = 0; s < NST; ++s) { mbar_init(s_full + s, 1); mbar_init(s_empty + s, 1); }
     for (int a = 0; a < TC_NACC; ++a) { mbar_init(t_full + a, 1); mbar_init(t_empty + a, 4); }
     mbar_init(drain, 1);
+    for (int cb = 0; cb < NCB; ++cb) { mbar_init(c_full + cb, (NG - 1) * 4); mbar_init(c_empty + cb, 4); }
     *abort_flag = 0;
-    *issued_slot = 0;
+    issued_slot[0] = 0;
+    issued_slot[1] = 0;
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -155,42 +181,55 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(r_full, OP_BYTES);
-      for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sR + kc * TC_BOX_BYTES, mapR, kc * 64, Rb * TC_BM, u, r_full);
-      int it = 0;
-      for (; it < n_tiles; ++it) {
-        const int s = it % NST;
-        if (it >= NST && !wait_bar(s_empty + s, (uint32_t)((it / NST - 1) & 1), abort_flag)) {
-          *abort_flag = 1;
-          atomicExch(P.err, ERR_TIMEOUT);
-          break;
+      int gt = 0, k = 0;     // streamed tiles and items issued so far
+      bool ok = true;
+      for (int u, Rb; ok && item_at(k, u, Rb); ++k) {
+        // the resident block may be replaced once the MMAs of the previous item have read it
+        if (k > 0 && !wait_bar(r_empty, (uint32_t)((k - 1) & 1), abort_flag)) { ok = false; break; }
+        mbar_expect_tx(r_full, OP_BYTES);
+        for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sR + kc * TC_BOX_BYTES, mapR, kc * 64, Rb * TC_BM, u, r_full);
+        issued_slot[1] = k + 1;
+        const int t_begin = SWEEP2 ? Rb : 0, n_tiles = tiles_of(Rb);
+        for (int it = 0; it < n_tiles; ++it, ++gt) {
+          const int s = gt % NST;
+          if (gt >= NST && !wait_bar(s_empty + s, (uint32_t)((gt / NST - 1) & 1), abort_flag)) { ok = false; break; }
+          mbar_expect_tx(s_full + s, OP_BYTES);
+          unsigned char* dst = sS + (size_t)s * OP_BYTES;
+          for (int kc = 0; kc < KCH; ++kc) tma_load_3d(dst + kc * TC_BOX_BYTES, mapS, kc * 64, (t_begin + it) * TC_BN, u, s_full + s);
         }
-        mbar_expect_tx(s_full + s, OP_BYTES);
-        unsigned char* dst = sS + (size_t)s * OP_BYTES;
-        for (int kc = 0; kc < KCH; ++kc) tma_load_3d(dst + kc * TC_BOX_BYTES, mapS, kc * 64, (t_begin + it) * TC_BN, u, s_full + s);
       }
-      *issued_slot = it;
+      if (!ok) {
+        *abort_flag = 1;
+        atomicExch(P.err, ERR_TIMEOUT);
+      }
+      issued_slot[0] = gt;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      bool ok = wait_bar(r_full, 0, abort_flag);
+      bool ok = true;
       const uint32_t r_addr = smem_u32(sR);
-      for (int it = 0; ok && it < n_tiles; ++it) {
-        const int s = it % NST, a = it % TC_NACC;
-        ok = wait_bar(s_full + s, (uint32_t)((it / NST) & 1), abort_flag);
-        if (ok && it >= TC_NACC) ok = wait_bar(t_empty + a, (uint32_t)((it / TC_NACC - 1) & 1), abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t s_addr = smem_u32(sS + (size_t)s * OP_BYTES);
-        const uint32_t d_addr = tmem_base + (uint32_t)(a * TC_BN);
+      int gt = 0;
+      for (int k = 0, u, Rb; ok && item_at(k, u, Rb); ++k) {
+        ok = wait_bar(r_full, (uint32_t)(k & 1), abort_flag);
+        const int n_tiles = tiles_of(Rb);
+        for (int it = 0; ok && it < n_tiles; ++it, ++gt) {
+          const int s = gt % NST, a = gt % TC_NACC;
+          ok = wait_bar(s_full + s, (uint32_t)((gt / NST) & 1), abort_flag);
+          if (ok && gt >= TC_NACC) ok = wait_bar(t_empty + a, (uint32_t)((gt / TC_NACC - 1) & 1), abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t s_addr = smem_u32(sS + (size_t)s * OP_BYTES);
+          const uint32_t d_addr = tmem_base + (uint32_t)(a * TC_BN);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (uint32_t)((kk >> 2) * TC_BOX_BYTES + (kk & 3) * 32);  // box, then 16 columns = 32 bytes
-          umma_f16(d_addr, umma_smem_desc(r_addr + off), umma_smem_desc(s_addr + off), UMMA_IDESC, kk > 0 ? 1u : 0u);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (uint32_t)((kk >> 2) * TC_BOX_BYTES + (kk & 3) * 32);  // box, then 16 columns = 32 bytes
+            umma_f16(d_addr, umma_smem_desc(r_addr + off), umma_smem_desc(s_addr + off), UMMA_IDESC, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(s_empty + s);   // the stage may be refilled once these MMAs have read it
+          umma_commit(t_full + a);    // the accumulator tile is complete
         }
-        umma_commit(s_empty + s);   // the stage may be refilled once these MMAs have read it
-        umma_commit(t_full + a);    // the accumulator tile is complete
+        if (ok) umma_commit(r_empty); // the resident block may be replaced once this item's MMAs have read it
       }
       if (!ok) {
         *abort_flag = 1;
@@ -202,35 +241,58 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
   } else {
     // ------------------------------------------------------------ compute warps
     const int cw = warp - 2;            // 0..7
-    const int grp = cw >> 2;            // which accumulator tiles: it = grp, grp + NG, ...
+    const int grp = cw >> 2;            // takes the accumulator tiles whose running index is grp mod NG
     const int quarter = warp & 3;       // accumulator lanes this warp may read
     const int row = quarter * 32 + lane;               // row of the resident block owned by this thread
-    const int g_row = Rb * TC_BM + row;                // query i (sweep 1) or key j (sweep 2)
-    const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
     const float A = P.a_scale;
     const float n_mult = NOISE == NOISE_GAUSS_T ? P.gauss_scale : -P.inv_tau;
     const float n_off = NOISE == NOISE_GUMBEL_T ? -P.inv_tau * LG2_LN2 : P.const_term;   // additive term common to all logits
-    float sb = 0.f;
-    if (ALIBI) sb = P.slopes[h] * P.c1;
     float* my_x = xbuf + cw * TC_XBUF_FLOATS;
     float* my_lse = lse_s + cw * 128;
-    const float* lse_u = P.lse2 + (size_t)u * nblk * TC_BN;
     bool ok = true;
 
+    // sweep 2: the lse2 values of the next tile this group will take (of this item or the next one) are requested
+    // one tile ahead; (lse_u_next, lse_t_next) say which tile they belong to
     float4 lse_next = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (SWEEP2 && grp < n_tiles) lse_next = reinterpret_cast<const float4*>(lse_u + (size_t)(t_begin + grp) * TC_BN)[lane];
+    int lse_u_next = -1, lse_t_next = -1;
+    auto fetch_lse = [&](int uu, int tt) {
+      lse_next = reinterpret_cast<const float4*>(P.lse2 + ((size_t)uu * nblk + tt) * TC_BN)[lane];
+      lse_u_next = uu; lse_t_next = tt;
+    };
 
-    for (int it = grp; it < n_tiles; it += NG) {
-      const int a = it % TC_NACC;
+    int gt_base = 0;   // streamed tiles of the items before this one: tile `it` of the item is the CTA's tile gt_base + it
+    for (int k = 0, u, Rb; item_at(k, u, Rb); ++k) {
+    const int t_begin = SWEEP2 ? Rb : 0, n_tiles = tiles_of(Rb);
+    const int g_row = Rb * TC_BM + row;                // query i (sweep 1) or key j (sweep 2)
+    const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
+    float sb = 0.f;
+    if (ALIBI) sb = P.slopes[h] * P.c1;
+    row_m = 0.f; row_l = 0.f; started = false;
+    rowx_m = 0.f; rowx_l = 0.f; started_x = false;
+    col_sum = 0.f;
+
+    // the groups take the CTA's accumulator tiles in turn, across item boundaries
+    for (int it = (grp + NG - gt_base % NG) % NG; ok && it < n_tiles; it += NG) {
+      const int gt = gt_base + it;
+      const int a = gt % TC_NACC;
       const int t = t_begin + it;
       const bool diag = (t == Rb);
       if (SWEEP2) {
+        if (lse_u_next != u || lse_t_next != t) fetch_lse(u, t);
         __syncwarp();
         reinterpret_cast<float4*>(my_lse)[lane] = lse_next;
-        if (it + NG < n_tiles) lse_next = reinterpret_cast<const float4*>(lse_u + (size_t)(t + NG) * TC_BN)[lane];
+        if (it + NG < n_tiles) {
+          fetch_lse(u, t + NG);
+        } else {
+          int u2, Rb2;
+          if (item_at(k + 1, u2, Rb2)) {
+            const int it2 = (grp + NG - (gt_base + n_tiles) % NG) % NG;
+            if (it2 < tiles_of(Rb2)) fetch_lse(u2, Rb2 + it2);   // sweep 2: an item's first tile is its diagonal one
+          }
+        }
         __syncwarp();
       }
-      ok = wait_bar(t_full + a, (uint32_t)((it / TC_NACC) & 1), abort_flag);
+      ok = wait_bar(t_full + a, (uint32_t)((gt / TC_NACC) & 1), abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -395,58 +457,75 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive(t_empty + a);
     }
+    gt_base += n_tiles;
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicExch(P.err, ERR_TIMEOUT);
     }
-    if (grp > 0) {
-      float* mine = comb + (grp - 1) * 512;
+
+    // ---- the item is complete: the group that took its last tile (most likely the last to finish) collects
+    //      the partial results of the others from a ring of hand-over buffers and stores the rows' results.
+    //      Nobody else waits for it: a group only has to find a free buffer, NCB items later.
+    const int merger = (gt_base - 1) % NG;
+    const int cb = k % NCB;
+    float* cmb = comb + cb * COMB_FLOATS;
+    if (grp != merger) {
+      if (ok && k >= NCB) ok = __all_sync(0xffffffffu, wait_bar(c_empty + cb, (uint32_t)((k / NCB - 1) & 1), abort_flag));
+      float* mine = cmb + grp * 512;
       mine[row] = SWEEP2 ? col_sum : row_m;
       mine[128 + row] = row_l;
       mine[256 + row] = rowx_m;
       mine[384 + row] = rowx_l;
-    }
-  }
-
-  __syncthreads();
-  if (warp >= 2 && warp < 6) {
-    const int row = (warp & 3) * 32 + lane;
-    const int g_row = Rb * TC_BM + row;
-    if (!SWEEP2) {
-      // merge the groups' (reference, sum) pairs; a sum of 0 marks a group that had no tile
-      auto merged = [&](float m, float l, int off) -> float {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(c_full + cb);
+    } else {
+      if (ok) ok = __all_sync(0xffffffffu, wait_bar(c_full + cb, (uint32_t)((k / NCB) & 1), abort_flag));
+      if (!SWEEP2) {
+        // merge the groups' (reference, sum) pairs; a sum of 0 marks a group that had no tile
+        auto merged = [&](float m, float l, int off) -> float {
 #pragma unroll
-        for (int g = 1; g < NG; ++g) {
-          const float m1 = comb[(g - 1) * 512 + off + row], l1 = comb[(g - 1) * 512 + off + 128 + row];
-          if (l1 > 0.f) {
-            if (l > 0.f) {
-              const float mm = fmaxf(m, m1);
-              l = l * fast_exp2(m - mm) + l1 * fast_exp2(m1 - mm);
-              m = mm;
-            } else {
-              m = m1; l = l1;
+          for (int g = 0; g < NG; ++g) {
+            if (g == merger) continue;
+            const float m1 = cmb[g * 512 + off + row], l1 = cmb[g * 512 + off + 128 + row];
+            if (l1 > 0.f) {
+              if (l > 0.f) {
+                const float mm = fmaxf(m, m1);
+                l = l * fast_exp2(m - mm) + l1 * fast_exp2(m1 - mm);
+                m = mm;
+              } else {
+                m = m1; l = l1;
+              }
             }
           }
-        }
-        return m + log2f(l);
-      };
-      // rows past the prompt get +inf: their scores vanish in sweep 2 (and their attention weights likewise)
-      P.lse2[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? merged(row_m, row_l, 0) : INFINITY;
-      if (WANT_X) P.lse_x[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? merged(rowx_m, rowx_l, 256) : INFINITY;
-    } else if (g_row < P.n) {
-      float total = col_sum;
+          return m + log2f(l);
+        };
+        // rows past the prompt get +inf: their scores vanish in sweep 2 (and their attention weights likewise)
+        P.lse2[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? merged(row_m, row_l, 0) : INFINITY;
+        if (WANT_X) P.lse_x[(size_t)u * nblk * TC_BN + g_row] = g_row < P.n ? merged(rowx_m, rowx_l, 256) : INFINITY;
+      } else {
+        // a fixed order of summation (group 0, 1, ...), whichever group collects
+        float total = 0.f;
 #pragma unroll
-      for (int g = 1; g < NG; ++g) total += comb[(g - 1) * 512 + row];
-      P.acc_full[(size_t)u * P.n + g_row] = total;
+        for (int g = 0; g < NG; ++g) total += g == merger ? col_sum : cmb[g * 512 + row];
+        if (g_row < P.n) P.acc_full[(size_t)u * P.n + g_row] = total;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(c_empty + cb);
     }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicExch(P.err, ERR_TIMEOUT);
+    }
+    }   // items
   }
 
   // ---- teardown: on the failure path give the copies still in flight a bounded wait, then free tensor memory
+  __syncthreads();
   if (tid == 0 && *abort_flag) {
-    const int issued = *issued_slot;
+    const int issued = issued_slot[0], items = issued_slot[1];
     for (int it = issued > NST ? issued - NST : 0; it < issued; ++it)
       (void)mbar_wait_bounded(s_full + (it % NST), (uint32_t)((it / NST) & 1), TC_WAIT_LIMIT);
-    (void)mbar_wait_bounded(r_full, 0, TC_WAIT_LIMIT);
+    if (items > 0) (void)mbar_wait_bounded(r_full, (uint32_t)((items - 1) & 1), TC_WAIT_LIMIT);
   }
   tc_fence_before();
   __syncthreads();
@@ -496,7 +575,7 @@ namespace {
 template <int D, int NST, int NG>
 constexpr size_t tc_smem_bytes() {
   size_t b = 1024 + (size_t)(1 + NST) * TC_BM * D * 2 + (size_t)4 * NG * TC_XBUF_FLOATS * 4 + (size_t)4 * NG * 128 * 4 +
-             (size_t)(NG - 1) * 4 * 128 * 4 + 32 * 8 + 64;
+             (size_t)tc_comb_buffers(D) * NG * 4 * 128 * 4 + 40 * 8 + 64;
   return b < 120 * 1024 ? 120 * 1024 : b;   // one CTA per SM: each takes all of tensor memory
 }
 
@@ -504,7 +583,13 @@ template <int D, int NST, int NG, bool SWEEP2>
 cudaError_t launch_variant(const PrefillTcParams& P, int units, int noise, bool alibi, cudaStream_t st) {
   constexpr size_t smem = tc_smem_bytes<D, NST, NG>();
   static_assert(smem <= 227 * 1024, "shared memory budget of one CTA");
-  dim3 grid((unsigned)P.nblk, (unsigned)units);
+  // persistent grid: one CTA per SM (each takes all of tensor memory), fewer when there are fewer item pairs
+  int dev = 0, sms = 0;
+  cudaError_t e0 = cudaGetDevice(&dev);
+  if (e0 == cudaSuccess) e0 = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e0 != cudaSuccess) return e0;
+  const long long pairs = ((long long)P.nblk * units + 1) / 2;
+  dim3 grid((unsigned)(pairs < sms ? pairs : sms));
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -544,6 +629,7 @@ cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int un
   P.err = a.err;
   P.n = a.n;
   P.nblk = (a.n + TC_BM - 1) / TC_BM;
+  P.units = units;
   P.H = a.H;
   P.layer = a.layer;
   P.inv_tau = a.inv_tau;
