@@ -133,7 +133,6 @@ __global__ void __launch_bounds__(SEL_T) prefill_select(const __grid_constant__ 
   __shared__ unsigned int hist[256];
   __shared__ unsigned int sh_prefix, sh_remaining;
   __shared__ unsigned int warp_a[SEL_T / 32], warp_b[SEL_T / 32];
-  __shared__ unsigned int base_eq, base_out;
   const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = P.n, k = P.k, w = P.w;
   const float* acc = P.acc_full + (size_t)u * n;
@@ -160,21 +159,30 @@ __global__ void __launch_bounds__(SEL_T) prefill_select(const __grid_constant__ 
         if ((bits & mask) == prefix) atomicAdd(&hist[(bits >> shift) & 0xFFu], 1u);
       }
       __syncthreads();
-      if (tid == 0) {
-        unsigned int remaining = sh_remaining, digit = 0;
-        for (int dgt = 255; dgt >= 0; --dgt) {
-          if (hist[dgt] >= remaining) { digit = (unsigned)dgt; break; }
-          remaining -= hist[dgt];
-        }
-        sh_prefix = prefix | (digit << shift);
-        sh_remaining = remaining;
+      // the digit where the count of larger-or-equal digits first reaches `remaining`: thread d holds bin d
+      // and the suffix sum above[d] = sum of the bins d' > d (warp shuffles, then the warps' totals)
+      const unsigned int remaining = sh_remaining;
+      const unsigned int mine = hist[tid];
+      unsigned int incl = mine;   // bins tid .. end of this warp
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int other = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += other;
+      }
+      if (lane == 0) warp_a[warp] = incl;
+      __syncthreads();
+      unsigned int above = incl - mine;
+      for (int wi = warp + 1; wi < SEL_T / 32; ++wi) above += warp_a[wi];
+      if (above < remaining && above + mine >= remaining) {   // exactly one thread
+        sh_prefix = prefix | ((unsigned)tid << shift);
+        sh_remaining = remaining - above;
       }
       __syncthreads();
     }
     thresh = sh_prefix;      // score bits of the r-th largest candidate
     need_eq = sh_remaining;  // how many candidates equal to it are kept (lowest positions first)
   }
-  if (tid == 0) { base_eq = 0u; base_out = 0u; }
+  unsigned int base_eq = 0u, base_out = 0u;   // every thread keeps the same running totals
   __syncthreads();
 
   for (int j0 = 0; j0 < n; j0 += SEL_T) {
@@ -212,9 +220,8 @@ __global__ void __launch_bounds__(SEL_T) prefill_select(const __grid_constant__ 
       if (out_before < (unsigned)k) idx[out_before] = j;
       else atomicExch(P.err, ERR_BOUNDS);
     }
-    __syncthreads();
-    if (tid == 0) { base_eq += eq_total; base_out += out_total; }
-    __syncthreads();
+    base_eq += eq_total;
+    base_out += out_total;
   }
   if (tid == 0) {
     if (base_out != (unsigned)k) atomicExch(P.err, ERR_BOUNDS);
