@@ -34,6 +34,24 @@ def test_prompt_lengths_around_tile_edges(n, noise):
     lockstep.run_workload(wl, noise=noise)
 
 
+@pytest.mark.parametrize("impl", [kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_SIMT])
+def test_prompts_shorter_than_the_maximum_and_a_context_used_again(impl):
+    """A context sized for 700 positions takes prompts of 700, 129 and 300 tokens on the same layer one after
+    the other (scratch of a longer prompt must not leak into a shorter one), each followed by decode steps."""
+    for n in (700, 129, 300):
+        wl = _wl(head_dim=128, prompt_len=n, budget_k=96, recent_w=24, gen_len_T=4, data_seed=100 + n)
+        if n == 700:
+            gpu = lockstep.make_gpu(wl, max_prompt_len=700, prefill_impl=impl)
+        ls = lockstep.LockStep(wl, gpu, 0, W.unit_list(wl, 0))
+        ls.prefill(*W.make_prompt(wl, 0, DEV))
+        for s in range(1, 5):
+            ls.decode_step(s, *W.make_step(wl, 0, s, DEV))
+    with pytest.raises(kf.KeyformerError) as e:
+        gpu.kf_prefill_score_prune(0, *W.make_prompt(_wl(head_dim=128, prompt_len=701), 0, DEV))
+    assert e.value.code == kf.KF_EINVAL
+    gpu.kf_destroy()
+
+
 @pytest.mark.parametrize("scale", [2.0, 16.0])
 def test_prompt_scores_with_extreme_logits(scale):
     """Logits hundreds of units apart (a scale far above 1/sqrt(d)): the prompt softmax must not overflow,
