@@ -343,6 +343,11 @@ def run_ours(args, wl):
 #   FP32:    uniform and 1 - u (2), repair series (2), noise and logit FMAs (2), sum (1)                   ->  7
 #   MUFU:    two logarithms, one exponential (one issue slot each; 8 cycles each on the 16-lane XU)       ->  3
 PREFILL_INT_INSTR, PREFILL_FP_INSTR, PREFILL_MUFU_INSTR = 13, 7, 3
+# dram__bytes_read.sum + dram__bytes_write.sum of the two prefill_tc launches of one call on c5_prefill_2k (B8 H32 d128,
+# n 2048: Q + K = 268 MB, each read from DRAM once per sweep), from the ncu capture summarised in
+# profiles/prefill_tc_c5_prefill_sweep.md.  It does not scale with the logit count (re-reads are served by L2), so the
+# other prompt lengths report no traffic figure.
+C5_2K_PREFILL_TRAFFIC_BYTES = (268.5 + 4.8 + 270.6 + 5.4) * 1e6
 PREFILL_LANE_INSTR_PER_LOGIT_SWEEP = 2 * PREFILL_INT_INSTR + PREFILL_FP_INSTR + PREFILL_MUFU_INSTR   # 36 FP32-lane slots
 ALU_LANES_PER_SM, N_SM = 128, 148
 
@@ -406,7 +411,8 @@ def run_prefill(args, wl):
                        "qk_tflops_both_sweeps": 2 * 2 * logits * wl.head_dim / (ms * 1e-3) / 1e12,
                        "l2": "Q, K, V of the call (%.0f MB) exceed L2" % (3 * units * n * wl.head_dim * 2 / 1e6)},
             "roofline": {"bound": "alu", "kernel": "prefill_tc (two sweeps)", "achieved": achieved, "peak": peak,
-                         "unit": "T FP32-lane issue slots/s (INT32 instructions count twice)", "frac": achieved / peak, "traffic": None,
+                         "unit": "T FP32-lane issue slots/s (INT32 instructions count twice)", "frac": achieved / peak,
+                         "traffic": C5_2K_PREFILL_TRAFFIC_BYTES if (wl.name == "c5_prefill_2k" and not args.prefill_simt) else None,
                          "lane_instr_per_logit_sweep": PREFILL_LANE_INSTR_PER_LOGIT_SWEEP,
                          "peak_kind": "148 SMs x 128 lanes x 1965 MHz", "sm_mhz_seen": sm_mhz},
             "gpu_launches": int(launches), "clocks": clocks,
