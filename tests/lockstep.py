@@ -98,6 +98,19 @@ class LockStep:
         score = torch.empty(wl.batch, wl.n_heads, n, dtype=torch.float32, device=q.device)
         gpu.kf_prefill_score_prune(self.layer, q, k, v, score_out=score)
         assert gpu.kf_poll_error() == 0
+        # every unit of the layer, sampled by the oracle or not: each of the n softmax rows adds 1 to the scores,
+        # the kept positions ascend and end with the w most recent ones
+        kk_, w_ = wl.budget_k, wl.recent_w
+        tot = score.double().sum(-1)
+        assert ((tot - n).abs() <= 1e-4 * n).all(), "prompt scores do not add up to the number of query rows"
+        _, _, pos_all, _, len_all = gpu.kf_view_state(self.layer)
+        L_all = min(n, kk_)
+        assert (len_all == L_all).all()
+        assert (pos_all[..., 1:L_all] > pos_all[..., :L_all - 1]).all() and (pos_all[..., :L_all] >= 0).all()
+        n_rec = min(w_, L_all)
+        if n_rec > 0:
+            assert torch.equal(pos_all[..., L_all - n_rec:L_all].long(),
+                               torch.arange(n - n_rec, n, device=pos_all.device).expand(wl.batch, wl.n_heads, n_rec))
         Qs, Ks, Vs = self._rows(q), self._rows(k), self._rows(v)
         acc_ref = self.st.prefill_score(Qs, Ks)
         acc_gpu = self._rows(score).astype(np.float64)
@@ -134,9 +147,34 @@ class LockStep:
         _, _, pos_before, _, len_before = self.gpu_state(rows=False)
         out = torch.empty(wl.batch, wl.n_heads, wl.head_dim, dtype=torch.float16, device=q.device)
         score = torch.zeros(wl.batch, wl.n_heads, wl.budget_k + 1, dtype=torch.float32, device=q.device)
+        len_all_before = self.gpu.kf_view_state(self.layer)[4].clone()
         self.gpu.kf_decode_step(self.layer, step, q, knew, vnew, out, score_out=score)
         assert self.gpu.kf_poll_error() == 0
+        self._check_all_units(step, out, score, len_all_before)
         return self._compare_decode(step, q, knew, vnew, out, score, pos_before, len_before, check_state)
+
+    def _check_all_units(self, step, out, score, len_before):
+        """Properties that hold for every unit of the layer, sampled by the oracle or not (computed on the GPU
+        with library ops): Eq. 11 is a softmax, one entry at most leaves, positions stay distinct, and the new
+        token and the w most recent positions are always in the cache."""
+        wl = self.wl
+        kk, w = wl.budget_k, wl.recent_w
+        p = self.n + step - 1
+        _, _, pos, acc, ln = self.gpu.kf_view_state(self.layer)
+        m = len_before.long() + 1                                            # entries scored this step
+        col = torch.arange(kk + 1, device=score.device)
+        zsum = torch.where(col < m[..., None], score, torch.zeros_like(score)).sum(-1)
+        assert torch.isfinite(out.float()).all() and (zsum - 1).abs().max().item() < 1e-4, f"step {step}: scores do not sum to 1"
+        assert torch.equal(ln.long(), torch.clamp(m, max=kk)), f"step {step}: entry counts"
+        valid = torch.arange(kk, device=pos.device) < ln[..., None]
+        ps = torch.where(valid, pos, torch.full_like(pos, -1)).long()
+        srt = ps.sort(-1).values
+        dup = (srt[..., 1:] == srt[..., :-1]) & (srt[..., 1:] >= 0)
+        assert not dup.any(), f"step {step}: a position is cached twice"
+        assert (ps.max(-1).values == p).all() or w == 0, f"step {step}: the new token is missing"
+        recent = ((ps > p - w) & valid).sum(-1)
+        assert torch.equal(recent, torch.clamp(ln.long(), max=min(w, p + 1))), f"step {step}: recent window incomplete"
+        assert (acc[valid] >= 0).all()
 
     def _compare_decode(self, step, q, knew, vnew, out, score, pos_before, len_before, check_state):
         wl = self.wl
