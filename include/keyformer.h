@@ -217,6 +217,17 @@ int kf_decode_step_static(const kf_static_step* args,
 int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V,
                   const int32_t** d_pos, const float** d_acc, const int32_t** d_len);
 
+/* In-place compaction of one layer's cache into position order (Algorithm 1 describes the reduced cache as a
+ * subsequence of the token sequence, S_key and the recent window S_w; section 3.4).  kf_decode_step keeps each
+ * unit's entries as an unordered set -- the token that leaves is overwritten by the one that arrives -- and
+ * identifies them by their positions, so no call needs this one.  It exists for callers that want the layout the
+ * prompt phase produces back: slot s of every (batch row, head) holds the entry with the s-th smallest position
+ * (K row, V row, position, f_theta), e.g. to compare or store state images independent of the eviction history.
+ * The permutation is applied in place, cycle by cycle, with no staging buffer; asynchronous on `stream`.
+ * KF_ESTATE before the layer's prompt phase; KF_EINVAL when budget_k exceeds 16384 (the ranks of a unit's
+ * entries are computed in shared memory). */
+int kf_compact_layer(kf_ctx* ctx, int32_t layer, void* stream);
+
 /* KF_POS_NEW only: borrowed DEVICE pointer to the places, int32 [B][H][k]; entry j of a unit holds the
  * number of entries of that unit with a smaller position.  KF_EINVAL in the other mode. */
 int kf_view_place(kf_ctx* ctx, int32_t layer, const int32_t** d_place);

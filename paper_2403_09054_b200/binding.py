@@ -23,7 +23,7 @@ KF_POS_ORIGINAL, KF_POS_NEW = 0, 1
 EXPORTS = ("kf_workspace_bytes", "kf_create", "kf_prefill_score_prune", "kf_decode_step",
            "kf_decode_step_host", "kf_view_state", "kf_poll_error", "kf_launch_count",
            "kf_destroy", "kf_strerror", "kf_decode_step_static", "kf_state_bytes", "kf_export_state", "kf_import_state",
-           "kf_prefill_attend", "kf_prefill_attend_score_prune", "kf_view_place")
+           "kf_prefill_attend", "kf_prefill_attend_score_prune", "kf_view_place", "kf_compact_layer")
 
 
 class kf_config(C.Structure):
@@ -80,6 +80,8 @@ def _load() -> C.CDLL:
     lib.kf_export_state.argtypes = [vp, i32, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32), vp]
     lib.kf_import_state.restype = C.c_int
     lib.kf_import_state.argtypes = [vp, i32, vp, C.c_size_t, i32, i32, vp]
+    lib.kf_compact_layer.restype = C.c_int
+    lib.kf_compact_layer.argtypes = [vp, i32, vp]
     lib.kf_view_place.restype = C.c_int
     lib.kf_view_place.argtypes = [vp, i32, C.POINTER(vp)]
     lib.kf_view_state.restype = C.c_int
@@ -262,6 +264,10 @@ class Keyformer:
         acc = view(ptrs[3], B * H * k * 4, torch.float32, (B, H, k))
         ln = view(ptrs[4], B * H * 4, torch.int32, (B, H))
         return K, V, pos, acc, ln
+
+    def kf_compact_layer(self, layer, stream=None):
+        """Reorder the layer's cache entries into ascending position, in place."""
+        _check(LIB.kf_compact_layer(self._h, layer, _stream_ptr(stream)), "kf_compact_layer")
 
     def kf_view_place(self, layer):
         """Zero-copy torch view of one layer's places (KF_POS_NEW only), int32 [B, H, k]."""

@@ -434,6 +434,24 @@ int kf_view_state(kf_ctx* ctx, int32_t layer, const void** d_K, const void** d_V
   return KF_OK;
 }
 
+int kf_compact_layer(kf_ctx* ctx, int32_t layer, void* stream) {
+  if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return KF_EINVAL;
+  if (ctx->n_prompt[layer] < 0) return KF_ESTATE;
+  const kf_config& c = ctx->cfg;
+  if (c.budget_k > kf::compact_max_k()) return KF_EINVAL;
+  const Layout& L = ctx->lay;
+  if (kf::launch_compact(reinterpret_cast<__half*>(ctx->ws + L.K + (size_t)layer * L.kv_layer),
+                         reinterpret_cast<__half*>(ctx->ws + L.V + (size_t)layer * L.kv_layer),
+                         reinterpret_cast<float*>(ctx->ws + L.acc + (size_t)layer * L.sc_layer),
+                         reinterpret_cast<int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer),
+                         reinterpret_cast<const int32_t*>(ctx->ws + L.len + (size_t)layer * L.len_layer),
+                         c.pos_mode == KF_POS_NEW ? reinterpret_cast<int32_t*>(ctx->ws + L.place + (size_t)layer * L.sc_layer) : nullptr,
+                         c.budget_k, c.head_dim, L.units, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return KF_ECUDA;
+  ctx->launches += 1;
+  return KF_OK;
+}
+
 int kf_view_place(kf_ctx* ctx, int32_t layer, const int32_t** d_place) {
   if (!ctx || !d_place || layer < 0 || layer >= ctx->cfg.n_layers || ctx->cfg.pos_mode != KF_POS_NEW) return KF_EINVAL;
   *d_place = reinterpret_cast<const int32_t*>(ctx->ws + ctx->lay.place + (size_t)layer * ctx->lay.sc_layer);

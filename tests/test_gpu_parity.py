@@ -190,6 +190,45 @@ def test_new_positions_differ_from_original_positions_and_survive_import():
     assert org.kf_poll_error() == 0 and new.kf_poll_error() == 0 and again.kf_poll_error() == 0
 
 
+@pytest.mark.parametrize("d,pos_mode", [(64, 0), (128, 1), (256, 0)])
+def test_compaction_restores_position_order_in_place(d, pos_mode):
+    """After enough steps the slots of a unit are a permutation of the position order.  kf_compact_layer must apply
+    exactly the sorting permutation to K, V, positions and scores (compared with a gather done here by library
+    ops), leave a layer it is not asked about alone, and the generation that follows must still match the oracle."""
+    wl = W.get_config("c3_mpt").scaled(n_layers=2, n_heads=3, batch=2, head_dim=d, prompt_len=200, budget_k=77,
+                                       recent_w=20, gen_len_T=40)
+    gpu = lockstep.make_gpu(wl, pos_mode=pos_mode)
+    with pytest.raises(kf.KeyformerError) as e:
+        gpu.kf_compact_layer(0)
+    assert e.value.code == kf.KF_ESTATE
+    drivers = [lockstep.LockStep(wl, gpu, l, W.unit_list(wl, l), pos_mode=pos_mode) for l in range(2)]
+    for ls in drivers:
+        ls.prefill(*W.make_prompt(wl, ls.layer, DEV))
+    for s in range(1, 26):
+        for ls in drivers:
+            ls.decode_step(s, *W.make_step(wl, ls.layer, s, DEV), check_state=(s == 25))
+    before = [[t.clone() for t in gpu.kf_view_state(l)] for l in range(2)]
+    assert not torch.equal(before[0][2], before[0][2].sort(-1).values)       # the slots are out of order by now
+    gpu.kf_compact_layer(0)
+    assert gpu.kf_poll_error() == 0
+    K, V, pos, acc, ln = gpu.kf_view_state(0)
+    order = before[0][2].argsort(-1)
+    assert torch.equal(pos, before[0][2].gather(-1, order)) and torch.equal(acc, before[0][3].gather(-1, order))
+    rows = order[..., None].expand(-1, -1, -1, d)
+    assert torch.equal(K, before[0][0].gather(2, rows)) and torch.equal(V, before[0][1].gather(2, rows))
+    assert torch.equal(ln, before[0][4])
+    if pos_mode == 1:
+        assert torch.equal(gpu.kf_view_place(0).long(), torch.arange(77, device=DEV).expand(2, 3, 77))
+    for x, y in zip(gpu.kf_view_state(1), before[1]):
+        assert torch.equal(x, y)
+    gpu.kf_compact_layer(0)                                                   # already in order: nothing moves
+    assert torch.equal(gpu.kf_view_state(0)[2], pos) and torch.equal(gpu.kf_view_state(0)[0], K)
+    for s in range(26, 41):
+        for ls in drivers:
+            ls.decode_step(s, *W.make_step(wl, ls.layer, s, DEV))
+    gpu.kf_destroy()
+
+
 def test_heavy_hitter_multi_layer_scaled_down():
     wl = W.get_config("c4_cerebras").scaled(n_layers=3, batch=2, n_heads=4, prompt_len=400, budget_k=200, recent_w=50, gen_len_T=8)
     lockstep.run_workload(wl)
