@@ -446,9 +446,10 @@ int kf_compact_layer(kf_ctx* ctx, int32_t layer, void* stream) {
                          reinterpret_cast<int32_t*>(ctx->ws + L.pos + (size_t)layer * L.sc_layer),
                          reinterpret_cast<const int32_t*>(ctx->ws + L.len + (size_t)layer * L.len_layer),
                          c.pos_mode == KF_POS_NEW ? reinterpret_cast<int32_t*>(ctx->ws + L.place + (size_t)layer * L.sc_layer) : nullptr,
+                         reinterpret_cast<int32_t*>(ctx->ws + L.idx),   // the prompt phase's index scratch is free here
                          c.budget_k, c.head_dim, L.units, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return KF_ECUDA;
-  ctx->launches += 1;
+  ctx->launches += 2;
   return KF_OK;
 }
 

@@ -37,10 +37,10 @@ int decode_max_splits();
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 
 // Reorders every unit's entries of one layer into ascending position, in place (see kf_compact.cu).  `place` may be
-// null.  Budgets above compact_max_k() are refused (cudaErrorInvalidValue).
+// null; `dst_scratch` is [units][k] int32 of scratch.  Budgets above compact_max_k() are refused (cudaErrorInvalidValue).
 int compact_max_k();
-cudaError_t launch_compact(__half* K, __half* V, float* acc, int32_t* pos, const int32_t* len, int32_t* place, int k,
-                           int head_dim, int units, cudaStream_t stream);
+cudaError_t launch_compact(__half* K, __half* V, float* acc, int32_t* pos, const int32_t* len, int32_t* place,
+                           int32_t* dst_scratch, int k, int head_dim, int units, cudaStream_t stream);
 
 // place[j] = number of entries of the unit with a smaller position, for every unit of a layer (after a state import).
 cudaError_t launch_rebuild_place(const int32_t* pos, const int32_t* len, int32_t* place, int k, int units,
