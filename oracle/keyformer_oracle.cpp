@@ -1,7 +1,7 @@
 // Keyformer CPU oracle -- TEST INFRASTRUCTURE, not a product path.
 //
 // A plain, slow, double-precision restatement of the Keyformer method
-// (Algorithm 1 with Eq. 1, 4, 7, 11, 12 of the paper), one (batch, layer, head)
+// (Algorithm 1 with Eq. 1, 4, 7, 11, 12 of the paper), one (batch, layer, key/value head)
 // unit at a time.  It shares no code with the CUDA library.  Only the test
 // suite, the smoke check and the benchmark's cpu_baseline leg may call it.
 //
@@ -49,7 +49,17 @@ struct ko_params {
   double noise_sigma;    // Gaussian std
   uint64_t noise_seed;
   const double* alibi_slopes;  // [H] or null
+  int32_t n_kv_heads;    // key/value heads; H / n_kv_heads query heads share each of them (0 = H: none shared)
 };
+
+// Query heads per key/value head (section 6 names multi-query / grouped-query attention as compatible with the
+// method without giving the rule).  Reading: a cache and its f_theta belong to a key/value head; every query head
+// h = kv_head * g + r of the group has its own logits, its own noise (drawn with its own head index) and its own
+// softmax of Eq. 11; f_theta accumulates the mean of the group's scores, so a step still adds a total of 1 to a
+// cache and g = 1 is the method as printed.
+static int group_size(const ko_params* P) {
+  return (P->n_kv_heads > 0 && P->n_kv_heads < P->n_heads) ? P->n_heads / P->n_kv_heads : 1;
+}
 
 // ---------------------------------------------------------------------------
 // IEEE binary16 -> double, by decoding the bit fields.
@@ -224,39 +234,51 @@ void ko_select(const int32_t* pos, const double* acc, int32_t m, int32_t k, int3
 // by tau_init and normalised (Eq. 11); the result is added into f_theta(j).
 //   Q, K: [n][d] binary16 bit patterns of this unit.   acc_out: [n].
 // ---------------------------------------------------------------------------
-static void prefill_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t h, int32_t n,
-                               const uint16_t* Q, const uint16_t* K, double* acc_out) {
+static void prefill_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t hk, int32_t n,
+                               const uint16_t* Q /* [g][n][d] */, const uint16_t* K, double* acc_out) {
   const int d = P->head_dim;
+  const int g = group_size(P);
   const double tau = ko_tau(P, 0);
   std::vector<double> y(n), z(n);
   for (int j = 0; j < n; ++j) acc_out[j] = 0.0;
-  for (int i = 0; i < n; ++i) {
-    const int m = i + 1;
-    for (int j = 0; j < m; ++j) {
-      const double x = P->logit_scale * dot_half(Q + (size_t)i * d, K + (size_t)j * d, d)
-                     + position_bias(P, h, i, j);                       // Eq. 4: x
-      y[j] = (x + ko_noise(P, b, l, h, i, j)) / tau;                    // Eq. 4 then Eq. 11
+  for (int r = 0; r < g; ++r) {
+    const int h = hk * g + r;                                             // query head r of this key/value head
+    const uint16_t* Qh = Q + (size_t)r * n * d;
+    for (int i = 0; i < n; ++i) {
+      const int m = i + 1;
+      for (int j = 0; j < m; ++j) {
+        const double x = P->logit_scale * dot_half(Qh + (size_t)i * d, K + (size_t)j * d, d)
+                       + position_bias(P, h, i, j);                       // Eq. 4: x
+        y[j] = (x + ko_noise(P, b, l, h, i, j)) / tau;                    // Eq. 4 then Eq. 11
+      }
+      softmax_inplace(y.data(), z.data(), m);
+      for (int j = 0; j < m; ++j) acc_out[j] += z[j] / (double)g;         // accumulate f_theta (group mean)
     }
-    softmax_inplace(y.data(), z.data(), m);
-    for (int j = 0; j < m; ++j) acc_out[j] += z[j];                     // accumulate f_theta
   }
 }
 
 // Attention output of the prompt phase (Eq. 1 with the causal mask): row i attends to keys j <= i with the
 // plain softmax of x (no adjustment, temperature 1), exactly what the model's attention layer produces.
-static void prefill_attend_unit(const ko_params* P, int32_t h, int32_t n,
-                                const uint16_t* Q, const uint16_t* K, const uint16_t* V, double* out) {
+static void prefill_attend_unit(const ko_params* P, int32_t hk, int32_t n,
+                                const uint16_t* Q /* [g][n][d] */, const uint16_t* K, const uint16_t* V,
+                                double* out /* [g][n][d] */) {
   const int d = P->head_dim;
+  const int g = group_size(P);
   std::vector<double> x(n), p(n);
-  for (int i = 0; i < n; ++i) {
-    const int m = i + 1;
-    for (int j = 0; j < m; ++j)
-      x[j] = P->logit_scale * dot_half(Q + (size_t)i * d, K + (size_t)j * d, d) + position_bias(P, h, i, j);
-    softmax_inplace(x.data(), p.data(), m);
-    for (int c = 0; c < d; ++c) {
-      double s = 0.0;
-      for (int j = 0; j < m; ++j) s += p[j] * h2d(V[(size_t)j * d + c]);
-      out[(size_t)i * d + c] = s;
+  for (int r = 0; r < g; ++r) {
+    const int h = hk * g + r;
+    const uint16_t* Qh = Q + (size_t)r * n * d;
+    double* outh = out + (size_t)r * n * d;
+    for (int i = 0; i < n; ++i) {
+      const int m = i + 1;
+      for (int j = 0; j < m; ++j)
+        x[j] = P->logit_scale * dot_half(Qh + (size_t)i * d, K + (size_t)j * d, d) + position_bias(P, h, i, j);
+      softmax_inplace(x.data(), p.data(), m);
+      for (int c = 0; c < d; ++c) {
+        double s = 0.0;
+        for (int j = 0; j < m; ++j) s += p[j] * h2d(V[(size_t)j * d + c]);
+        outh[(size_t)i * d + c] = s;
+      }
     }
   }
 }
@@ -294,13 +316,14 @@ static void prefill_prune_unit(const ko_params* P, int32_t n, const uint16_t* K,
 //   z    = softmax((x + zeta) / tau_s)        (Eq. 11, Eq. 12)
 //   acc += z                                  (Algorithm 1 accumulation)
 // ---------------------------------------------------------------------------
-static void decode_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t h,
+static void decode_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t hk,
                               int32_t step, int32_t n_prompt,
-                              const uint16_t* q, const uint16_t* knew, const uint16_t* vnew,
+                              const uint16_t* q /* [g][d] */, const uint16_t* knew, const uint16_t* vnew,
                               int32_t* st_len, int32_t* st_pos, double* st_acc,
                               uint16_t* st_K, uint16_t* st_V,
-                              double* out, double* z_out) {
+                              double* out /* [g][d] */, double* z_out /* [cap]: the group's mean score */) {
   const int d = P->head_dim;
+  const int g = group_size(P);
   const int p = n_prompt + step - 1;
   int len = *st_len;
   st_pos[len] = p;
@@ -311,21 +334,26 @@ static void decode_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t 
   *st_len = len;
   const int m = len;
   const double tau = ko_tau(P, step);
-  std::vector<double> x(m), y(m), a(m);
-  for (int j = 0; j < m; ++j) {
-    // "New Pos" (section 4.4.2): the bias sees the entries' places in the reduced cache, which this list
-    // keeps in position order, so entry j sits at place j and the current token at place m - 1.
-    const double bias = P->pos_mode == 1 ? position_bias(P, h, m - 1, j) : position_bias(P, h, p, st_pos[j]);
-    x[j] = P->logit_scale * dot_half(q, st_K + (size_t)j * d, d) + bias;
-    y[j] = (x[j] + ko_noise(P, b, l, h, p, st_pos[j])) / tau;
+  std::vector<double> x(m), y(m), a(m), z(m);
+  for (int j = 0; j < m; ++j) z_out[j] = 0.0;
+  for (int r = 0; r < g; ++r) {
+    const int h = hk * g + r;                                             // query head r of this key/value head
+    for (int j = 0; j < m; ++j) {
+      // "New Pos" (section 4.4.2): the bias sees the entries' places in the reduced cache, which this list
+      // keeps in position order, so entry j sits at place j and the current token at place m - 1.
+      const double bias = P->pos_mode == 1 ? position_bias(P, h, m - 1, j) : position_bias(P, h, p, st_pos[j]);
+      x[j] = P->logit_scale * dot_half(q + (size_t)r * d, st_K + (size_t)j * d, d) + bias;
+      y[j] = (x[j] + ko_noise(P, b, l, h, p, st_pos[j])) / tau;
+    }
+    softmax_inplace(x.data(), a.data(), m);
+    for (int c = 0; c < d; ++c) {
+      double s = 0.0;
+      for (int j = 0; j < m; ++j) s += a[j] * h2d(st_V[(size_t)j * d + c]);
+      out[(size_t)r * d + c] = s;
+    }
+    softmax_inplace(y.data(), z.data(), m);
+    for (int j = 0; j < m; ++j) z_out[j] += z[j] / (double)g;
   }
-  softmax_inplace(x.data(), a.data(), m);
-  for (int c = 0; c < d; ++c) {
-    double s = 0.0;
-    for (int j = 0; j < m; ++j) s += a[j] * h2d(st_V[(size_t)j * d + c]);
-    out[c] = s;
-  }
-  softmax_inplace(y.data(), z_out, m);
   for (int j = 0; j < m; ++j) st_acc[j] += z_out[j];
 }
 
@@ -362,26 +390,28 @@ static void decode_evict_unit(const ko_params* P, int32_t step, int32_t n_prompt
 
 // ---------------------------------------------------------------------------
 // Batched entry points: U independent units, OpenMP across units only.
-//   lbh: [U][3] = (layer, batch, head) of each unit.
+//   lbh: [U][3] = (layer, batch, key/value head) of each unit; with shared key/value heads the q arrays carry
+//   the g query heads of the unit's group one after the other.
 //   state arrays have capacity cap = k + 1 entries per unit.
 // ---------------------------------------------------------------------------
 void ko_prefill_score_units(const ko_params* P, int32_t U, const int32_t* lbh, int32_t n,
                             const uint16_t* Q, const uint16_t* K, double* acc_full) {
-  const size_t d = (size_t)P->head_dim;
+  const size_t d = (size_t)P->head_dim, g = (size_t)group_size(P);
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < U; ++u) {
     prefill_score_unit(P, lbh[3 * u + 1], lbh[3 * u + 0], lbh[3 * u + 2], n,
-                       Q + (size_t)u * n * d, K + (size_t)u * n * d, acc_full + (size_t)u * n);
+                       Q + (size_t)u * g * n * d, K + (size_t)u * n * d, acc_full + (size_t)u * n);
   }
 }
 
 void ko_prefill_attend_units(const ko_params* P, int32_t U, const int32_t* lbh, int32_t n,
-                             const uint16_t* Q, const uint16_t* K, const uint16_t* V, double* out /* [U][n][d] */) {
-  const size_t d = (size_t)P->head_dim;
+                             const uint16_t* Q /* [U][g][n][d] */, const uint16_t* K, const uint16_t* V,
+                             double* out /* [U][g][n][d] */) {
+  const size_t d = (size_t)P->head_dim, g = (size_t)group_size(P);
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < U; ++u) {
-    prefill_attend_unit(P, lbh[3 * u + 2], n, Q + (size_t)u * n * d, K + (size_t)u * n * d, V + (size_t)u * n * d,
-                        out + (size_t)u * n * d);
+    prefill_attend_unit(P, lbh[3 * u + 2], n, Q + (size_t)u * g * n * d, K + (size_t)u * n * d, V + (size_t)u * n * d,
+                        out + (size_t)u * g * n * d);
   }
 }
 
@@ -406,15 +436,15 @@ void ko_decode_score_units(const ko_params* P, int32_t U, const int32_t* lbh,
                            const uint16_t* q, const uint16_t* knew, const uint16_t* vnew,
                            int32_t* st_len, int32_t* st_pos, double* st_acc,
                            uint16_t* st_K, uint16_t* st_V,
-                           double* out /* [U][d] */, double* z /* [U][cap] */) {
-  const size_t d = (size_t)P->head_dim;
+                           double* out /* [U][g][d] */, double* z /* [U][cap] */) {
+  const size_t d = (size_t)P->head_dim, g = (size_t)group_size(P);
   const size_t cap = (size_t)P->budget_k + 1;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int u = 0; u < U; ++u) {
     decode_score_unit(P, lbh[3 * u + 1], lbh[3 * u + 0], lbh[3 * u + 2], step, n_prompt,
-                      q + u * d, knew + u * d, vnew + u * d,
+                      q + u * g * d, knew + u * d, vnew + u * d,
                       st_len + u, st_pos + u * cap, st_acc + u * cap,
-                      st_K + u * cap * d, st_V + u * cap * d, out + u * d, z + u * cap);
+                      st_K + u * cap * d, st_V + u * cap * d, out + u * g * d, z + u * cap);
   }
 }
 

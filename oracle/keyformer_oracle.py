@@ -41,7 +41,7 @@ class _Params(C.Structure):
         ("bias_mode", C.c_int32), ("pos_mode", C.c_int32),
         ("tau_init", C.c_double), ("tau_end", C.c_double), ("logit_scale", C.c_double),
         ("noise_const", C.c_double), ("noise_mu", C.c_double), ("noise_sigma", C.c_double),
-        ("noise_seed", C.c_uint64), ("alibi_slopes", C.POINTER(C.c_double)),
+        ("noise_seed", C.c_uint64), ("alibi_slopes", C.POINTER(C.c_double)), ("n_kv_heads", C.c_int32),
     ]
 
 
@@ -116,7 +116,13 @@ class Params:
     noise_mu: float = 0.5772
     noise_sigma: float = 1.2825
     pos_mode: int = 0                 # 0 original positions in the bias, 1 places within the reduced cache
+    n_kv_heads: int = 0               # key/value heads shared by groups of n_heads / n_kv_heads query heads (0 = none shared)
     _keep: list = field(default_factory=list, repr=False)
+
+    @property
+    def group(self) -> int:
+        """Query heads per key/value head."""
+        return self.n_heads // self.n_kv_heads if 0 < self.n_kv_heads < self.n_heads else 1
 
     def c(self) -> _Params:
         scale = self.logit_scale if self.logit_scale else 1.0 / float(np.sqrt(np.float64(self.head_dim)))
@@ -127,6 +133,7 @@ class Params:
         p.tau_init, p.tau_end, p.logit_scale = self.tau_init, self.tau_end, scale
         p.noise_const, p.noise_mu, p.noise_sigma = self.noise_const, self.noise_mu, self.noise_sigma
         p.noise_seed = self.noise_seed & 0xFFFFFFFFFFFFFFFF
+        p.n_kv_heads = self.n_kv_heads
         if self.alibi_slopes is not None:
             s = np.ascontiguousarray(self.alibi_slopes, dtype=np.float64)
             self._keep.append(s)
@@ -197,18 +204,20 @@ class State:
         """Accumulated prompt scores f_theta[U][n] before pruning (Algorithm 1, t = 0)."""
         Qb, Kb = _half_bits(Q), _half_bits(K)
         U, n, d = Kb.shape
-        assert U == self.U and d == self.P.head_dim and Qb.shape == Kb.shape
+        assert U == self.U and d == self.P.head_dim and Qb.size == Kb.size * self.P.group    # Q: [U][g][n][d]
         acc = np.zeros((U, n), dtype=np.float64)
         cp = self.P.c()
         _load().ko_prefill_score_units(C.byref(cp), U, _ptr(self.lbh), n, _ptr(Qb), _ptr(Kb), _ptr(acc))
         return acc
 
     def prefill_attend(self, Q, K, V) -> np.ndarray:
-        """Causal attention output of the prompt [U][n][d] (Eq. 1; plain softmax, no adjustment)."""
+        """Causal attention output of the prompt [U][n][d] ([U][g][n][d] with shared key/value heads)
+        (Eq. 1; plain softmax, no adjustment)."""
         Qb, Kb, Vb = _half_bits(Q), _half_bits(K), _half_bits(V)
         U, n, d = Kb.shape
-        assert U == self.U and d == self.P.head_dim and Qb.shape == Kb.shape == Vb.shape
-        out = np.zeros((U, n, d), dtype=np.float64)
+        g = self.P.group
+        assert U == self.U and d == self.P.head_dim and Kb.shape == Vb.shape and Qb.size == Kb.size * g
+        out = np.zeros((U, n, d) if g == 1 else (U, g, n, d), dtype=np.float64)
         cp = self.P.c()
         _load().ko_prefill_attend_units(C.byref(cp), U, _ptr(self.lbh), n, _ptr(Qb), _ptr(Kb), _ptr(Vb), _ptr(out))
         return out
@@ -226,12 +235,13 @@ class State:
 
     # -- generation phase ---------------------------------------------------
     def decode_score(self, step: int, q, knew, vnew):
-        """Append the new token, attend, score, accumulate.  Returns (out[U][d], z[U][cap])."""
+        """Append the new token, attend, score, accumulate.  Returns (out[U][d] -- [U][g][d] with g query heads
+        per key/value head --, z[U][cap] = the score added to f_theta: the group's mean)."""
         qb, kb, vb = _half_bits(q), _half_bits(knew), _half_bits(vnew)
-        d = self.P.head_dim
-        assert qb.shape == (self.U, d) and kb.shape == (self.U, d) and vb.shape == (self.U, d)
+        d, g = self.P.head_dim, self.P.group
+        assert qb.size == self.U * g * d and kb.shape == (self.U, d) and vb.shape == (self.U, d)    # q: [U][g][d]
         assert int(self.len.max(initial=0)) < self.cap
-        out = np.zeros((self.U, d), dtype=np.float64)
+        out = np.zeros((self.U, d) if g == 1 else (self.U, g, d), dtype=np.float64)
         z = np.zeros((self.U, self.cap), dtype=np.float64)
         cp = self.P.c()
         _load().ko_decode_score_units(C.byref(cp), self.U, _ptr(self.lbh), step, self.n_prompt,

@@ -519,3 +519,109 @@ def test_new_positions_equal_original_positions_until_something_is_evicted():
         if n + s <= 12:                # nothing evicted before this step's scoring: places are positions
             assert np.array_equal(res[0][s], res[1][s])
     assert not np.array_equal(res[0][7], res[1][7])
+
+
+# ---------------------------------------------------------------- shared key/value heads (section 6: MQA / GQA)
+def _grouped_case(seed, B, Hkv, g, n, d):
+    """Q [B*Hkv][g][n][d], K, V [B*Hkv][n][d] and the same data laid out for H = Hkv * g independent heads
+    (K, V repeated for every query head of a group)."""
+    gen = torch.Generator().manual_seed(400 + seed)
+    U = B * Hkv
+    Q = torch.randn(U, g, n, d, generator=gen).half().numpy()
+    K = torch.randn(U, n, d, generator=gen).half().numpy()
+    V = torch.randn(U, n, d, generator=gen).half().numpy()
+    lbh_kv = np.array([(1, u // Hkv, u % Hkv) for u in range(U)], dtype=np.int32)
+    lbh_q = np.array([(1, u // Hkv, (u % Hkv) * g + r) for u in range(U) for r in range(g)], dtype=np.int32)
+    return Q, K, V, lbh_kv, lbh_q
+
+
+@pytest.mark.parametrize("g", [2, 4])
+def test_grouped_heads_prompt_scores_are_the_group_mean_of_independent_heads(g):
+    """With K/V repeated for every query head, multi-head scoring (pinned above to library softmax) gives each
+    query head's f_theta; the shared-head score must be their mean over the group, noise, temperature and ALiBi
+    slope of every head being that head's own."""
+    B, Hkv, n, d = 2, 3, 29, 16
+    H = Hkv * g
+    Q, K, V, lbh_kv, lbh_q = _grouped_case(g, B, Hkv, g, n, d)
+    slopes = W.alibi_slopes(H)
+    common = dict(head_dim=d, n_heads=H, budget_k=12, recent_w=3, gen_len_T=4, noise_seed=77, tau_init=1.3,
+                  bias_mode=1, alibi_slopes=slopes)
+    grouped = ko.State(ko.Params(n_kv_heads=Hkv, **common), lbh_kv).prefill_score(Q, K)
+    single = ko.State(ko.Params(**common), lbh_q).prefill_score(Q.reshape(-1, n, d), np.repeat(K, g, axis=0))
+    assert np.abs(grouped - single.reshape(B * Hkv, g, n).mean(axis=1)).max() < 1e-12
+    assert np.abs(grouped.sum(axis=1) - n).max() < 1e-9                 # a cache still receives mass 1 per query row
+    # and the heads of a group really differ (own noise, own slope): the mean is not one head's score
+    assert np.abs(single.reshape(B * Hkv, g, n)[:, 0] - grouped).max() > 1e-3
+
+
+@pytest.mark.parametrize("g", [2, 8])
+def test_grouped_heads_decode_against_library_attention_with_repeated_kv(g):
+    B, Hkv, n, d = 1, 2, 26, 16
+    H = Hkv * g
+    U = B * Hkv
+    Q, K, V, lbh_kv, _ = _grouped_case(10 + g, B, Hkv, g, n, d)
+    P = ko.Params(head_dim=d, n_heads=H, n_kv_heads=Hkv, budget_k=10, recent_w=3, gen_len_T=4, noise_mode=ko.NOISE_NONE,
+                  tau_init=1.0, tau_end=1.0)
+    st = ko.State(P, lbh_kv)
+    st.prefill_prune(K, V, st.prefill_score(Q, K))
+    gen = torch.Generator().manual_seed(5)
+    q = torch.randn(U, g, d, generator=gen).half().numpy()
+    kn, vn = torch.randn(U, d, generator=gen).half().numpy(), torch.randn(U, d, generator=gen).half().numpy()
+    total_before = st.acc[:, :10].sum(axis=1)
+    out, z = st.decode_score(1, q, kn, vn)
+    m = 11
+    Kc = torch.from_numpy(st.K[:, :m].view(np.float16).astype(np.float64))
+    Vc = torch.from_numpy(st.V[:, :m].view(np.float16).astype(np.float64))
+    qt = torch.from_numpy(q.astype(np.float64))
+    # library attention with every key/value head repeated for the g query heads of its group
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        qt.reshape(1, U * g, 1, d), Kc.repeat_interleave(g, 0)[None], Vc.repeat_interleave(g, 0)[None])
+    assert out.shape == (U, g, d) and np.abs(out - ref.reshape(U, g, d).numpy()).max() < 1e-12
+    # zero noise, temperature 1: the accumulated score is the mean attention weight of the group
+    w = torch.softmax(torch.einsum("ugd,umd->ugm", qt, Kc) / math.sqrt(d), -1).mean(1).numpy()
+    assert np.abs(z[:, :m] - w).max() < 1e-12
+    assert np.abs(st.acc[:, :m].sum(axis=1) - (total_before + 1.0)).max() < 1e-12      # +1 per step per cache
+
+
+def test_grouped_heads_decode_noise_is_drawn_per_query_head():
+    B, Hkv, g, n, d = 1, 2, 4, 20, 16
+    H, U = Hkv * g, B * Hkv
+    Q, K, V, lbh_kv, _ = _grouped_case(3, B, Hkv, g, n, d)
+    P = ko.Params(head_dim=d, n_heads=H, n_kv_heads=Hkv, budget_k=8, recent_w=2, gen_len_T=4, noise_seed=123)
+    st = ko.State(P, lbh_kv)
+    st.prefill_prune(K, V, st.prefill_score(Q, K))
+    gen = torch.Generator().manual_seed(6)
+    q = torch.randn(U, g, d, generator=gen).half().numpy()
+    kn, vn = torch.randn(U, d, generator=gen).half().numpy(), torch.randn(U, d, generator=gen).half().numpy()
+    _, z = st.decode_score(2, q, kn, vn)
+    m, p, tau = 9, n + 1, 1.0 + 2 * 0.25
+    for u in range(U):
+        l, b, hk = st.lbh[u]
+        Kc = st.K[u, :m].view(np.float16).astype(np.float64)
+        ref = np.zeros(m)
+        for r in range(g):
+            x = Kc @ q[u, r].astype(np.float64) / math.sqrt(d)
+            y = (x + np.array([ko.noise(P, b, l, hk * g + r, p, int(pj)) for pj in st.pos[u, :m]])) / tau
+            e = np.exp(y - y.max())
+            ref += e / e.sum() / g
+        assert np.abs(z[u, :m] - ref).max() < 1e-12
+
+
+def test_one_query_head_per_key_value_head_is_the_plain_method_bit_for_bit():
+    """n_kv_heads = n_heads (or 0) must not change a single bit of any result."""
+    U, n, d = 4, 33, 16
+    Q, K, V = _tiny_prompt(21, U, n, d)
+    res = []
+    for nkv in (0, 2):
+        P = _params(budget_k=9, recent_w=2, noise_seed=17, n_kv_heads=nkv)
+        st = ko.State(P, _lbh(U, 2))
+        acc = st.prefill_score(Q, K)
+        st.prefill_prune(K, V, acc)
+        outs = [acc, st.prefill_attend(Q, K, V)]
+        for s in (1, 2, 3):
+            out, z = st.decode_score(s, *_step_inputs(s, U, d))
+            st.decode_evict(s)
+            outs += [out, z, st.acc.copy(), st.pos.copy()]
+        res.append(outs)
+    for a, b in zip(*res):
+        assert a.shape == b.shape and np.array_equal(a, b)

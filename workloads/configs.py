@@ -26,10 +26,21 @@ class Workload:
     rotary_dims: int = 0           # leading dims rotated when positional == "rotary"
     heavy_frac: float = 0.0        # fraction of key positions that are heavy hitters
     heavy_logit: float = 0.0       # logit shift those keys receive (in units of scaled logits)
+    n_kv_heads: int = 0            # key/value heads shared by groups of query heads (0 = one per query head)
+
+    @property
+    def kv_heads(self) -> int:
+        return self.n_kv_heads if self.n_kv_heads > 0 else self.n_heads
+
+    @property
+    def group(self) -> int:
+        """Query heads per key/value head."""
+        return self.n_heads // self.kv_heads
 
     @property
     def units(self) -> int:
-        return self.n_layers * self.batch * self.n_heads
+        """Caches of the workload: one per (layer, batch row, key/value head)."""
+        return self.n_layers * self.batch * self.kv_heads
 
     def scaled(self, **kw) -> "Workload":
         return replace(self, **kw)
@@ -49,6 +60,9 @@ CONFIGS = {
                        positional="alibi"),
     "c4_cerebras": Workload("c4_cerebras", 32, 32, 32, 128, 4096, 2048, 512, 256, data_seed=4, noise_seed=4,
                             heavy_frac=0.05, heavy_logit=3.0),
+    # the same model with its 32 query heads sharing 8 key/value heads (grouped-query attention, 4 heads per group)
+    "c4_cerebras_gqa8": Workload("c4_cerebras_gqa8", 32, 32, 32, 128, 4096, 2048, 512, 256, data_seed=4, noise_seed=4,
+                                 heavy_frac=0.05, heavy_logit=3.0, n_kv_heads=8),
     # prefill sweep: one entry per prompt length; budgets are swept by the caller
     "c5_prefill_1k": Workload("c5_prefill_1k", 1, 8, 32, 128, 1024, 512, 128, 0, data_seed=5, noise_seed=5),
     "c5_prefill_2k": Workload("c5_prefill_2k", 1, 8, 32, 128, 2048, 1024, 256, 0, data_seed=5, noise_seed=5),

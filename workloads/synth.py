@@ -44,8 +44,8 @@ def _rotary(x: torch.Tensor, positions: torch.Tensor, rot_dims: int) -> torch.Te
 
 
 def _heavy_direction(wl: Workload, layer: int, device) -> torch.Tensor:
-    """Per (batch, head) unit vector along which heavy-hitter keys are shifted."""
-    e = _randn((wl.batch, wl.n_heads, wl.head_dim), _gen(wl, layer, "hh_dir", 0, device), device)
+    """Per (batch, key/value head) unit vector along which heavy-hitter keys are shifted."""
+    e = _randn((wl.batch, wl.kv_heads, wl.head_dim), _gen(wl, layer, "hh_dir", 0, device), device)
     return e / e.norm(dim=-1, keepdim=True)
 
 
@@ -54,17 +54,22 @@ def _heavy_amplitude(wl: Workload) -> float:
     return math.sqrt(wl.heavy_logit * math.sqrt(wl.head_dim))
 
 
+def _per_query_head(wl: Workload, e: torch.Tensor) -> torch.Tensor:
+    """[B, Hkv, ...] -> [B, H, ...]: every query head of a group sees its key/value head's entry."""
+    return e.repeat_interleave(wl.group, dim=1) if wl.group > 1 else e
+
+
 def make_prompt(wl: Workload, layer: int, device="cpu"):
-    """Prompt tensors Q, K, V of one layer: fp16 [B, H, n, d]."""
-    B, H, n, d = wl.batch, wl.n_heads, wl.prompt_len, wl.head_dim
+    """Prompt tensors of one layer: Q fp16 [B, H, n, d]; K, V fp16 [B, Hkv, n, d] (Hkv = H without shared heads)."""
+    B, H, Hkv, n, d = wl.batch, wl.n_heads, wl.kv_heads, wl.prompt_len, wl.head_dim
     q = _randn((B, H, n, d), _gen(wl, layer, "q", 0, device), device)
-    k = _randn((B, H, n, d), _gen(wl, layer, "k", 0, device), device)
-    v = _randn((B, H, n, d), _gen(wl, layer, "v", 0, device), device)
+    k = _randn((B, Hkv, n, d), _gen(wl, layer, "k", 0, device), device)
+    v = _randn((B, Hkv, n, d), _gen(wl, layer, "v", 0, device), device)
     if wl.heavy_frac > 0:
         e = _heavy_direction(wl, layer, device)[:, :, None, :]
         a = _heavy_amplitude(wl)
-        mask = torch.rand((B, H, n), generator=_gen(wl, layer, "hh_mask", 0, device), device=device) < wl.heavy_frac
-        q = q + a * e
+        mask = torch.rand((B, Hkv, n), generator=_gen(wl, layer, "hh_mask", 0, device), device=device) < wl.heavy_frac
+        q = q + a * _per_query_head(wl, e)
         k = k + a * e * mask[..., None].to(torch.float32)
     if wl.positional == "rotary":
         pos = torch.arange(n, device=device)
@@ -74,17 +79,17 @@ def make_prompt(wl: Workload, layer: int, device="cpu"):
 
 
 def make_step(wl: Workload, layer: int, step: int, device="cpu", prompt_len: int | None = None):
-    """Decode-step tensors q, k_new, v_new of one layer: fp16 [B, H, d]; step = 1..T."""
-    B, H, d = wl.batch, wl.n_heads, wl.head_dim
+    """Decode-step tensors of one layer: q fp16 [B, H, d]; k_new, v_new fp16 [B, Hkv, d]; step = 1..T."""
+    B, H, Hkv, d = wl.batch, wl.n_heads, wl.kv_heads, wl.head_dim
     n = wl.prompt_len if prompt_len is None else prompt_len
     q = _randn((B, H, d), _gen(wl, layer, "q", step, device), device)
-    k = _randn((B, H, d), _gen(wl, layer, "k", step, device), device)
-    v = _randn((B, H, d), _gen(wl, layer, "v", step, device), device)
+    k = _randn((B, Hkv, d), _gen(wl, layer, "k", step, device), device)
+    v = _randn((B, Hkv, d), _gen(wl, layer, "v", step, device), device)
     if wl.heavy_frac > 0:
         e = _heavy_direction(wl, layer, device)
         a = _heavy_amplitude(wl)
-        mask = torch.rand((B, H), generator=_gen(wl, layer, "hh_mask", step, device), device=device) < wl.heavy_frac
-        q = q + a * e
+        mask = torch.rand((B, Hkv), generator=_gen(wl, layer, "hh_mask", step, device), device=device) < wl.heavy_frac
+        q = q + a * _per_query_head(wl, e)
         k = k + a * e * mask[..., None].to(torch.float32)
     if wl.positional == "rotary":
         pos = torch.full((1,), n + step - 1, device=device)
@@ -94,9 +99,9 @@ def make_step(wl: Workload, layer: int, step: int, device="cpu", prompt_len: int
 
 
 def unit_list(wl: Workload, layer: int | None = None) -> np.ndarray:
-    """All (layer, batch, head) triples of the workload (or of one layer), int32 [U, 3]."""
+    """All (layer, batch, key/value head) triples of the workload (or of one layer), int32 [U, 3]."""
     layers = range(wl.n_layers) if layer is None else [layer]
-    out = [(l, b, h) for l in layers for b in range(wl.batch) for h in range(wl.n_heads)]
+    out = [(l, b, h) for l in layers for b in range(wl.batch) for h in range(wl.kv_heads)]
     return np.asarray(out, dtype=np.int32).reshape(-1, 3)
 
 
