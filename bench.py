@@ -36,15 +36,20 @@ UNIT = "steps/s"
 
 # ----------------------------------------------------------------------------- helpers
 def algorithmic_bytes_per_launch(wl: W.Workload) -> int:
-    """Bytes one layer call must move: K and V once, score/position state, the step's vectors."""
-    d, m = wl.head_dim, wl.budget_k + 1
-    per_unit = 4 * d * m + 12 * m + 12 * d
-    return wl.batch * wl.n_heads * per_unit
+    """Bytes one layer call must move per cache (batch row, key/value head): K and V once, score/position
+    state, the step's vectors (q in and out per query head of the group; k_new, v_new in; the new row written)."""
+    d, m, g = wl.head_dim, wl.budget_k + 1, wl.group
+    per_unit = 4 * d * m + 12 * m + (4 * g + 8) * d
+    return wl.batch * wl.kv_heads * per_unit
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one layer call (decode_kernel<128,4,2> + decode_close_kernel<128>) on a
-# c4_cerebras layer (1024 units, k = 2048, d = 128), from the ncu capture summarised in profiles/decode_kernel_c4_cerebras.md.
-C4_DECODE_TRAFFIC_BYTES = 1.124e9
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, both kernels of one layer call) from ncu captures, keyed by
+# what kf_describe_decode reports for the launch that was captured.  A launch of any other variant, split plan or
+# shape reports "traffic": null.
+CAPTURED_DECODE_TRAFFIC = {
+    # 1-layer case of the Cerebras-shaped workload (same per-launch shape as the 32-layer one)
+    "decode_kernel<128,5,2,0> + decode_close_kernel<128>; units=1024 k=2048 splits=3 tiles_per_split=24 group=1": 1.124e9,
+}
 
 
 def measured_peaks():
@@ -56,54 +61,62 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock, power and clock-event reasons through NVML (read-only queries) from a thread, every few
+    milliseconds, with host timestamps: started before the warm-up, and `summary(t0, t1)` keeps the samples taken
+    while the timed region ran."""
+    REASONS = (("hw_slowdown", "nvmlClocksEventReasonHwSlowdown"), ("hw_thermal_slowdown", "nvmlClocksEventReasonHwThermalSlowdown"),
+               ("sw_thermal_slowdown", "nvmlClocksEventReasonSwThermalSlowdown"), ("sw_power_cap", "nvmlClocksEventReasonSwPowerCap"))
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, device_index: int, period_s: float = 0.004):
+        self.rows, self.period, self.stop_flag, self.thread, self.h, self.nv = [], period_s, False, None, None, None
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = nv.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode() if not uuid.startswith("GPU-") else uuid.encode())
+            except Exception:
+                self.h = nv.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = nv
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(self.h, nv.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "25"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.t = threading.Thread(target=self._read, daemon=True)
-            self.t.start()
-        except Exception:
-            self.proc = None
+        if self.nv is None:
+            return
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append(line.strip())
+    def _run(self):
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                t = time.perf_counter()
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                watts = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                self.rows.append((t, float(mhz), int(mask), watts))
+            except Exception:
+                pass
+            time.sleep(self.period)
 
     def stop(self):
-        if not self.proc:
+        self.stop_flag = True
+        if self.thread:
+            self.thread.join(timeout=2)
+
+    def summary(self, t0: float, t1: float):
+        """Clock record of the samples taken between host times t0 and t1 (the timed region)."""
+        if self.nv is None:
             return None
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        self.t.join(timeout=2)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            f = [x.strip() for x in r.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for name, val in zip(names, f[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        if not sm:
+        rows = [r for r in self.rows if t0 <= r[0] <= t1]
+        if not rows:
             return None
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm), "reasons": sorted(reasons)}
+        reasons = sorted(name for name, attr in self.REASONS if any(r[2] & getattr(self.nv, attr) for r in rows))
+        return {"sm_mhz": statistics.median(r[1] for r in rows), "sm_mhz_min": min(r[1] for r in rows),
+                "sm_max_mhz": self.max_mhz, "samples": len(rows), "power_w_max": max(r[3] for r in rows),
+                "reasons": reasons, "source": "NVML queries every %d ms during the timed region" % round(self.period * 1e3)}
 
 
 def dist_setup(n_gpus: int):
@@ -144,6 +157,15 @@ def barrier(world: int):
         torch.cuda.synchronize()
 
 
+# ----------------------------------------------------------------------------- shared pieces
+def shape_config(wl: W.Workload, **extra) -> dict:
+    """The workload's shape, the same keys in both arms' `config`."""
+    c = {"workload": wl.name, "layers": wl.n_layers, "batch": wl.batch, "heads": wl.n_heads, "kv_heads": wl.kv_heads,
+         "head_dim": wl.head_dim, "prompt": wl.prompt_len, "budget_k": wl.budget_k, "recent_w": wl.recent_w}
+    c.update(extra)
+    return c
+
+
 # ----------------------------------------------------------------------------- oracle arm
 def oracle_sample_rate(wl: W.Workload, units: int, steps: int, seed: int = 0):
     """Times the CPU oracle's generation step on `units` sampled units for `steps` steps.
@@ -152,12 +174,13 @@ def oracle_sample_rate(wl: W.Workload, units: int, steps: int, seed: int = 0):
     Returns (unit_steps_per_second, threads, description)."""
     from oracle import keyformer_oracle as ko
     P = ko.Params(head_dim=wl.head_dim, n_heads=wl.n_heads, budget_k=wl.budget_k, recent_w=wl.recent_w,
-                  gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed)
+                  gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
+                  n_kv_heads=wl.kv_heads)
     lbh = W.sample_units(wl, units, seed)
-    U, d, k = lbh.shape[0], wl.head_dim, wl.budget_k
+    U, d, k, g = lbh.shape[0], wl.head_dim, wl.budget_k, wl.group
     n = min(wl.prompt_len, k + 64)
-    g = torch.Generator().manual_seed(seed)
-    mk = lambda *shape: torch.randn(*shape, generator=g).half().numpy()
+    gen = torch.Generator().manual_seed(seed)
+    mk = lambda *shape: torch.randn(*shape, generator=gen).half().numpy()
     K, V = mk(U, n, d), mk(U, n, d)
     keep = np.zeros((U, n), dtype=np.uint8)
     keep[:, n - k:] = 1
@@ -165,7 +188,7 @@ def oracle_sample_rate(wl: W.Workload, units: int, steps: int, seed: int = 0):
     st.prefill_prune(K, V, np.zeros((U, n)), keep_override=keep)
     st.n_prompt = wl.prompt_len
     st.pos[:, :k] += wl.prompt_len - n
-    inputs = [(mk(U, d), mk(U, d), mk(U, d)) for _ in range(steps)]
+    inputs = [(mk(U, g, d), mk(U, d), mk(U, d)) for _ in range(steps)]
     t0 = time.perf_counter()
     for s, (q, kn, vn) in enumerate(inputs, start=1):
         st.decode_score(s, q, kn, vn)
@@ -191,7 +214,7 @@ def run_reference(args, wl):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "note": "CPU oracle, extrapolated from a bounded sample per step"},
+            "config": shape_config(wl, note="CPU oracle; each step times a bounded sample of units and is extrapolated to all of them"),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0, "wall_s": wall}
@@ -199,139 +222,214 @@ def run_reference(args, wl):
 
 
 # ----------------------------------------------------------------------------- our arm
+class DecodeRun:
+    """A context of `wl` with its prompt phase done and the per-step inputs resident on the device."""
+
+    def __init__(self, wl, wl_data, dev, total_steps, splits=0, new_pos=False):
+        import paper_2403_09054_b200 as kf
+        self.kf, self.wl, self.dev = kf, wl, dev
+        self.gpu = kf.Keyformer(device=dev, n_layers=wl.n_layers, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
+                                n_kv_heads=wl.kv_heads,
+                                budget_k=wl.budget_k, recent_w=wl.recent_w, max_prompt_len=wl.prompt_len,
+                                gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
+                                bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
+                                alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None,
+                                decode_splits=splits, pos_mode=kf.KF_POS_NEW if new_pos else kf.KF_POS_ORIGINAL)
+        t0 = time.perf_counter()
+        for l in range(wl.n_layers):
+            q, k, v = W.make_prompt(wl_data, l, dev)
+            self.gpu.kf_prefill_score_prune(l, q, k, v)
+            del q, k, v
+        torch.cuda.synchronize()
+        self.prefill_s = time.perf_counter() - t0
+        assert self.gpu.kf_poll_error() == 0
+        L, B, H, Hkv, d = wl.n_layers, wl.batch, wl.n_heads, wl.kv_heads, wl.head_dim
+        self.Qs = torch.empty((total_steps, L, B, H, d), dtype=torch.float16, device=dev)
+        self.Kn = torch.empty((total_steps, L, B, Hkv, d), dtype=torch.float16, device=dev)
+        self.Vn = torch.empty_like(self.Kn)
+        for st_i in range(total_steps):
+            for l in range(L):
+                self.Qs[st_i, l], self.Kn[st_i, l], self.Vn[st_i, l] = W.make_step(wl_data, l, st_i + 1, dev)
+        self.out = torch.empty((L, B, H, d), dtype=torch.float16, device=dev)
+        self.stream = torch.cuda.current_stream()
+        self.s = 1            # next step number
+
+    def device_step(self, st=None):
+        s = self.s
+        for l in range(self.wl.n_layers):
+            self.gpu.kf_decode_step(l, s, self.Qs[s - 1, l], self.Kn[s - 1, l], self.Vn[s - 1, l], self.out[l], stream=st or self.stream)
+        self.s += 1
+
+    def time_device(self, steps, warmup, graph, world):
+        """`warmup` untimed steps, then `steps` timed ones between CUDA events on the launching stream.
+        Returns (total_ms, per-step ms list or None, launches, host times of the region)."""
+        for _ in range(warmup):
+            self.device_step()
+        barrier(world)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        launches0 = self.gpu.kf_launch_count()
+        if graph:
+            # The timed steps (distinct step numbers, each executed once, in order) are recorded into one CUDA
+            # graph before the timed region and replayed once inside it: the host's launch cost leaves the timing.
+            g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream(device=self.dev)
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(steps):
+                    self.device_step(torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            ev[0].record(self.stream)
+            g.replay()
+            ev[-1].record(self.stream)
+        else:
+            t0 = time.perf_counter()
+            ev[0].record(self.stream)
+            for i in range(steps):
+                self.device_step()
+                ev[i + 1].record(self.stream)
+        barrier(world)
+        t1 = time.perf_counter()
+        launches = self.gpu.kf_launch_count() - launches0
+        total_ms = ev[0].elapsed_time(ev[-1])
+        step_ms = None if graph else [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        assert self.gpu.kf_poll_error() == 0
+        return total_ms, step_ms, launches, (t0, t1)
+
+    def time_host(self, steps, world):
+        """End to end: host buffers in, host buffers out, through kf_decode_step_host.  Returns total ms."""
+        wl, L = self.wl, self.wl.n_layers
+        hq, hk, hv = self.Qs.cpu().pin_memory(), self.Kn.cpu().pin_memory(), self.Vn.cpu().pin_memory()
+        hout = torch.empty(self.out.shape, dtype=torch.float16).pin_memory()
+
+        def host_step():
+            s = self.s
+            for l in range(L):
+                self.gpu.kf_decode_step_host(l, s, hq[s - 1, l], hk[s - 1, l], hv[s - 1, l], hout[l],
+                                             wait=(l == L - 1), stream=self.stream)
+            self.s += 1
+
+        host_step()                   # warm-up of the copy path
+        barrier(world)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(self.stream)
+        for _ in range(steps):
+            host_step()
+        e1.record(self.stream)
+        barrier(world)
+        assert self.gpu.kf_poll_error() == 0
+        return e0.elapsed_time(e1)
+
+    def close(self):
+        self.gpu.kf_destroy()
+        del self.gpu, self.Qs, self.Kn, self.Vn, self.out
+        torch.cuda.empty_cache()
+
+
+def other_workload_point(name: str, dev, steps: int = 200, warmup: int = 5) -> dict:
+    """A single-layer workload whose step is shorter than a host launch: `steps` steps recorded into one CUDA
+    graph and replayed once.  Its KV state fits L2, so the bandwidth figure is algorithmic, not DRAM."""
+    wl = W.get_config(name)
+    run = DecodeRun(wl, wl, dev, warmup + steps)
+    total_ms, _, launches, _ = run.time_device(steps, warmup, True, 1)
+    us = total_ms * 1e3 / steps
+    kv_mb = 2 * wl.n_layers * wl.batch * wl.kv_heads * wl.budget_k * wl.head_dim * 2 / 1e6
+    point = {"workload": name, "steps_per_s": 1e6 / us, "us_per_step": us, "steps": steps,
+             "algorithmic_GBps": algorithmic_bytes_per_launch(wl) * wl.n_layers / (us * 1e-6) / 1e9,
+             "kv_state_MB": kv_mb, "note": "cache-resident (KV state fits L2), latency-bound; one CUDA graph of the timed steps",
+             "kernels": run.gpu.kf_describe_decode(), "gpu_launches": int(launches)}
+    run.close()
+    return point
+
+
 def run_ours(args, wl):
-    import paper_2403_09054_b200 as kf
     rank, world, local = dist_setup(args.gpus)
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
-    wl_r = rank_workload(wl, rank)
-    gpu = kf.Keyformer(device=dev, n_layers=wl.n_layers, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
-                       budget_k=wl.budget_k, recent_w=wl.recent_w, max_prompt_len=wl.prompt_len,
-                       gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
-                       bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
-                       alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None,
-                       decode_splits=args.splits,
-                       pos_mode=kf.KF_POS_NEW if args.new_pos else kf.KF_POS_ORIGINAL)
-    t_pre = time.perf_counter()
-    for l in range(wl.n_layers):
-        q, k, v = W.make_prompt(wl_r, l, dev)
-        gpu.kf_prefill_score_prune(l, q, k, v)
-        del q, k, v
-    torch.cuda.synchronize()
-    t_pre = time.perf_counter() - t_pre
-    assert gpu.kf_poll_error() == 0
-
-    L, B, H, d = wl.n_layers, wl.batch, wl.n_heads, wl.head_dim
-    total_steps = args.warmup + 2 * args.steps + 1
-    Qs = torch.empty((total_steps, L, B, H, d), dtype=torch.float16, device=dev)
-    Kn, Vn = torch.empty_like(Qs), torch.empty_like(Qs)
-    for st_i in range(total_steps):
-        for l in range(L):
-            Qs[st_i, l], Kn[st_i, l], Vn[st_i, l] = W.make_step(wl_r, l, st_i + 1, dev)
-    out = torch.empty((L, B, H, d), dtype=torch.float16, device=dev)
-    stream = torch.cuda.current_stream()
-
-    def device_step(s, st=None):
-        for l in range(L):
-            gpu.kf_decode_step(l, s, Qs[s - 1, l], Kn[s - 1, l], Vn[s - 1, l], out[l], stream=st or stream)
-
-    s = 1
-    for _ in range(args.warmup):
-        device_step(s); s += 1
-    barrier(world)
     sampler = ClockSampler(local)
-    sampler.start()
-    launches0 = gpu.kf_launch_count()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    if args.graph:
-        # The K timed steps (distinct step numbers, each executed once, in order) are recorded into one CUDA
-        # graph before the timed region and replayed once inside it: the host's launch cost leaves the timing.
-        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream(device=dev)
-        launches0 = gpu.kf_launch_count()
-        with torch.cuda.graph(graph, stream=side):
-            for i in range(args.steps):
-                device_step(s + i, torch.cuda.current_stream())
-        s += args.steps
-        torch.cuda.synchronize()
-        ev[0].record(stream)
-        graph.replay()
-        ev[-1].record(stream)
-    else:
-        ev[0].record(stream)
-        for i in range(args.steps):
-            device_step(s); s += 1
-            ev[i + 1].record(stream)
-    barrier(world)
-    clocks = sampler.stop()
-    launches = gpu.kf_launch_count() - launches0
-    total_ms = ev[0].elapsed_time(ev[-1])
-    step_ms = ([total_ms / args.steps] if args.graph else
-               [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)])
+    sampler.start()                                       # before the warm-up; the summary keeps the timed region's samples
+    wl_r = rank_workload(wl, rank)
+    run = DecodeRun(wl, wl_r, dev, args.warmup + 2 * args.steps + 1, splits=args.splits, new_pos=args.new_pos)
+    total_ms, step_ms, launches, (t0, t1) = run.time_device(args.steps, args.warmup, args.graph, world)
+    clocks = sampler.summary(t0, t1)
     total_ms = max_over_ranks(total_ms, world, dev)
-    assert gpu.kf_poll_error() == 0
     ms_per_step = total_ms / args.steps
     value = whole_job_rate(ms_per_step, world)
-
-    vec_bytes = B * H * d * 2
     e2e_ms = None
     if not args.no_e2e:
-        # end to end: host buffers in, host buffers out, through kf_decode_step_host
-        hq, hk, hv = Qs.cpu().pin_memory(), Kn.cpu().pin_memory(), Vn.cpu().pin_memory()
-        hout = torch.empty((L, B, H, d), dtype=torch.float16).pin_memory()
+        e2e_ms = max_over_ranks(run.time_host(args.steps, world), world, dev) / args.steps
+    describe = run.gpu.kf_describe_decode()
+    prefill_s = run.prefill_s
+    run.close()
+    sampler.stop()
 
-        def host_step(step):
-            for l in range(L):
-                gpu.kf_decode_step_host(l, step, hq[step - 1, l], hk[step - 1, l], hv[step - 1, l], hout[l],
-                                        wait=(l == L - 1), stream=stream)
-
-        host_step(s); s += 1          # warm-up of the copy path
-        barrier(world)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(args.steps):
-            host_step(s); s += 1
-        e1.record(stream)
-        barrier(world)
-        e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
-        assert gpu.kf_poll_error() == 0
-
+    L, B, H, d = wl.n_layers, wl.batch, wl.n_heads, wl.head_dim
+    vec_bytes_q, vec_bytes_kv = B * H * d * 2, B * wl.kv_heads * d * 2
+    kv_bytes = 2 * L * B * wl.kv_heads * wl.budget_k * d * 2
     line = None
-    kv_bytes = 2 * L * B * H * wl.budget_k * d * 2
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         abytes = algorithmic_bytes_per_launch(wl)
-        launch_ms = statistics.median(step_ms) / L      # one layer call (streaming + closing kernel), back to back
+        launch_ms = ms_per_step / L       # one layer call (streaming + closing kernel), back to back: the mean, as `value`
         achieved = abytes / (launch_ms * 1e-3) / 1e9
+        traffic = args.traffic if args.traffic is not None else CAPTURED_DECODE_TRAFFIC.get(describe)
         cpu_rate, threads, desc = oracle_sample_rate(wl, args.cpu_units, args.cpu_steps)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f16 storage, f32 arithmetic", "data": "synthetic",
-            "config": {"workload": wl.name, "layers": L, "batch": B, "heads": H, "head_dim": d, "prompt": wl.prompt_len,
-                       "budget_k": wl.budget_k, "recent_w": wl.recent_w, "tokens_per_s": value * B,
-                       "l2": ("inputs larger than L2 (KV state %.1f GB per GPU)" if kv_bytes > 126e6 else
-                              "KV state of this workload (%.3f GB) fits L2: cache-resident by nature, no flush") % (kv_bytes / 1e9),
-                       "prefill_s": t_pre, "decode_splits": args.splits,
-                       "positions_in_bias": "places within the reduced cache" if args.new_pos else "original",
-                       "launch_mode": "one CUDA graph of the timed steps" if args.graph else "stream launches"},
-            "roofline": {"bound": "hbm", "kernel": "decode_kernel (+ decode_close_kernel: the duration is one layer call)", "achieved": achieved, "peak": peaks["hbm_gbs"],
+            "config": shape_config(wl, tokens_per_s=value * B,
+                                   l2=("inputs larger than L2 (KV state %.1f GB per GPU)" if kv_bytes > 126e6 else
+                                       "KV state of this workload (%.3f GB) fits L2: cache-resident by nature, no flush") % (kv_bytes / 1e9),
+                                   prefill_s=prefill_s, decode_splits=args.splits,
+                                   positions_in_bias="places within the reduced cache" if args.new_pos else "original",
+                                   launch_mode="one CUDA graph of the timed steps" if args.graph else "stream launches"),
+            "roofline": {"bound": "hbm", "kernel": describe, "achieved": achieved, "peak": peaks["hbm_gbs"],
                          "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": abytes,
-                         "launch_ms": launch_ms,
-                         "traffic": args.traffic if args.traffic is not None else
-                         (C4_DECODE_TRAFFIC_BYTES if wl.name.startswith("c4_cerebras") and args.splits == 0 else None)},
+                         "launch_ms": launch_ms, "launch_ms_is": "ms_per_step / layers (mean over the timed steps; the duration of one layer call = both kernels)",
+                         "traffic": traffic,
+                         "traffic_is": ("DRAM bytes of one layer call from the ncu capture of exactly this kernel variant and shape"
+                                        if traffic is not None else "no capture of this kernel variant and shape")},
             "cpu_baseline": {"value": cpu_rate / wl.units, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
-            "e2e": {"value": (world * 1e3 / e2e_ms) if e2e_ms else None, "unit": UNIT, "h2d_bytes_per_step": 3 * L * vec_bytes,
-                    "d2h_bytes_per_step": L * vec_bytes},
+            "e2e": {"value": (world * 1e3 / e2e_ms) if e2e_ms else None, "unit": UNIT,
+                    "h2d_bytes_per_step": L * (vec_bytes_q + 2 * vec_bytes_kv), "d2h_bytes_per_step": L * vec_bytes_q},
             "gpu_launches": int(launches), "clocks": clocks,
-            "step_ms": {"min": min(step_ms), "median": statistics.median(step_ms), "max": max(step_ms)},
         }
+        if step_ms:
+            line["step_ms"] = {"mean": statistics.mean(step_ms), "median": statistics.median(step_ms),
+                               "min": min(step_ms), "max": max(step_ms)}
+            line["roofline"]["achieved_at_median_step"] = abytes * L / (statistics.median(step_ms) * 1e-3) / 1e9
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    if rank == 0:
+        if args.extras and world == 1:
+            # outside the timed region: the other workload shapes and the prompt phase, a few hundred ms each
+            line["other_workloads"] = [other_workload_point(n, dev) for n in ("c1_tiny", "c2_gptj", "c3_mpt")]
+            if wl.name == "c4_cerebras":
+                line["other_workloads"].append(gqa_point(dev))
+            line["prefill"] = prefill_point(W.get_config("c5_prefill_8k"), dev, budget_frac=0.5, steps=5, warmup=3)
         print(json.dumps(line))
-    gpu.kf_destroy()
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
     return line
+
+
+def gqa_point(dev, steps: int = 20, warmup: int = 3) -> dict:
+    """The Cerebras-shaped model with 8 KV heads shared by its 32 query heads (4 per group), 8 layers of it:
+    stream launches, inputs larger than L2."""
+    wl = W.get_config("c4_cerebras_gqa8").scaled(n_layers=8)
+    run = DecodeRun(wl, wl, dev, warmup + steps)
+    total_ms, step_ms, launches, _ = run.time_device(steps, warmup, False, 1)
+    peaks, peak_kind = measured_peaks()
+    ms = total_ms / steps
+    achieved = algorithmic_bytes_per_launch(wl) * wl.n_layers / (ms * 1e-3) / 1e9
+    point = {"workload": wl.name + "[layers=8]", "heads": wl.n_heads, "kv_heads": wl.kv_heads, "steps_per_s": 1e3 / ms,
+             "us_per_layer_call": ms * 1e3 / wl.n_layers, "algorithmic_GBps": achieved, "frac_of_measured_peak": achieved / peaks["hbm_gbs"],
+             "kv_state_MB": 2 * wl.n_layers * wl.batch * wl.kv_heads * wl.budget_k * wl.head_dim * 2 / 1e6,
+             "kernels": run.gpu.kf_describe_decode(), "gpu_launches": int(launches), "note": "stream launches; KV state larger than L2"}
+    run.close()
+    return point
 
 
 # ----------------------------------------------------------------------------- prompt phase
@@ -344,32 +442,31 @@ def run_ours(args, wl):
 #   MUFU:    two logarithms, one exponential (one issue slot each; 8 cycles each on the 16-lane XU)       ->  3
 PREFILL_INT_INSTR, PREFILL_FP_INSTR, PREFILL_MUFU_INSTR = 13, 7, 3
 # dram__bytes_read.sum + dram__bytes_write.sum of the two prefill_tc launches of one call on c5_prefill_2k (B8 H32 d128,
-# n 2048: Q + K = 268 MB, each read from DRAM once per sweep), from the ncu capture summarised in
-# profiles/prefill_tc_c5_prefill_sweep.md.  It does not scale with the logit count (re-reads are served by L2), so the
-# other prompt lengths report no traffic figure.
+# n 2048: Q + K = 268 MB, each read from DRAM once per sweep), from an ncu capture.  It does not scale with the logit
+# count (re-reads are served by L2), so the other prompt lengths report no traffic figure.
 C5_2K_PREFILL_TRAFFIC_BYTES = (268.5 + 4.8 + 270.6 + 5.4) * 1e6
+# sm__pipe_tensor_cycles_active / XU pipe / issue-active of the two sweeps in that capture (n = 2048), in percent
+C5_2K_PREFILL_COUNTERS = {"captured_at": "n = 2048", "tensor_pipe_pct": [8, 10], "xu_pipe_pct": [46, 56], "issue_active_pct": [57, 61]}
 PREFILL_LANE_INSTR_PER_LOGIT_SWEEP = 2 * PREFILL_INT_INSTR + PREFILL_FP_INSTR + PREFILL_MUFU_INSTR   # 36 FP32-lane slots
 ALU_LANES_PER_SM, N_SM = 128, 148
 
 
-def run_prefill(args, wl):
-    """Times kf_prefill_score_prune (prompt scoring on the tensor cores + select + gather) for one layer."""
+def prefill_point(wl, dev, budget_frac, steps, warmup, with_attention=False, simt=False, world=1, sampler=None):
+    """Times kf_prefill_score_prune (prompt scoring on the tensor cores + select + gather) for one layer.
+    Returns (ms per call, launches, clock summary, the scaled workload)."""
     import paper_2403_09054_b200 as kf
-    rank, world, local = dist_setup(args.gpus)
-    dev = torch.device("cuda", local)
-    torch.cuda.set_device(dev)
     n = wl.prompt_len
-    kk = max(1, int(round(n * args.budget_frac)))
-    wl = rank_workload(wl.scaled(budget_k=kk, recent_w=kk // 4), rank)
-    gpu = kf.Keyformer(device=dev, n_layers=1, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
+    kk = max(1, int(round(n * budget_frac)))
+    wl = wl.scaled(budget_k=kk, recent_w=kk // 4)
+    gpu = kf.Keyformer(device=dev, n_layers=1, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim, n_kv_heads=wl.kv_heads,
                        budget_k=wl.budget_k, recent_w=wl.recent_w, max_prompt_len=n, gen_len_T=0,
                        tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
                        bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
                        alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None,
-                       prefill_impl=kf.KF_PREFILL_SIMT if args.prefill_simt else kf.KF_PREFILL_TENSOR)
+                       prefill_impl=kf.KF_PREFILL_SIMT if simt else kf.KF_PREFILL_TENSOR)
     q, k, v = W.make_prompt(wl, 0, dev)
     stream = torch.cuda.current_stream()
-    attn_out = torch.empty_like(q) if args.with_attention else None
+    attn_out = torch.empty_like(q) if with_attention else None
 
     def call():
         if attn_out is None:
@@ -377,48 +474,66 @@ def run_prefill(args, wl):
         else:
             gpu.kf_prefill_attend_score_prune(0, q, k, v, attn_out, stream=stream)
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         call()
     barrier(world)
-    sampler = ClockSampler(local)
-    sampler.start()
     launches0 = gpu.kf_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
     e0.record(stream)
-    for _ in range(args.steps):
+    for _ in range(steps):
         call()
     e1.record(stream)
     barrier(world)
-    clocks = sampler.stop()
+    t1 = time.perf_counter()
     launches = gpu.kf_launch_count() - launches0
-    ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    ms = e0.elapsed_time(e1) / steps
     assert gpu.kf_poll_error() == 0
-    if rank == 0:
-        units = wl.batch * wl.n_heads
-        logits = units * n * (n + 1) // 2
-        lane_instr = 2 * PREFILL_LANE_INSTR_PER_LOGIT_SWEEP * logits
-        sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
-        peak = N_SM * ALU_LANES_PER_SM * 1965.0e6 / 1e12
-        achieved = lane_instr / (ms * 1e-3) / 1e12
-        line = {
-            "metric": "prompt score-and-prune calls/sec (one layer)", "value": world * 1e3 / ms, "unit": "calls/s",
-            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f16 operands, f32 accumulate and score arithmetic",
-            "data": "synthetic",
-            "config": {"workload": wl.name, "phase": "prefill", "with_attention_output": bool(args.with_attention), "batch": wl.batch, "heads": wl.n_heads,
-                       "head_dim": wl.head_dim, "prompt": n, "budget_k": wl.budget_k, "recent_w": wl.recent_w,
-                       "causal_logits": logits, "G_logits_per_s": logits / ms / 1e6,
-                       "qk_tflops_both_sweeps": 2 * 2 * logits * wl.head_dim / (ms * 1e-3) / 1e12,
-                       "l2": "Q, K, V of the call (%.0f MB) exceed L2" % (3 * units * n * wl.head_dim * 2 / 1e6)},
-            "roofline": {"bound": "alu", "kernel": "prefill_tc (two sweeps)", "achieved": achieved, "peak": peak,
-                         "unit": "T FP32-lane issue slots/s (INT32 instructions count twice)", "frac": achieved / peak,
-                         "traffic": C5_2K_PREFILL_TRAFFIC_BYTES if (wl.name == "c5_prefill_2k" and not args.prefill_simt) else None,
-                         "lane_instr_per_logit_sweep": PREFILL_LANE_INSTR_PER_LOGIT_SWEEP,
-                         "peak_kind": "148 SMs x 128 lanes x 1965 MHz", "sm_mhz_seen": sm_mhz},
-            "gpu_launches": int(launches), "clocks": clocks,
-        }
-        print(json.dumps(line))
     gpu.kf_destroy()
+    del q, k, v, attn_out, gpu
+    torch.cuda.empty_cache()
+    units = wl.batch * wl.n_heads
+    logits = units * n * (n + 1) // 2
+    peak = N_SM * ALU_LANES_PER_SM * 1965.0e6 / 1e12
+    achieved = 2 * PREFILL_LANE_INSTR_PER_LOGIT_SWEEP * logits / (ms * 1e-3) / 1e12
+    point = {"workload": wl.name, "prompt": n, "budget_k": wl.budget_k, "recent_w": wl.recent_w, "batch": wl.batch,
+             "heads": wl.n_heads, "kv_heads": wl.kv_heads, "head_dim": wl.head_dim, "with_attention_output": bool(with_attention),
+             "ms_per_call": ms, "steps": steps, "causal_logits": logits, "G_logits_per_s": logits / ms / 1e6,
+             "qk_tflops_both_sweeps": 2 * 2 * logits * wl.head_dim / (ms * 1e-3) / 1e12,
+             "roofline": {"bound": "alu", "kernel": "prefill_tc (two sweeps)", "achieved": achieved, "peak": peak,
+                          "unit": "T FP32-lane issue slots/s (INT32 instructions count twice)", "frac": achieved / peak,
+                          "lane_instr_per_logit_sweep": PREFILL_LANE_INSTR_PER_LOGIT_SWEEP,
+                          "peak_kind": "148 SMs x 128 lanes x 1965 MHz",
+                          "traffic": C5_2K_PREFILL_TRAFFIC_BYTES if (wl.name == "c5_prefill_2k" and not simt) else None,
+                          "ncu_counters": C5_2K_PREFILL_COUNTERS},
+             "gpu_launches": int(launches)}
+    if sampler is not None:
+        point["clocks"] = sampler.summary(t0, t1)
+    return point
+
+
+def run_prefill(args, wl):
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    sampler = ClockSampler(local)
+    sampler.start()
+    pt = prefill_point(rank_workload(wl, rank), dev, args.budget_frac, args.steps, args.warmup,
+                       with_attention=args.with_attention, simt=args.prefill_simt, world=world, sampler=sampler)
+    sampler.stop()
+    ms = max_over_ranks(pt["ms_per_call"], world, dev)
+    if rank == 0:
+        line = {"metric": "prompt score-and-prune calls/sec (one layer)", "value": world * 1e3 / ms, "unit": "calls/s",
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f16 operands, f32 accumulate and score arithmetic",
+                "data": "synthetic",
+                "config": {k: pt[k] for k in ("workload", "prompt", "budget_k", "recent_w", "batch", "heads", "kv_heads", "head_dim",
+                                              "with_attention_output", "causal_logits", "G_logits_per_s", "qk_tflops_both_sweeps")},
+                "roofline": pt["roofline"], "gpu_launches": pt["gpu_launches"], "clocks": pt.get("clocks")}
+        line["config"]["phase"] = "prefill"
+        line["config"]["l2"] = "Q, K, V of the call (%.0f MB) exceed L2" % (
+            (pt["heads"] + 2 * pt["kv_heads"]) * pt["batch"] * pt["prompt"] * pt["head_dim"] * 2 / 1e6)
+        print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
@@ -435,8 +550,8 @@ def main():
     ap.add_argument("--cpu-units", type=int, default=512)
     ap.add_argument("--cpu-steps", type=int, default=64)
     ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per launch of the decode kernel from an ncu capture (default: the committed "
-                         "capture of the current kernel on the Cerebras-shaped layer, see profiles/)")
+                    help="DRAM bytes per layer call from an ncu capture (default: the stored capture of exactly the "
+                         "kernel variant and shape that is launched, else null)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling a small case)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (a scaled copy of the workload)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (profiling a small case)")
@@ -451,6 +566,9 @@ def main():
     ap.add_argument("--new-pos", action="store_true",
                     help="decode phase: the bias counts places within the reduced cache (only matters with ALiBi workloads)")
     ap.add_argument("--prefill-simt", action="store_true", help="prefill phase: CUDA-core scoring instead of tcgen05")
+    ap.add_argument("--no-extras", dest="extras", action="store_false",
+                    help="decode phase: skip the blocks measured after the timed region (the three single-layer workloads, "
+                         "the shared-KV-head point and the prompt phase)")
     args = ap.parse_args()
     wl = W.get_config(args.workload)
     if args.layers > 0:

@@ -88,6 +88,12 @@ typedef struct kf_config {
   float   noise_mu;        /* mean of KF_NOISE_GAUSS (the paper matches Gumbel's 0.5772)          */
   float   noise_sigma;     /* standard deviation of KF_NOISE_GAUSS (1.2825 in the paper)         */
   int32_t pos_mode;        /* KF_POS_*; KF_POS_NEW keeps one more int32 per cache slot            */
+  int32_t debug_canaries;  /* 1: a 256-byte guard of a known pattern follows every sub-buffer of the workspace
+                              (kf_workspace_bytes grows accordingly); kf_check_canaries verifies them.  0: none */
+  int32_t debug_fail_first_wait; /* self-test of the error path: 1 makes every warp of the generation kernel give up
+                              its first wait for a cache tile at once, as if the bounded wait had run out: the step
+                              reports KF_ETIMEOUT through kf_poll_error (after waiting, with the full limit, for the
+                              copies in flight) and leaves the layer's state undefined.  0 in normal use.          */
 } kf_config;
 
 /* Bytes of device workspace kf_create needs for this configuration
@@ -107,7 +113,8 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
  * top-(k-w) of the others by f_theta (ties: lower position), and store the
  * kept K/V rows, positions and scores in ascending position order.  If
  * n_prompt <= k everything is kept.
- *   d_q, d_k, d_v : DEVICE fp16 [B][H][n_prompt][d], read only, 16-byte aligned (KF_EINVAL otherwise).
+ *   d_q, d_k, d_v : DEVICE fp16 [B][H][n_prompt][d], read only, each 16-byte aligned (KF_EINVAL otherwise,
+ *                   with either scoring implementation).
  *   d_score_opt   : DEVICE fp32 [B][H][n_prompt] or NULL; receives f_theta
  *                   before pruning.
  * Must be called once per layer before that layer's first kf_decode_step. */
@@ -138,11 +145,15 @@ int kf_prefill_attend_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
  *   the w most recent (ties: the higher position leaves); the new token's
  *   row takes the freed slot.  Slot order is therefore arbitrary; the
  *   position array identifies the entries.
- *   d_q, d_knew, d_vnew : DEVICE fp16 [B][H][d].
- *   d_out               : DEVICE fp16 [B][H][d].
+ *   d_q, d_knew, d_vnew : DEVICE fp16 [B][H][d], each 16-byte aligned (KF_EINVAL otherwise).
+ *   d_out               : DEVICE fp16 [B][H][d], 16-byte aligned.
  *   d_score_opt         : DEVICE fp32 [B][H][k+1] or NULL; receives z for the
  *                         slots [0, len) followed by the new token at index len.
- * Steps of a layer must be issued in increasing order starting from 1. */
+ * The steps of a layer must be consecutive: the first call after the prompt phase (or after kf_import_state with
+ * last_step = s) has step 1 (s + 1), every later call the previous step plus one; anything else is KF_ESTATE and
+ * enqueues nothing.  (The position of the token, hence its noise and temperature, follows from the step.)
+ * A unit whose entry count in the workspace is outside 0..k (a damaged or foreign state image) is left untouched
+ * and reported as KF_EBOUNDS by kf_poll_error. */
 int kf_decode_step(kf_ctx* ctx, int32_t layer, int32_t step,
                    const void* d_q, const void* d_knew, const void* d_vnew,
                    void* d_out, float* d_score_opt, void* stream);
@@ -168,8 +179,9 @@ typedef struct kf_static_step {
   int32_t budget_k, recent_w;         /* k, w                                               */
   int32_t layer;                      /* layer index (part of the noise coordinates)        */
   int32_t position;                   /* p: original position of the token being generated  */
-  int32_t noise_mode, bias_mode;      /* KF_NOISE_*, KF_BIAS_*                              */
-  int32_t reserved;                   /* must be 0                                          */
+  int32_t noise_mode, bias_mode;      /* KF_NOISE_GUMBEL, KF_NOISE_NONE or KF_NOISE_CONST (the Gaussian alternative needs
+                                         its mean and deviation: use a context); KF_BIAS_*  */
+  int32_t reserved;                   /* must be 0 (KF_EINVAL otherwise)                    */
   double  tau;                        /* temperature of this step (Eq. 12, computed by the caller) */
   uint64_t noise_seed;
   float   logit_scale;                /* 0 => 1/sqrt(d)                                     */
@@ -194,6 +206,8 @@ typedef struct kf_static_step {
  *   d_acc     : DEVICE fp32 [B][H][k]      accumulated scores f_theta, updated in place
  *   d_len     : DEVICE int32 [B][H]        entries in use, updated in place
  *   d_q, d_knew, d_vnew, d_out, d_score_opt : as in kf_decode_step
+ *   d_K, d_V, d_q, d_knew, d_vnew, d_out must be 16-byte aligned, d_pos, d_acc, d_len 4-byte aligned (KF_EINVAL
+ *   otherwise).  A unit whose d_len entry is outside 0..k is skipped: nothing of it is read or written.
  *
  * Limits and rules
  *   - The step needs about 4*B*H*(k+1) + 4*B*H*splits*(d+4) bytes of scratch; if that exceeds the
@@ -249,6 +263,19 @@ int kf_import_state(kf_ctx* ctx, int32_t layer, const void* d_src, size_t bytes,
 /* Waits for `stream`, then returns and clears the device error word:
  * 0, KF_ETIMEOUT or KF_EBOUNDS. */
 int kf_poll_error(kf_ctx* ctx, void* stream);
+
+/* Debug layout only (kf_config.debug_canaries = 1): waits for `stream`, then compares the guard behind every
+ * sub-buffer of the workspace with its pattern.  KF_OK if all are intact; KF_EBOUNDS if one was overwritten, with
+ * *first_bad (may be NULL) = index of the sub-buffer in front of it, in layout order: K, V, scores, positions,
+ * entry counts, adjusted-logit scratch, split partials, error word, slopes, prompt scores, kept indices, host
+ * staging, the two row-statistics arrays, places.  KF_EINVAL for a context without guards. */
+int kf_check_canaries(kf_ctx* ctx, void* stream, int32_t* first_bad);
+
+/* Writes into buf (n bytes, always terminated) which kernels a kf_decode_step of this context launches, with their
+ * template arguments, and how a layer call is cut into CTAs, e.g.
+ * "decode_kernel<128,5,2,0> + decode_close_kernel<128>; units=1024 k=2048 splits=3 tiles_per_split=24 group=1".
+ * Profiles are keyed by this string.  Returns the length the full text needs (as snprintf does) or KF_EINVAL. */
+int kf_describe_decode(const kf_ctx* ctx, char* buf, size_t n);
 
 /* Number of kernel launches this context has enqueued so far. */
 int64_t kf_launch_count(const kf_ctx* ctx);

@@ -23,7 +23,7 @@ KF_POS_ORIGINAL, KF_POS_NEW = 0, 1
 EXPORTS = ("kf_workspace_bytes", "kf_create", "kf_prefill_score_prune", "kf_decode_step",
            "kf_decode_step_host", "kf_view_state", "kf_poll_error", "kf_launch_count",
            "kf_destroy", "kf_strerror", "kf_decode_step_static", "kf_state_bytes", "kf_export_state", "kf_import_state",
-           "kf_prefill_attend", "kf_prefill_attend_score_prune", "kf_view_place", "kf_compact_layer")
+           "kf_prefill_attend", "kf_prefill_attend_score_prune", "kf_view_place", "kf_compact_layer", "kf_check_canaries", "kf_describe_decode")
 
 
 class kf_config(C.Structure):
@@ -35,6 +35,7 @@ class kf_config(C.Structure):
         ("logit_scale", C.c_float), ("noise_const", C.c_float),
         ("decode_splits", C.c_int32), ("prefill_impl", C.c_int32),
         ("noise_mu", C.c_float), ("noise_sigma", C.c_float), ("pos_mode", C.c_int32),
+        ("debug_canaries", C.c_int32), ("debug_fail_first_wait", C.c_int32),
     ]
 
 
@@ -88,6 +89,10 @@ def _load() -> C.CDLL:
     lib.kf_view_state.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
     lib.kf_poll_error.restype = C.c_int
     lib.kf_poll_error.argtypes = [vp, vp]
+    lib.kf_check_canaries.restype = C.c_int
+    lib.kf_check_canaries.argtypes = [vp, vp, C.POINTER(i32)]
+    lib.kf_describe_decode.restype = C.c_int
+    lib.kf_describe_decode.argtypes = [vp, C.c_char_p, C.c_size_t]
     lib.kf_launch_count.restype = C.c_int64
     lib.kf_launch_count.argtypes = [vp]
     lib.kf_destroy.restype = C.c_int
@@ -119,7 +124,8 @@ def kf_strerror(code: int) -> str:
 def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_prompt_len, gen_len_T,
                 tau_init=1.0, tau_end=2.0, noise_seed=0, noise_mode=KF_NOISE_GUMBEL, bias_mode=KF_BIAS_NONE,
                 alibi_slopes=None, logit_scale=0.0, noise_const=0.5772, decode_splits=0,
-                prefill_impl=KF_PREFILL_TENSOR, noise_mu=0.5772, noise_sigma=1.2825, pos_mode=KF_POS_ORIGINAL):
+                prefill_impl=KF_PREFILL_TENSOR, noise_mu=0.5772, noise_sigma=1.2825, pos_mode=KF_POS_ORIGINAL,
+                debug_canaries=0, debug_fail_first_wait=0):
     """Fill a kf_config; returns (config, keepalive) where keepalive holds the slopes array."""
     cfg = kf_config()
     cfg.n_layers, cfg.batch, cfg.n_heads, cfg.head_dim = n_layers, batch, n_heads, head_dim
@@ -135,6 +141,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
     cfg.decode_splits, cfg.prefill_impl = decode_splits, prefill_impl
     cfg.noise_mu, cfg.noise_sigma = noise_mu, noise_sigma
     cfg.pos_mode = pos_mode
+    cfg.debug_canaries, cfg.debug_fail_first_wait = debug_canaries, debug_fail_first_wait
     return cfg, keep
 
 
@@ -293,6 +300,17 @@ class Keyformer:
 
     def kf_poll_error(self, stream=None) -> int:
         return int(LIB.kf_poll_error(self._h, _stream_ptr(stream)))
+
+    def kf_check_canaries(self, stream=None):
+        """(status, index of the first sub-buffer whose guard was overwritten or -1); debug layout only."""
+        bad = C.c_int32(-1)
+        rc = int(LIB.kf_check_canaries(self._h, _stream_ptr(stream), C.byref(bad)))
+        return rc, bad.value
+
+    def kf_describe_decode(self) -> str:
+        buf = C.create_string_buffer(256)
+        _check(min(0, int(LIB.kf_describe_decode(self._h, buf, len(buf)))), "kf_describe_decode")
+        return buf.value.decode()
 
     def kf_launch_count(self) -> int:
         return int(LIB.kf_launch_count(self._h))

@@ -15,6 +15,10 @@ namespace {
 
 constexpr size_t ALIGN = 256;
 inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+inline bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+constexpr size_t GUARD_BYTES = 256;
+constexpr int GUARD_BYTE = 0xA5;
 
 struct Layout {
   size_t K, V, acc, pos, len;          // per-layer strides are kv_layer / sc_layer / len_layer
@@ -24,6 +28,9 @@ struct Layout {
   size_t total;
   size_t kv_layer, sc_layer, len_layer; // bytes per layer
   int units, max_splits;
+  // debug_canaries: a guard of GUARD_BYTES follows every sub-buffer; `guards` holds their offsets in layout order
+  // (K, V, acc, pos, len, y_scratch, partials, err, slopes, acc_full, idx, staging, lse2, lse_x, place)
+  std::vector<size_t> guards;
 };
 
 bool config_ok(const kf_config* c) {
@@ -41,10 +48,9 @@ bool config_ok(const kf_config* c) {
   if (c->prefill_impl != KF_PREFILL_TENSOR && c->prefill_impl != KF_PREFILL_SIMT) return false;
   if (c->pos_mode != KF_POS_ORIGINAL && c->pos_mode != KF_POS_NEW) return false;
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
+  if (c->debug_canaries < 0 || c->debug_canaries > 1 || c->debug_fail_first_wait < 0 || c->debug_fail_first_wait > 1) return false;
   return true;
 }
-
-int tiles_of(int k) { return (k + kf::decode_tile_rows() - 1) / kf::decode_tile_rows(); }
 
 Layout make_layout(const kf_config* c) {
   Layout L{};
@@ -56,21 +62,28 @@ Layout make_layout(const kf_config* c) {
   L.sc_layer = align_up(units * k * 4);
   L.len_layer = align_up(units * 4);
   size_t off = 0;
-  L.K = off; off += nl * L.kv_layer;
-  L.V = off; off += nl * L.kv_layer;
-  L.acc = off; off += nl * L.sc_layer;
-  L.pos = off; off += nl * L.sc_layer;
-  L.len = off; off += nl * L.len_layer;
-  L.y_scratch = off; off += align_up(units * (k + 1) * 4);
-  L.partials = off; off += align_up(units * (size_t)L.max_splits * (4 + d) * 4);
-  L.err = off; off += ALIGN;
-  L.slopes = off; off += align_up((size_t)c->n_heads * 4);
-  L.acc_full = off; off += align_up(units * (size_t)c->max_prompt_len * 4);
-  L.idx = off; off += align_up(units * k * 4);
-  L.staging = off; off += 8 * align_up(units * d * 2);   // two sets of (q, k_new, v_new, out)
-  L.lse2 = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
-  L.lse_x = off; off += align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4);
-  L.place = off; if (c->pos_mode == KF_POS_NEW) off += nl * L.sc_layer;
+  auto carve = [&](size_t bytes) {   // appends a sub-buffer (and, in the debug layout, the guard behind it)
+    const size_t at = off;
+    off += bytes;
+    if (c->debug_canaries) { L.guards.push_back(off); off += GUARD_BYTES; }
+    return at;
+  };
+  L.K = carve(nl * L.kv_layer);
+  L.V = carve(nl * L.kv_layer);
+  L.acc = carve(nl * L.sc_layer);
+  L.pos = carve(nl * L.sc_layer);
+  L.len = carve(nl * L.len_layer);
+  L.y_scratch = carve(align_up(units * (k + 1) * 4));
+  L.partials = carve(align_up(units * (size_t)L.max_splits * (4 + d) * 4));
+  L.err = carve(ALIGN);
+  L.slopes = carve(align_up((size_t)c->n_heads * 4));
+  L.acc_full = carve(align_up(units * (size_t)c->max_prompt_len * 4));
+  L.idx = carve(align_up(units * k * 4));
+  L.staging = carve(8 * align_up(units * d * 2));   // two sets of (q, k_new, v_new, out)
+  L.lse2 = carve(align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4));
+  L.lse_x = carve(align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4));
+  L.place = off;
+  if (c->pos_mode == KF_POS_NEW) L.place = carve(nl * L.sc_layer);
   L.total = off;
   return L;
 }
@@ -125,6 +138,8 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
   if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI)
     e = cudaMemcpyAsync(ctx->ws + lay.slopes, cfg->h_alibi_slopes, (size_t)cfg->n_heads * 4, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI) e = cudaStreamSynchronize(st);  // host array may go away
+  for (size_t g = 0; e == cudaSuccess && g < lay.guards.size(); ++g)   // after the clears above, which span some guards
+    e = cudaMemsetAsync(ctx->ws + lay.guards[g], GUARD_BYTE, GUARD_BYTES, st);
   if (e != cudaSuccess) { delete ctx; return KF_ECUDA; }
   *out = ctx;
   return KF_OK;
@@ -139,6 +154,8 @@ static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt
   const kf_config& c = ctx->cfg;
   if (layer < 0 || layer >= c.n_layers) return KF_EINVAL;
   if (n_prompt < 1 || n_prompt > c.max_prompt_len) return KF_EINVAL;
+  // rows are read 16 bytes at a time (TMA boxes, 128-bit loads in the gather)
+  if (misaligned16(d_q) || misaligned16(d_k) || misaligned16(d_v)) return KF_EINVAL;
   const Layout& L = ctx->lay;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float* acc_full = d_score_opt ? d_score_opt : reinterpret_cast<float*>(ctx->ws + L.acc_full);
@@ -146,8 +163,6 @@ static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt
   const float* slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   const float inv_tau = (float)(1.0 / (double)c.tau_init);  // the prompt phase is iteration t = 0 of Eq. 12
   if (c.prefill_impl == KF_PREFILL_TENSOR) {
-    // TMA reads the prompt tensors: their base addresses must be 16-byte aligned
-    if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k)) & 15u) return KF_EINVAL;
     kf::PrefillTcArgs A{};
     A.Q = static_cast<const __half*>(d_q);
     A.K = static_cast<const __half*>(d_k);
@@ -282,17 +297,8 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.k = c.budget_k; P.w = c.recent_w;
   P.p = ctx->n_prompt[layer] + step - 1;
 
-  // split the slots of a unit over CTAs so that the grid fills the 148 SMs several times over
-  const int tiles = tiles_of(c.budget_k);
-  int splits = c.decode_splits;
-  if (splits <= 0) {
-    const int target_ctas = 148 * 20;   // about ten waves of the two resident CTAs per SM
-    splits = (target_ctas + L.units - 1) / L.units;
-  }
-  splits = std::max(1, std::min(splits, std::min(L.max_splits, (tiles + 3) / 4)));
-  int tps = (tiles + splits - 1) / splits;
-  tps = (tps + 3) / 4 * 4;  // whole rounds of the CTA's four warps
-  splits = (tiles + tps - 1) / tps;
+  int splits = 1, tps = 4;
+  kf::decode_plan(L.units, c.budget_k, c.decode_splits, &splits, &tps);
   P.splits = splits; P.tiles_per_split = tps;
   P.H = c.n_heads; P.layer = layer; P.noise_mode = c.noise_mode; P.bias_mode = c.bias_mode;
   P.scale = ctx->scale;
@@ -305,6 +311,7 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.inv_tau = (float)(1.0 / tau);
   P.noise_const = c.noise_const;
   P.noise_mu = c.noise_mu; P.noise_sigma = c.noise_sigma;
+  P.first_wait_limit = c.debug_fail_first_wait ? 0u : kf::DECODE_WAIT_LIMIT;
   P.pk = ctx->pk;
   if (kf::launch_decode(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
   ctx->launches += 2;   // streaming kernel + closing kernel
@@ -326,6 +333,7 @@ int kf_decode_step(kf_ctx* ctx, int32_t layer, int32_t step,
   const int rc = decode_check(ctx, layer, step);
   if (rc != KF_OK) return rc;
   if (!d_q || !d_knew || !d_vnew || !d_out) return KF_EINVAL;
+  if (misaligned16(d_q) || misaligned16(d_knew) || misaligned16(d_vnew) || misaligned16(d_out)) return KF_EINVAL;
   return decode_impl(ctx, layer, step, d_q, d_knew, d_vnew, d_out, d_score_opt, static_cast<cudaStream_t>(stream));
 }
 
@@ -386,14 +394,19 @@ int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t
   if (a->head_dim != 64 && a->head_dim != 128 && a->head_dim != 256) return KF_EINVAL;
   if (a->budget_k < 1 || a->recent_w < 0 || a->recent_w > a->budget_k) return KF_EINVAL;
   if (a->layer < 0 || a->position < 0 || !(a->tau > 0.0) || a->logit_scale < 0.f) return KF_EINVAL;
-  if (a->noise_mode < KF_NOISE_GUMBEL || a->noise_mode > KF_NOISE_CONST) return KF_EINVAL;
+  if (a->reserved != 0) return KF_EINVAL;
+  if (a->noise_mode < KF_NOISE_GUMBEL || a->noise_mode > KF_NOISE_CONST) return KF_EINVAL;   // no Gaussian here (no mu, sigma)
+  // rows of the cache are sources of 16-byte bulk copies; the step's vectors are read 16 bytes at a time
+  if (misaligned16(d_K) || misaligned16(d_V) || misaligned16(d_q) || misaligned16(d_knew) || misaligned16(d_vnew) ||
+      misaligned16(d_out))
+    return KF_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(d_pos) | reinterpret_cast<uintptr_t>(d_acc) | reinterpret_cast<uintptr_t>(d_len)) & 3u)
+    return KF_EINVAL;
   if (a->bias_mode != KF_BIAS_NONE && a->bias_mode != KF_BIAS_ALIBI) return KF_EINVAL;
   if (a->bias_mode == KF_BIAS_ALIBI && !a->d_alibi_slopes) return KF_EINVAL;
   const int units = a->batch * a->n_heads;
-  const int tiles = tiles_of(a->budget_k);
-  int splits = std::max(1, std::min((148 * 20 + units - 1) / units, std::min(64, (tiles + 3) / 4)));
-  int tps = ((tiles + splits - 1) / splits + 3) / 4 * 4;
-  splits = (tiles + tps - 1) / tps;
+  int splits = 1, tps = 4;
+  kf::decode_plan(units, a->budget_k, 0, &splits, &tps);
   const size_t y_bytes = align_up((size_t)units * ((size_t)a->budget_k + 1) * 4);
   const size_t partial_bytes = align_up((size_t)units * splits * (4 + (size_t)a->head_dim) * 4);
   if (y_bytes + partial_bytes + 256 > kf::STATIC_SCRATCH_BYTES) return KF_ENOSPC;  // before any CUDA call
@@ -415,6 +428,7 @@ int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t
   P.scale = a->logit_scale > 0.f ? a->logit_scale : (float)(1.0 / std::sqrt((double)a->head_dim));
   P.inv_tau = (float)(1.0 / a->tau);
   P.noise_const = a->noise_const;
+  P.first_wait_limit = kf::DECODE_WAIT_LIMIT;
   P.pk = kf::philox_expand_key(a->noise_seed);
   const cudaError_t e = kf::launch_decode_static(P, a->head_dim, units, y_bytes, partial_bytes,
                                                  static_cast<cudaStream_t>(stream));
@@ -529,6 +543,33 @@ int kf_poll_error(kf_ctx* ctx, void* stream) {
     if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
   }
   return word;
+}
+
+int kf_check_canaries(kf_ctx* ctx, void* stream, int32_t* first_bad) {
+  if (first_bad) *first_bad = -1;
+  if (!ctx || !ctx->cfg.debug_canaries) return KF_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const std::vector<size_t>& guards = ctx->lay.guards;
+  std::vector<unsigned char> host(guards.size() * GUARD_BYTES);
+  for (size_t g = 0; g < guards.size(); ++g)
+    if (cudaMemcpyAsync(host.data() + g * GUARD_BYTES, ctx->ws + guards[g], GUARD_BYTES, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+      return KF_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ECUDA;
+  for (size_t i = 0; i < host.size(); ++i)
+    if (host[i] != (unsigned char)GUARD_BYTE) {
+      if (first_bad) *first_bad = (int32_t)(i / GUARD_BYTES);
+      return KF_EBOUNDS;
+    }
+  return KF_OK;
+}
+
+int kf_describe_decode(const kf_ctx* ctx, char* buf, size_t n) {
+  if (!ctx || !buf || n == 0) return KF_EINVAL;
+  int splits = 1, tps = 4;
+  kf::decode_plan(ctx->lay.units, ctx->cfg.budget_k, ctx->cfg.decode_splits, &splits, &tps);
+  const int len = kf::decode_describe(buf, n, ctx->cfg.head_dim, ctx->lay.units, ctx->cfg.budget_k, splits, tps,
+                                      ctx->cfg.pos_mode == KF_POS_NEW);
+  return len < 0 ? KF_EINVAL : len;
 }
 
 int64_t kf_launch_count(const kf_ctx* ctx) { return ctx ? ctx->launches : 0; }

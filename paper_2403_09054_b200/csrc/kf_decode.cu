@@ -15,6 +15,8 @@
 // them into f_theta, picks the entry to evict and writes the new token's row into the freed slot.
 #include "kf_decode.cuh"
 
+#include <algorithm>
+#include <cstdio>
 #include <mutex>
 
 namespace kf {
@@ -285,6 +287,10 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane % LPR, grp = lane / LPR;
   const int len = P.len[u];
+  if (len < 0 || len > P.k) {   // a damaged entry count: touch nothing of this unit, report it
+    if (tid == 0 && s == 0) atomicExch(P.err, ERR_BOUNDS);
+    return;
+  }
   const int row_begin = s * P.tiles_per_split * TILE_ROWS;
   const int row_end = min(len, row_begin + P.tiles_per_split * TILE_ROWS);
   const int n_tiles = row_end > row_begin ? (row_end - row_begin + TILE_ROWS - 1) / TILE_ROWS : 0;
@@ -353,7 +359,8 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
     float x_mine;
     {
       const int it = 2 * ti;
-      const bool ok = mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1));
+      const bool ok = mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1),
+                                        ti == 0 ? P.first_wait_limit : DECODE_WAIT_LIMIT);
       if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       const unsigned char* krow = ring + (size_t)(it % NSTAGE) * TILE_BYTES + (size_t)lane * D * 2;
       const unsigned char* qb = reinterpret_cast<const unsigned char*>(sh_q);
@@ -478,7 +485,9 @@ template <int D>
 __global__ void __launch_bounds__(128, 8) decode_close_kernel(const __grid_constant__ DecodeParams P) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // lets the next kernel's CTAs queue up behind this grid
   const int u = blockIdx.x;
-  combine_and_evict<D, 128>(P, u, P.len[u]);
+  const int len = P.len[u];
+  if (len < 0 || len > P.k) return;   // reported by the streaming kernel; nothing of the unit is written
+  combine_and_evict<D, 128>(P, u, len);
 }
 
 template <int D, int NW, int NSTAGE>
@@ -534,14 +543,44 @@ cudaError_t launch_rebuild_place(const int32_t* pos, const int32_t* len, int32_t
 int decode_tile_rows() { return TILE_ROWS; }
 int decode_max_splits() { return MAX_SPLITS; }
 
+void decode_plan(int units, int budget_k, int requested, int* splits_out, int* tiles_per_split_out) {
+  const int tiles = (budget_k + TILE_ROWS - 1) / TILE_ROWS;
+  int splits = requested;
+  if (splits <= 0) {
+    const int target_ctas = 148 * 20;   // about ten waves of the two resident CTAs per SM
+    splits = (target_ctas + units - 1) / units;
+  }
+  splits = std::max(1, std::min(splits, std::min(MAX_SPLITS, (tiles + 3) / 4)));
+  int tps = (tiles + splits - 1) / splits;
+  tps = (tps + 3) / 4 * 4;  // whole rounds of the CTA's four warps
+  *splits_out = (tiles + tps - 1) / tps;
+  *tiles_per_split_out = tps;
+}
+
+// Template arguments <D, NW, NSTAGE> of the streaming kernel launch_decode picks for a shape (one table for the
+// launcher and for kf_describe_decode).
+static void decode_variant(int head_dim, int tiles_per_split, int* nw, int* nstage) {
+  *nw = (head_dim == 128 && tiles_per_split >= 16) ? 5 : 4;
+  *nstage = head_dim == 64 ? 4 : 2;
+}
+
+int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos) {
+  int nw = 4, nstage = 2;
+  decode_variant(head_dim, tiles_per_split, &nw, &nstage);
+  return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d> + decode_close_kernel<%d>; units=%d k=%d splits=%d tiles_per_split=%d group=1",
+                  head_dim, nw, nstage, new_pos ? 1 : 0, head_dim, units, budget_k, splits, tiles_per_split);
+}
+
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
   if (P.splits < 1 || P.splits > MAX_SPLITS) return cudaErrorInvalidValue;
+  int nw = 4, nstage = 2;
+  decode_variant(head_dim, P.tiles_per_split, &nw, &nstage);
   switch (head_dim) {
     case 64: return launch_one<64, 4, 4>(P, units, stream);
     case 128:
       // long items (bandwidth-bound workloads): five warps and 80 KB of ring per CTA, two CTAs per SM, measured best;
       // short items (few units, latency-bound): four warps, three CTAs per SM
-      return P.tiles_per_split >= 16 ? launch_one<128, 5, 2>(P, units, stream) : launch_one<128, 4, 2>(P, units, stream);
+      return nw == 5 ? launch_one<128, 5, 2>(P, units, stream) : launch_one<128, 4, 2>(P, units, stream);
     case 256: return launch_one<256, 4, 2>(P, units, stream);
     default: return cudaErrorInvalidValue;
   }

@@ -26,15 +26,24 @@ struct DecodeParams {
   int32_t splits, tiles_per_split;
   int32_t H, layer, noise_mode, bias_mode;
   float scale, inv_tau, noise_const, noise_mu, noise_sigma;
+  uint32_t first_wait_limit;   // polls the streaming kernel grants its first tile (DECODE_WAIT_LIMIT; 0 in the self-test
+                               // that makes a wait run out: the warp gives up at once, then drains with the full limit)
   PhiloxKeys pk;
 };
+
+constexpr uint32_t DECODE_WAIT_LIMIT = 1u << 22;   // polls of a bounded wait in the generation kernels
 
 // Size of the built-in scratch block used by kf_decode_step_static (16 MiB per GPU).
 constexpr size_t STATIC_SCRATCH_BYTES = (size_t)16 << 20;
 
 int decode_tile_rows();
 int decode_max_splits();
+// How a layer call is cut into CTAs: `splits` CTAs per unit, each streaming `tiles_per_split` 32-row tiles.
+// `requested` = 0 lets the grid fill the 148 SMs several times over.  The scratch layout follows from it.
+void decode_plan(int units, int budget_k, int requested, int* splits, int* tiles_per_split);
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
+// Names the kernels (with their template arguments) and the split plan of a layer call of this shape; snprintf semantics.
+int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos);
 
 // Reorders every unit's entries of one layer into ascending position, in place (see kf_compact.cu).  `place` may be
 // null; `dst_scratch` is [units][k] int32 of scratch.  Budgets above compact_max_k() are refused (cudaErrorInvalidValue).

@@ -35,6 +35,9 @@ def oracle_params(wl: W.Workload, noise_mode=ko.NOISE_GUMBEL, logit_scale=0.0, p
 
 
 def make_gpu(wl: W.Workload, noise_mode=kf.KF_NOISE_GUMBEL, max_prompt_len=None, **kw) -> kf.Keyformer:
+    """A context for `wl`.  Unless told otherwise the workspace carries guard blocks between its sub-buffers
+    (see check_guards): the kernels and their launch shapes are the same with and without them."""
+    kw.setdefault("debug_canaries", 1)
     return kf.Keyformer(n_layers=wl.n_layers, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
                         budget_k=wl.budget_k, recent_w=wl.recent_w,
                         max_prompt_len=max_prompt_len or wl.prompt_len, gen_len_T=wl.gen_len_T,
@@ -42,6 +45,13 @@ def make_gpu(wl: W.Workload, noise_mode=kf.KF_NOISE_GUMBEL, max_prompt_len=None,
                         noise_mode=noise_mode,
                         bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
                         alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None, **kw)
+
+
+def check_guards(gpu: kf.Keyformer):
+    """No kernel wrote past the end of a workspace sub-buffer (and no bounded wait ran out)."""
+    assert gpu.kf_poll_error() == 0
+    rc, bad = gpu.kf_check_canaries()
+    assert rc == kf.KF_OK, f"guard behind workspace sub-buffer {bad} was overwritten ({kf.kf_strerror(rc)})"
 
 
 def check_band(acc_ref, cand_mask, kept_mask, n_keep, what):
@@ -196,25 +206,25 @@ class LockStep:
             L = int(len_before[u])
             m = L + 1
             assert int(self.st.len[u]) == m
-            ref_pos = self.st.pos[u, :m]
+            ref_pos = self.st.pos[u, :m]                       # the oracle keeps its entries in position order
             gpu_pos = np.concatenate([pos_before[u, :L], [p]])
-            assert sorted(ref_pos.tolist()) == sorted(gpu_pos.tolist()), f"{tag}: cached positions differ"
-            order = {int(pp): j for j, pp in enumerate(ref_pos)}
-            perm = np.array([order[int(pp)] for pp in gpu_pos])
+            assert (np.diff(ref_pos) > 0).all()
+            assert np.array_equal(ref_pos, np.sort(gpu_pos)), f"{tag}: cached positions differ"
+            perm = np.searchsorted(ref_pos, gpu_pos)
             zr, zg = z_ref[u, perm], z_gpu[u, :m]
             serr = np.abs(zg - zr) - (SCORE_RTOL * np.abs(zr) + SCORE_ATOL)
             self.max_score_err = max(self.max_score_err, float((np.abs(zg - zr) / np.maximum(zr, 1e-6)).max()))
             assert serr.max() <= 0, f"{tag}: score off by {serr.max():.3e} beyond tolerance"
             La = int(len_after[u])
             assert La == min(m, kk), f"{tag}: cache length {La}"
-            after = set(pos_after[u, :La].tolist())
-            assert len(after) == La and after <= set(gpu_pos.tolist()), f"{tag}: duplicate or foreign positions"
-            gone = set(gpu_pos.tolist()) - after
+            after = np.sort(pos_after[u, :La])
+            assert (np.diff(after) > 0).all() and np.isin(after, ref_pos).all(), f"{tag}: duplicate or foreign positions"
+            gone = np.setdiff1d(ref_pos, after)
             if m <= kk:
-                assert not gone
+                assert gone.size == 0
             else:
-                assert len(gone) == 1, f"{tag}: {len(gone)} entries left the cache"
-                ev = gone.pop()
+                assert gone.size == 1, f"{tag}: {gone.size} entries left the cache"
+                ev = int(gone[0])
                 acc_r = self.st.acc[u, :m]
                 cand_mask = ref_pos <= p - w
                 check_band(acc_r, cand_mask, ref_pos != ev, kk - int((~cand_mask).sum()), tag)
@@ -232,9 +242,9 @@ class LockStep:
         if check_state:
             for u in range(U):
                 La = int(len_after[u])
-                ref = {int(pp): j for j, pp in enumerate(self.st.pos[u, :La])}
-                assert set(ref) == set(pos_after[u, :La].tolist())
-                idx = np.array([ref[int(pp)] for pp in pos_after[u, :La]])
+                ref_pos = self.st.pos[u, :La]
+                assert np.array_equal(ref_pos, np.sort(pos_after[u, :La]))
+                idx = np.searchsorted(ref_pos, pos_after[u, :La])
                 a_ref = self.st.acc[u, idx]
                 aerr = np.abs(acc_after[u, :La] - a_ref) - (SCORE_RTOL * np.abs(a_ref) + 1e-6)
                 assert aerr.max() <= 0, f"step {step}: accumulated score off by {aerr.max():.3e}"
@@ -268,5 +278,6 @@ def run_workload(wl: W.Workload, units_per_layer=None, steps=None, layers=None, 
                max_out_err=max(d.max_out_err for d in drivers),
                max_score_err=max(d.max_score_err for d in drivers),
                units=sum(len(d.units) for d in drivers), steps=steps)
+    check_guards(gpu)
     gpu.kf_destroy()
     return res

@@ -70,3 +70,41 @@ def test_no_cpu_fallback():
     cfg = _cfg()
     h = C.c_void_p()
     assert kf.LIB.kf_create(C.byref(cfg), 256, 1 << 40, None, C.byref(h)) == kf.KF_ECUDA
+
+
+def test_static_step_validates_before_touching_the_device():
+    """kf_decode_step_static checks its arguments before its first CUDA call: reserved field, noise mode,
+    alignment (all refused with KF_EINVAL and nothing launched; this runs without a device)."""
+    a = kf.kf_static_step()
+    a.batch, a.n_heads, a.head_dim, a.budget_k, a.recent_w = 1, 2, 64, 32, 8
+    a.tau = 1.0
+    ok = 4096                                            # a 16-byte aligned (never dereferenced) address
+    call = lambda *p: kf.LIB.kf_decode_step_static(C.byref(a), *p, None, None)
+    a.reserved = 1
+    assert call(ok, ok, ok, ok, ok, ok, ok, ok, ok) == kf.KF_EINVAL
+    a.reserved = 0
+    a.noise_mode = kf.KF_NOISE_GAUSS
+    assert call(ok, ok, ok, ok, ok, ok, ok, ok, ok) == kf.KF_EINVAL
+    a.noise_mode = kf.KF_NOISE_GUMBEL
+    for i in (0, 1, 5, 6, 7, 8):                         # K, V, q, k_new, v_new, out: 16-byte alignment
+        p = [ok] * 9
+        p[i] = ok + 2
+        assert call(*p) == kf.KF_EINVAL
+    for i in (2, 3, 4):                                  # positions, scores, entry counts: 4-byte alignment
+        p = [ok] * 9
+        p[i] = ok + 2
+        assert call(*p) == kf.KF_EINVAL
+    a.budget_k = 1 << 22                                 # scratch beyond the built-in block
+    assert call(ok, ok, ok, ok, ok, ok, ok, ok, ok) == kf.KF_ENOSPC
+
+
+def test_error_codes_have_messages():
+    for code in (kf.KF_EINVAL, kf.KF_ENOSPC, kf.KF_ESTATE, kf.KF_ECUDA, kf.KF_ETIMEOUT, kf.KF_EBOUNDS):
+        assert kf.kf_strerror(code) not in ("ok", "unknown error")
+    assert kf.kf_strerror(-99) == "unknown error"
+
+
+def test_guard_blocks_enlarge_the_workspace():
+    base, dbg = kf.kf_workspace_bytes(_cfg()), kf.kf_workspace_bytes(_cfg(debug_canaries=1))
+    assert dbg - base == 14 * 256                        # one guard behind each of the 14 sub-buffers (no places)
+    assert kf.kf_workspace_bytes(_cfg(debug_canaries=2)) == 0 and kf.kf_workspace_bytes(_cfg(debug_fail_first_wait=3)) == 0

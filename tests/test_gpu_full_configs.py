@@ -13,29 +13,37 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def test_config2_gptj_all_units():
+def _report(tag, r):
+    """One line per workload for the test log: units and steps compared, eviction choices adopted from the GPU
+    (decisions inside the tolerance band), largest relative errors seen."""
+    print(f"\nLOCKSTEP {tag}: units={r['units']} steps={r['steps']} adoptions={r['adoptions']} "
+          f"max_out_err={r['max_out_err']:.3e} max_score_err={r['max_score_err']:.3e}")
+
+
+def test_config2_gptj_all_units_all_steps():
     wl = W.get_config("c2_gptj")
-    r = lockstep.run_workload(wl, steps=24, check_state_every=8)
-    print("c2", r)
+    r = lockstep.run_workload(wl, check_state_every=32)
+    assert r["units"] == 16 and r["steps"] == 256
+    _report("c2_gptj", r)
 
 
-def test_config3_mpt_sampled_units():
+@pytest.mark.parametrize("pos_mode", [0, 1])
+def test_config3_mpt_sampled_units_all_steps(pos_mode):
+    """The ALiBi workload at full size for all 512 steps, with original positions in the bias and with the bias
+    counted in places of the reduced cache (section 4.4.2)."""
     wl = W.get_config("c3_mpt")
-    r = lockstep.run_workload(wl, units_per_layer=6, steps=12, check_state_every=6)
-    print("c3", r)
+    r = lockstep.run_workload(wl, units_per_layer=8, check_state_every=64, pos_mode=pos_mode)
+    assert r["units"] == 8 and r["steps"] == 512
+    _report("c3_mpt" + (" new positions" if pos_mode else ""), r)
 
 
-def test_config3_mpt_new_positions_sampled_units():
-    """The ALiBi workload at full size with the bias counted in places of the reduced cache (section 4.4.2)."""
-    wl = W.get_config("c3_mpt")
-    r = lockstep.run_workload(wl, units_per_layer=4, steps=8, check_state_every=4, pos_mode=1)
-    print("c3 new positions", r)
-
-
-def test_config4_cerebras_first_and_last_layer_sampled_units():
+def test_config4_cerebras_three_layers_sampled_units_all_steps():
+    """66 units sampled from the first, the middle and the last layer, all 256 steps.  The context is the full
+    32-layer one (the launch configuration the benchmark times); only the three layers are given a prompt."""
     wl = W.get_config("c4_cerebras")
-    r = lockstep.run_workload(wl, units_per_layer=8, steps=6, layers=[0, wl.n_layers - 1], check_state_every=3)
-    print("c4", r)
+    r = lockstep.run_workload(wl, units_per_layer=22, layers=[0, wl.n_layers // 2 - 1, wl.n_layers - 1], check_state_every=64)
+    assert r["units"] == 66 and r["steps"] == 256
+    _report("c4_cerebras", r)
 
 
 @pytest.mark.parametrize("name", ["c5_prefill_1k", "c5_prefill_2k", "c5_prefill_4k", "c5_prefill_8k"])
@@ -43,8 +51,9 @@ def test_config5_prefill_sweep(name):
     base = W.get_config(name)
     n = base.prompt_len
     q, k, v = W.make_prompt(base, 0, DEV)
-    units = W.sample_units(base, 4 if n >= 4096 else 8, seed=n, layer=0)
+    units = W.sample_units(base, 16, seed=n, layer=0)
     acc_ref = None
+    adoptions = []
     for frac in C5_BUDGET_FRACTIONS:
         kk, w = c5_budget(n, frac)
         wl = base.scaled(budget_k=kk, recent_w=w)
@@ -61,4 +70,8 @@ def test_config5_prefill_sweep(name):
         assert (ln == kk).all()
         assert (pos[..., -w:] == torch.arange(n - w, n, device=DEV, dtype=torch.int32)).all()
         assert (pos[..., 1:] > pos[..., :-1]).all()
+        adoptions.append(ls.adoptions)
+        lockstep.check_guards(gpu)
         gpu.kf_destroy()
+    print(f"\nLOCKSTEP {name}: units={len(units)} budgets={list(C5_BUDGET_FRACTIONS)} adoptions={adoptions} "
+          f"max_score_err={ls.max_score_err:.3e}")

@@ -49,6 +49,7 @@ def test_prompts_shorter_than_the_maximum_and_a_context_used_again(impl):
     with pytest.raises(kf.KeyformerError) as e:
         gpu.kf_prefill_score_prune(0, *W.make_prompt(_wl(head_dim=128, prompt_len=701), 0, DEV))
     assert e.value.code == kf.KF_EINVAL
+    lockstep.check_guards(gpu)
     gpu.kf_destroy()
 
 
@@ -72,6 +73,7 @@ def test_prompt_scores_tensor_core_vs_cuda_core():
         gpu.kf_prefill_score_prune(0, q, k, v, score_out=s)
         assert gpu.kf_poll_error() == 0
         scores.append(s)
+        lockstep.check_guards(gpu)
         gpu.kf_destroy()
     assert torch.equal(scores[0], scores[1])
     assert torch.allclose(scores[0], scores[2], rtol=2e-4, atol=1e-6)
@@ -187,7 +189,8 @@ def test_new_positions_differ_from_original_positions_and_survive_import():
     assert torch.equal(again.kf_view_place(0), new.kf_view_place(0))
     pos = new.kf_view_state(0)[2]
     assert torch.equal(new.kf_view_place(0).long(), pos.argsort(-1).argsort(-1))
-    assert org.kf_poll_error() == 0 and new.kf_poll_error() == 0 and again.kf_poll_error() == 0
+    for g in (org, new, again):
+        lockstep.check_guards(g)
 
 
 @pytest.mark.parametrize("d,pos_mode", [(64, 0), (128, 1), (256, 0)])
@@ -219,6 +222,16 @@ def test_compaction_restores_position_order_in_place(d, pos_mode):
     assert torch.equal(ln, before[0][4])
     if pos_mode == 1:
         assert torch.equal(gpu.kf_view_place(0).long(), torch.arange(77, device=DEV).expand(2, 3, 77))
+    # the oracle keeps its entries in position order, so after the compaction the GPU's slots line up with it one to one
+    st = drivers[0].st
+    for u in range(st.U):
+        b, h = int(st.lbh[u, 1]), int(st.lbh[u, 2])
+        L = int(st.len[u])
+        assert int(ln[b, h]) == L and np.array_equal(pos[b, h, :L].cpu().numpy(), st.pos[u, :L])
+        a_ref = st.acc[u, :L]
+        assert (np.abs(acc[b, h, :L].cpu().numpy() - a_ref) <= lockstep.SCORE_RTOL * np.abs(a_ref) + 1e-6).all()
+        assert np.array_equal(K[b, h, :L].cpu().numpy().view(np.uint16), st.K[u, :L])
+        assert np.array_equal(V[b, h, :L].cpu().numpy().view(np.uint16), st.V[u, :L])
     for x, y in zip(gpu.kf_view_state(1), before[1]):
         assert torch.equal(x, y)
     gpu.kf_compact_layer(0)                                                   # already in order: nothing moves
@@ -226,6 +239,7 @@ def test_compaction_restores_position_order_in_place(d, pos_mode):
     for s in range(26, 41):
         for ls in drivers:
             ls.decode_step(s, *W.make_step(wl, ls.layer, s, DEV))
+    lockstep.check_guards(gpu)
     gpu.kf_destroy()
 
 
@@ -299,7 +313,8 @@ def test_export_import_state_resumes_bit_exactly():
     for l in range(2):
         for x, y in zip(a.kf_view_state(l), b.kf_view_state(l)):
             assert torch.equal(x, y)
-    assert a.kf_poll_error() == 0 and b.kf_poll_error() == 0
+    lockstep.check_guards(a)
+    lockstep.check_guards(b)
 
 
 def test_host_buffer_variant_matches_device_variant():
@@ -338,3 +353,87 @@ def test_host_buffer_variant_matches_device_variant():
             assert torch.allclose(x, y, rtol=1e-5, atol=1e-6)
         else:
             assert torch.equal(x, y)
+
+
+# ------------------------------------------------------------------ error paths (nothing here faults or hangs the GPU)
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
+    """debug_fail_first_wait makes every warp of the streaming kernel treat its first wait for a cache tile as
+    run out: the warp flags KF_ETIMEOUT, waits (with the full limit) for its copies in flight and leaves.  The
+    error word is returned once and cleared; a fresh context on the same device then runs in lock step."""
+    wl = _wl(head_dim=128, prompt_len=300, budget_k=200, recent_w=20, gen_len_T=4)
+    gpu = lockstep.make_gpu(wl, debug_fail_first_wait=1)
+    gpu.kf_prefill_score_prune(0, *W.make_prompt(wl, 0, DEV))
+    assert gpu.kf_poll_error() == 0                                     # the prompt phase has no such switch
+    q, kn, vn = W.make_step(wl, 0, 1, DEV)
+    out = torch.empty_like(q)
+    gpu.kf_decode_step(0, 1, q, kn, vn, out)
+    assert gpu.kf_poll_error() == kf.KF_ETIMEOUT
+    assert kf.kf_strerror(kf.KF_ETIMEOUT) == "a bounded device-side wait ran out"
+    assert gpu.kf_poll_error() == 0                                     # read once, then cleared
+    rc, bad = gpu.kf_check_canaries()
+    assert rc == kf.KF_OK, bad                                          # the aborted step stayed inside its buffers
+    gpu.kf_destroy()
+    r = lockstep.run_workload(wl)                                       # the device and the library are fine
+    assert r["steps"] == 4
+
+
+@pytest.mark.parametrize("bad_len", [-1, 41, 1 << 20])
+def test_a_damaged_entry_count_is_reported_and_the_unit_left_alone(bad_len):
+    wl = _wl(prompt_len=100, budget_k=40, recent_w=10)
+    gpu = lockstep.make_gpu(wl)
+    gpu.kf_prefill_score_prune(0, *W.make_prompt(wl, 0, DEV))
+    K, V, pos, acc, ln = gpu.kf_view_state(0)
+    torch.cuda.synchronize()
+    ln[1, 2] = bad_len                                                  # what a foreign state image could contain
+    before = [t.clone() for t in (K, V, pos, acc, ln)]
+    q, kn, vn = W.make_step(wl, 0, 1, DEV)
+    out = torch.zeros_like(q)
+    gpu.kf_decode_step(0, 1, q, kn, vn, out)
+    assert gpu.kf_poll_error() == kf.KF_EBOUNDS
+    assert kf.kf_strerror(kf.KF_EBOUNDS) == "a device-side bounds check failed"
+    after = gpu.kf_view_state(0)
+    for x, y in zip(before, after):
+        assert torch.equal(x[1, 2], y[1, 2])                            # nothing of the damaged unit was written
+    assert (out[1, 2] == 0).all()
+    assert (after[4].flatten()[:5] == 40).all() and not torch.equal(before[2][0, 0], after[2][0, 0])   # the others stepped
+    lockstep.check_guards(gpu)
+    gpu.kf_destroy()
+
+
+def test_guard_blocks_detect_a_write_past_a_sub_buffer():
+    wl = _wl()
+    gpu = lockstep.make_gpu(wl)
+    assert gpu.kf_check_canaries() == (kf.KF_OK, -1)
+    K = gpu.kf_view_state(0)[0]
+    off = K.data_ptr() - gpu.workspace.data_ptr() + K.numel() * 2      # first byte behind the K cache (a guard)
+    gpu.workspace[off + 7] = 0                                          # a write one row too far would land here
+    assert gpu.kf_check_canaries() == (kf.KF_EBOUNDS, 0)
+    plain = lockstep.make_gpu(wl, debug_canaries=0)
+    assert plain.kf_check_canaries()[0] == kf.KF_EINVAL
+    assert gpu.workspace_bytes > plain.workspace_bytes
+
+
+def test_misaligned_pointers_are_rejected_on_the_host():
+    wl = _wl(head_dim=64)
+    gpu = lockstep.make_gpu(wl)
+    n, d = wl.prompt_len, wl.head_dim
+    numel = wl.batch * wl.n_heads * n * d
+    big = torch.zeros(numel + 8, dtype=torch.float16, device=DEV)
+    Q, K, V = W.make_prompt(wl, 0, DEV)
+    odd = big[1:1 + numel].view(Q.shape)                                # contiguous, but 2 bytes off a 16-byte boundary
+    launches = gpu.kf_launch_count()
+    for args in ((odd, K, V), (Q, odd, V), (Q, K, odd)):
+        with pytest.raises(kf.KeyformerError) as e:
+            gpu.kf_prefill_score_prune(0, *args)
+        assert e.value.code == kf.KF_EINVAL
+    gpu.kf_prefill_score_prune(0, Q, K, V)
+    q, kn, vn = W.make_step(wl, 0, 1, DEV)
+    out = torch.empty_like(q)
+    small = big[1:1 + q.numel()].view(q.shape)
+    for args in ((small, kn, vn, out), (q, small, vn, out), (q, kn, small, out), (q, kn, vn, small)):
+        with pytest.raises(kf.KeyformerError) as e:
+            gpu.kf_decode_step(0, 1, *args)
+        assert e.value.code == kf.KF_EINVAL
+    assert gpu.kf_launch_count() == launches + 4                        # only the accepted prompt call launched
+    gpu.kf_decode_step(0, 1, q, kn, vn, out)
+    lockstep.check_guards(gpu)

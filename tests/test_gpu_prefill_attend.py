@@ -28,6 +28,7 @@ def _check(wl, units=None):
     scale = np.abs(ref).max(axis=-1, keepdims=True)
     err = np.abs(got - ref) / scale
     assert err.max() <= lockstep.OUT_RTOL, f"attention output off by {err.max():.3e} of the row's largest value"
+    lockstep.check_guards(gpu)
     gpu.kf_destroy()
     return float(err.max())
 
