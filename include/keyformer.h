@@ -88,6 +88,13 @@ typedef struct kf_config {
   float   noise_mu;        /* mean of KF_NOISE_GAUSS (the paper matches Gumbel's 0.5772)          */
   float   noise_sigma;     /* standard deviation of KF_NOISE_GAUSS (1.2825 in the paper)         */
   int32_t pos_mode;        /* KF_POS_*; KF_POS_NEW keeps one more int32 per cache slot            */
+  int32_t n_kv_heads;      /* key/value heads Hkv (section 6: multi-query / grouped-query attention).  0 or H: every head
+                              has its own cache, the method as printed.  Otherwise H / Hkv must be 2, 4 or 8: that many
+                              consecutive query heads share one cache and one f_theta; each of them has its own logits,
+                              noise (drawn with its own head index), bias slope and softmax of Eq. 11, and f_theta
+                              accumulates the mean of their scores.  Caches are then per (layer, batch row, key/value
+                              head): wherever a shape below says [B][H] for K, V, k_new, v_new, scores, positions or entry
+                              counts read [B][Hkv]; q and out stay [B][H].                                         */
   int32_t debug_canaries;  /* 1: a 256-byte guard of a known pattern follows every sub-buffer of the workspace
                               (kf_workspace_bytes grows accordingly); kf_check_canaries verifies them.  0: none */
   int32_t debug_fail_first_wait; /* self-test of the error path: 1 makes every warp of the generation kernel give up

@@ -35,7 +35,7 @@ class kf_config(C.Structure):
         ("logit_scale", C.c_float), ("noise_const", C.c_float),
         ("decode_splits", C.c_int32), ("prefill_impl", C.c_int32),
         ("noise_mu", C.c_float), ("noise_sigma", C.c_float), ("pos_mode", C.c_int32),
-        ("debug_canaries", C.c_int32), ("debug_fail_first_wait", C.c_int32),
+        ("n_kv_heads", C.c_int32), ("debug_canaries", C.c_int32), ("debug_fail_first_wait", C.c_int32),
     ]
 
 
@@ -125,7 +125,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
                 tau_init=1.0, tau_end=2.0, noise_seed=0, noise_mode=KF_NOISE_GUMBEL, bias_mode=KF_BIAS_NONE,
                 alibi_slopes=None, logit_scale=0.0, noise_const=0.5772, decode_splits=0,
                 prefill_impl=KF_PREFILL_TENSOR, noise_mu=0.5772, noise_sigma=1.2825, pos_mode=KF_POS_ORIGINAL,
-                debug_canaries=0, debug_fail_first_wait=0):
+                n_kv_heads=0, debug_canaries=0, debug_fail_first_wait=0):
     """Fill a kf_config; returns (config, keepalive) where keepalive holds the slopes array."""
     cfg = kf_config()
     cfg.n_layers, cfg.batch, cfg.n_heads, cfg.head_dim = n_layers, batch, n_heads, head_dim
@@ -141,6 +141,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
     cfg.decode_splits, cfg.prefill_impl = decode_splits, prefill_impl
     cfg.noise_mu, cfg.noise_sigma = noise_mu, noise_sigma
     cfg.pos_mode = pos_mode
+    cfg.n_kv_heads = n_kv_heads
     cfg.debug_canaries, cfg.debug_fail_first_wait = debug_canaries, debug_fail_first_wait
     return cfg, keep
 
@@ -205,51 +206,52 @@ class Keyformer:
             h = C.c_void_p()
             _check(LIB.kf_create(C.byref(self.cfg), self._ws_ptr, nbytes, _stream_ptr(stream), C.byref(h)), "kf_create")
         self._h = h
-        self.units = self.cfg.batch * self.cfg.n_heads
+        self.kv_heads = self.cfg.n_kv_heads if self.cfg.n_kv_heads > 0 else self.cfg.n_heads
+        self.units_q = self.cfg.batch * self.cfg.n_heads       # (batch row, query head) pairs
+        self.units = self.cfg.batch * self.kv_heads            # caches per layer: (batch row, key/value head) pairs
 
     # ---- the C calls, same names ---------------------------------------------------------
     def kf_prefill_score_prune(self, layer, q, k, v, score_out=None, stream=None):
-        B, H, d = self.cfg.batch, self.cfg.n_heads, self.cfg.head_dim
+        d = self.cfg.head_dim
         n = q.shape[-2]
-        numel = B * H * n * d
         _check(LIB.kf_prefill_score_prune(
             self._h, layer, n,
-            _dev_ptr(q, torch.float16, numel, "q"), _dev_ptr(k, torch.float16, numel, "k"),
-            _dev_ptr(v, torch.float16, numel, "v"),
-            _dev_ptr(score_out, torch.float32, B * H * n, "score_out"), _stream_ptr(stream)),
+            _dev_ptr(q, torch.float16, self.units_q * n * d, "q"), _dev_ptr(k, torch.float16, self.units * n * d, "k"),
+            _dev_ptr(v, torch.float16, self.units * n * d, "v"),
+            _dev_ptr(score_out, torch.float32, self.units * n, "score_out"), _stream_ptr(stream)),
             "kf_prefill_score_prune")
 
     def kf_prefill_attend(self, q, k, v, out, stream=None):
-        B, H, d = self.cfg.batch, self.cfg.n_heads, self.cfg.head_dim
+        d = self.cfg.head_dim
         n = q.shape[-2]
-        numel = B * H * n * d
         _check(LIB.kf_prefill_attend(
-            self._h, n, _dev_ptr(q, torch.float16, numel, "q"), _dev_ptr(k, torch.float16, numel, "k"),
-            _dev_ptr(v, torch.float16, numel, "v"), _dev_ptr(out, torch.float16, numel, "out"), _stream_ptr(stream)),
-            "kf_prefill_attend")
+            self._h, n, _dev_ptr(q, torch.float16, self.units_q * n * d, "q"), _dev_ptr(k, torch.float16, self.units * n * d, "k"),
+            _dev_ptr(v, torch.float16, self.units * n * d, "v"), _dev_ptr(out, torch.float16, self.units_q * n * d, "out"),
+            _stream_ptr(stream)), "kf_prefill_attend")
 
     def kf_prefill_attend_score_prune(self, layer, q, k, v, out, score_out=None, stream=None):
-        B, H, d = self.cfg.batch, self.cfg.n_heads, self.cfg.head_dim
+        d = self.cfg.head_dim
         n = q.shape[-2]
-        numel = B * H * n * d
         _check(LIB.kf_prefill_attend_score_prune(
-            self._h, layer, n, _dev_ptr(q, torch.float16, numel, "q"), _dev_ptr(k, torch.float16, numel, "k"),
-            _dev_ptr(v, torch.float16, numel, "v"), _dev_ptr(out, torch.float16, numel, "out"),
-            _dev_ptr(score_out, torch.float32, B * H * n, "score_out"), _stream_ptr(stream)),
+            self._h, layer, n, _dev_ptr(q, torch.float16, self.units_q * n * d, "q"),
+            _dev_ptr(k, torch.float16, self.units * n * d, "k"), _dev_ptr(v, torch.float16, self.units * n * d, "v"),
+            _dev_ptr(out, torch.float16, self.units_q * n * d, "out"),
+            _dev_ptr(score_out, torch.float32, self.units * n, "score_out"), _stream_ptr(stream)),
             "kf_prefill_attend_score_prune")
 
     def kf_decode_step(self, layer, step, q, knew, vnew, out, score_out=None, stream=None):
-        numel = self.units * self.cfg.head_dim
+        d = self.cfg.head_dim
         _check(LIB.kf_decode_step(
             self._h, layer, step,
-            _dev_ptr(q, torch.float16, numel, "q"), _dev_ptr(knew, torch.float16, numel, "knew"),
-            _dev_ptr(vnew, torch.float16, numel, "vnew"), _dev_ptr(out, torch.float16, numel, "out"),
+            _dev_ptr(q, torch.float16, self.units_q * d, "q"), _dev_ptr(knew, torch.float16, self.units * d, "knew"),
+            _dev_ptr(vnew, torch.float16, self.units * d, "vnew"), _dev_ptr(out, torch.float16, self.units_q * d, "out"),
             _dev_ptr(score_out, torch.float32, self.units * (self.cfg.budget_k + 1), "score_out"),
             _stream_ptr(stream)), "kf_decode_step")
 
     def kf_decode_step_host(self, layer, step, q, knew, vnew, out, wait=True, stream=None):
-        numel = self.units * self.cfg.head_dim
-        for name, t in (("q", q), ("knew", knew), ("vnew", vnew), ("out", out)):
+        d = self.cfg.head_dim
+        for name, t, numel in (("q", q, self.units_q * d), ("knew", knew, self.units * d), ("vnew", vnew, self.units * d),
+                               ("out", out, self.units_q * d)):
             if t.is_cuda or not t.is_contiguous() or t.dtype != torch.float16 or t.numel() != numel:
                 raise ValueError(f"{name}: expected a contiguous host float16 tensor with {numel} elements")
         _check(LIB.kf_decode_step_host(self._h, layer, step, q.data_ptr(), knew.data_ptr(), vnew.data_ptr(),
@@ -259,7 +261,7 @@ class Keyformer:
         """Zero-copy torch views (K, V, pos, acc, len) of one layer's cache inside the workspace."""
         ptrs = [C.c_void_p() for _ in range(5)]
         _check(LIB.kf_view_state(self._h, layer, *[C.byref(p) for p in ptrs]), "kf_view_state")
-        B, H, k, d = self.cfg.batch, self.cfg.n_heads, self.cfg.budget_k, self.cfg.head_dim
+        B, H, k, d = self.cfg.batch, self.kv_heads, self.cfg.budget_k, self.cfg.head_dim   # one cache per key/value head
         base = self.workspace.data_ptr()
 
         def view(ptr, nbytes, dtype, shape):
@@ -280,7 +282,7 @@ class Keyformer:
         """Zero-copy torch view of one layer's places (KF_POS_NEW only), int32 [B, H, k]."""
         ptr = C.c_void_p()
         _check(LIB.kf_view_place(self._h, layer, C.byref(ptr)), "kf_view_place")
-        B, H, k = self.cfg.batch, self.cfg.n_heads, self.cfg.budget_k
+        B, H, k = self.cfg.batch, self.kv_heads, self.cfg.budget_k
         off = ptr.value - self.workspace.data_ptr()
         return self.workspace[off:off + B * H * k * 4].view(torch.int32).view(B, H, k)
 

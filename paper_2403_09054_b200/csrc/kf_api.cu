@@ -27,9 +27,11 @@ struct Layout {
   size_t acc_full, idx, staging, lse2, lse_x;
   size_t total;
   size_t kv_layer, sc_layer, len_layer; // bytes per layer
-  int units, max_splits;
+  int units, max_splits;               // units = caches of a layer = batch x key/value heads
+  int units_q, group;                  // batch x query heads; query heads per key/value head
+  size_t acc_q;                        // group > 1 only: prompt scores per query head, before the group mean
   // debug_canaries: a guard of GUARD_BYTES follows every sub-buffer; `guards` holds their offsets in layout order
-  // (K, V, acc, pos, len, y_scratch, partials, err, slopes, acc_full, idx, staging, lse2, lse_x, place)
+  // (K, V, acc, pos, len, y_scratch, partials, err, slopes, acc_full, idx, staging, lse2, lse_x, [place], [acc_q])
   std::vector<size_t> guards;
 };
 
@@ -48,15 +50,20 @@ bool config_ok(const kf_config* c) {
   if (c->prefill_impl != KF_PREFILL_TENSOR && c->prefill_impl != KF_PREFILL_SIMT) return false;
   if (c->pos_mode != KF_POS_ORIGINAL && c->pos_mode != KF_POS_NEW) return false;
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
+  if (c->n_kv_heads < 0 || c->n_kv_heads > c->n_heads) return false;
+  if (c->n_kv_heads > 0 && (c->n_heads % c->n_kv_heads != 0 || !kf::decode_group_supported(c->n_heads / c->n_kv_heads))) return false;
   if (c->debug_canaries < 0 || c->debug_canaries > 1 || c->debug_fail_first_wait < 0 || c->debug_fail_first_wait > 1) return false;
   return true;
 }
 
 Layout make_layout(const kf_config* c) {
   Layout L{};
-  const size_t units = (size_t)c->batch * c->n_heads;
+  const int hkv = c->n_kv_heads > 0 ? c->n_kv_heads : c->n_heads;
+  const size_t units = (size_t)c->batch * hkv, units_q = (size_t)c->batch * c->n_heads;
   const size_t k = (size_t)c->budget_k, d = (size_t)c->head_dim, nl = (size_t)c->n_layers;
   L.units = (int)units;
+  L.units_q = (int)units_q;
+  L.group = c->n_heads / hkv;
   L.max_splits = kf::decode_max_splits();
   L.kv_layer = align_up(units * k * d * 2);
   L.sc_layer = align_up(units * k * 4);
@@ -73,17 +80,19 @@ Layout make_layout(const kf_config* c) {
   L.acc = carve(nl * L.sc_layer);
   L.pos = carve(nl * L.sc_layer);
   L.len = carve(nl * L.len_layer);
-  L.y_scratch = carve(align_up(units * (k + 1) * 4));
-  L.partials = carve(align_up(units * (size_t)L.max_splits * (4 + d) * 4));
+  L.y_scratch = carve(align_up(units_q * (k + 1) * 4));
+  L.partials = carve(align_up(units_q * (size_t)L.max_splits * (4 + d) * 4));
   L.err = carve(ALIGN);
   L.slopes = carve(align_up((size_t)c->n_heads * 4));
   L.acc_full = carve(align_up(units * (size_t)c->max_prompt_len * 4));
   L.idx = carve(align_up(units * k * 4));
-  L.staging = carve(8 * align_up(units * d * 2));   // two sets of (q, k_new, v_new, out)
-  L.lse2 = carve(align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4));
-  L.lse_x = carve(align_up(kf::prefill_tc_lse_floats((int)units, c->max_prompt_len) * 4));
+  L.staging = carve(8 * align_up(units_q * d * 2));   // two sets of (q, k_new, v_new, out)
+  L.lse2 = carve(align_up(kf::prefill_tc_lse_floats((int)units_q, c->max_prompt_len) * 4));
+  L.lse_x = carve(align_up(kf::prefill_tc_lse_floats((int)units_q, c->max_prompt_len) * 4));
   L.place = off;
   if (c->pos_mode == KF_POS_NEW) L.place = carve(nl * L.sc_layer);
+  L.acc_q = off;
+  if (L.group > 1) L.acc_q = carve(align_up(units_q * (size_t)c->max_prompt_len * 4));
   L.total = off;
   return L;
 }
@@ -159,6 +168,8 @@ static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt
   const Layout& L = ctx->lay;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float* acc_full = d_score_opt ? d_score_opt : reinterpret_cast<float*>(ctx->ws + L.acc_full);
+  // with shared key/value heads the scoring kernels leave one f_theta per query head; their mean over a group is the cache's
+  float* acc_scored = L.group > 1 ? reinterpret_cast<float*>(ctx->ws + L.acc_q) : acc_full;
   int* err = reinterpret_cast<int*>(ctx->ws + L.err);
   const float* slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   const float inv_tau = (float)(1.0 / (double)c.tau_init);  // the prompt phase is iteration t = 0 of Eq. 12
@@ -168,30 +179,36 @@ static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt
     A.K = static_cast<const __half*>(d_k);
     A.lse2 = reinterpret_cast<float*>(ctx->ws + L.lse2);
     A.lse_x = want_x ? reinterpret_cast<float*>(ctx->ws + L.lse_x) : nullptr;
-    A.acc_full = acc_full;
+    A.acc_full = acc_scored;
     A.slopes = slopes;
     A.err = err;
+    A.group = L.group;
     A.n = n_prompt; A.H = c.n_heads; A.layer = layer; A.noise_mode = c.noise_mode; A.bias_mode = c.bias_mode;
     A.scale = ctx->scale; A.inv_tau = inv_tau; A.noise_const = c.noise_const;
     A.noise_mu = c.noise_mu; A.noise_sigma = c.noise_sigma;
     A.pk = ctx->pk;
-    if (kf::launch_prefill_score_tc(A, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+    if (kf::launch_prefill_score_tc(A, c.head_dim, L.units_q, st) != cudaSuccess) return KF_ECUDA;
     ctx->launches += 2;
   } else {
-    if (cudaMemsetAsync(acc_full, 0, (size_t)L.units * n_prompt * 4, st) != cudaSuccess) return KF_ECUDA;
+    if (cudaMemsetAsync(acc_scored, 0, (size_t)L.units_q * n_prompt * 4, st) != cudaSuccess) return KF_ECUDA;
     kf::PrefillParams P{};
     P.Q = static_cast<const __half*>(d_q);
     P.K = static_cast<const __half*>(d_k);
-    P.acc_full = acc_full;
+    P.acc_full = acc_scored;
     P.slopes = slopes;
     P.err = err;
+    P.group = L.group;
     P.n = n_prompt; P.H = c.n_heads; P.layer = layer; P.noise_mode = c.noise_mode; P.bias_mode = c.bias_mode;
     P.scale = ctx->scale;
     P.inv_tau = inv_tau;
     P.noise_const = c.noise_const;
     P.noise_mu = c.noise_mu; P.noise_sigma = c.noise_sigma;
     P.pk = ctx->pk;
-    if (kf::launch_prefill_score_simt(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+    if (kf::launch_prefill_score_simt(P, c.head_dim, L.units_q, st) != cudaSuccess) return KF_ECUDA;
+    ctx->launches += 1;
+  }
+  if (L.group > 1) {
+    if (kf::launch_group_mean(acc_scored, acc_full, L.units, L.group, n_prompt, st) != cudaSuccess) return KF_ECUDA;
     ctx->launches += 1;
   }
 
@@ -232,7 +249,7 @@ static int prefill_attend_impl(kf_ctx* ctx, int32_t n_prompt, const void* d_q, c
                                void* d_out, bool have_lse_x, void* stream) {
   if (!ctx || !d_q || !d_k || !d_v || !d_out) return KF_EINVAL;
   const kf_config& c = ctx->cfg;
-  if (n_prompt < 1) return KF_EINVAL;
+  if (n_prompt < 1 || n_prompt > c.max_prompt_len) return KF_EINVAL;
   if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) | reinterpret_cast<uintptr_t>(d_v) |
        reinterpret_cast<uintptr_t>(d_out)) & 15u)
     return KF_EINVAL;
@@ -246,8 +263,9 @@ static int prefill_attend_impl(kf_ctx* ctx, int32_t n_prompt, const void* d_q, c
   A.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   A.err = reinterpret_cast<int*>(ctx->ws + L.err);
   A.n = n_prompt; A.H = c.n_heads; A.bias_mode = c.bias_mode;
+  A.group = L.group;
   A.scale = ctx->scale;
-  if (kf::launch_prefill_attend(A, c.head_dim, L.units, static_cast<cudaStream_t>(stream)) != cudaSuccess) return KF_ECUDA;
+  if (kf::launch_prefill_attend(A, c.head_dim, L.units_q, static_cast<cudaStream_t>(stream)) != cudaSuccess) return KF_ECUDA;
   ctx->launches += 1;
   return KF_OK;
 }
@@ -301,6 +319,7 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   kf::decode_plan(L.units, c.budget_k, c.decode_splits, &splits, &tps);
   P.splits = splits; P.tiles_per_split = tps;
   P.H = c.n_heads; P.layer = layer; P.noise_mode = c.noise_mode; P.bias_mode = c.bias_mode;
+  P.group = L.group;
   P.scale = ctx->scale;
   // Eq. 12 with t = step, clamped at T; T = 0 keeps tau_init
   double tau = c.tau_init;
@@ -354,7 +373,8 @@ int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
     if (!ok) return KF_ECUDA;
   }
   const Layout& L = ctx->lay;
-  const size_t bytes = (size_t)L.units * ctx->cfg.head_dim * 2;
+  const size_t bytes = (size_t)L.units_q * ctx->cfg.head_dim * 2;      // q and out: one row per query head
+  const size_t bytes_kv = (size_t)L.units * ctx->cfg.head_dim * 2;     // k_new, v_new: one row per cache
   const size_t stride = align_up(bytes);
   const int set = (int)(ctx->host_calls & 1);
   unsigned char* sq = ctx->ws + L.staging + (size_t)set * 4 * stride;
@@ -365,8 +385,8 @@ int kf_decode_step_host(kf_ctx* ctx, int32_t layer, int32_t step,
   // read by the kernel of two calls ago.  (Waiting on an event that was never recorded is a no-op.)
   bool ok = cudaStreamWaitEvent(ctx->copy_in, ctx->kernel_done[set], 0) == cudaSuccess &&
             cudaMemcpyAsync(sq, h_q, bytes, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
-            cudaMemcpyAsync(sk, h_knew, bytes, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
-            cudaMemcpyAsync(sv, h_vnew, bytes, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
+            cudaMemcpyAsync(sk, h_knew, bytes_kv, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
+            cudaMemcpyAsync(sv, h_vnew, bytes_kv, cudaMemcpyHostToDevice, ctx->copy_in) == cudaSuccess &&
             cudaEventRecord(ctx->in_done[set], ctx->copy_in) == cudaSuccess &&
             cudaStreamWaitEvent(st, ctx->in_done[set], 0) == cudaSuccess &&
             cudaStreamWaitEvent(st, ctx->out_done[set], 0) == cudaSuccess;   // `out` of two calls ago has left
@@ -425,6 +445,7 @@ int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t
   P.k = a->budget_k; P.w = a->recent_w; P.p = a->position;
   P.splits = splits; P.tiles_per_split = tps;
   P.H = a->n_heads; P.layer = a->layer; P.noise_mode = a->noise_mode; P.bias_mode = a->bias_mode;
+  P.group = 1;
   P.scale = a->logit_scale > 0.f ? a->logit_scale : (float)(1.0 / std::sqrt((double)a->head_dim));
   P.inv_tau = (float)(1.0 / a->tau);
   P.noise_const = a->noise_const;
@@ -568,7 +589,7 @@ int kf_describe_decode(const kf_ctx* ctx, char* buf, size_t n) {
   int splits = 1, tps = 4;
   kf::decode_plan(ctx->lay.units, ctx->cfg.budget_k, ctx->cfg.decode_splits, &splits, &tps);
   const int len = kf::decode_describe(buf, n, ctx->cfg.head_dim, ctx->lay.units, ctx->cfg.budget_k, splits, tps,
-                                      ctx->cfg.pos_mode == KF_POS_NEW);
+                                      ctx->cfg.pos_mode == KF_POS_NEW, ctx->lay.group);
   return len < 0 ? KF_EINVAL : len;
 }
 

@@ -58,22 +58,25 @@ __device__ __forceinline__ unsigned long long evict_key(float a, int pos) {
 // Closing a unit: merge splits, normalise, accumulate, evict, replace.  Everything that does not depend on the
 // streaming kernel (scores and positions of the entries, the new token's own logit) is requested before
 // `griddepcontrol.wait`, i.e. while the streaming kernel's last CTAs are still running.
-template <int D, int NT>
+// G query heads share the unit's cache (G = 1: the method as printed): every head has its own split partials,
+// adjusted logits and output row; the score added to f_theta is the mean of the heads' softmaxes (Eq. 11).
+template <int D, int NT, int G>
 __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   __shared__ unsigned long long sh_key[NT / 32];
   __shared__ int sh_j[NT / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int H = P.H;
-  const uint32_t b = (uint32_t)(u / H), h = (uint32_t)(u % H), lh = (uint32_t)P.layer * H + h;
-  const __half* q = P.q + (size_t)u * D;
+  const int Hkv = P.H / G;
+  const uint32_t b = (uint32_t)(u / Hkv), h0 = (uint32_t)(u % Hkv) * G, lh0 = (uint32_t)P.layer * P.H + h0;
+  const __half* q = P.q + (size_t)u * G * D;
   const __half* kn = P.knew + (size_t)u * D;
   const __half* vn = P.vnew + (size_t)u * D;
   constexpr int PSTRIDE = 4 + D;
   constexpr int CPT = (D + NT - 1) / NT;   // output columns per thread
-  const float* part = P.partials + (size_t)u * P.splits * PSTRIDE;
+  constexpr float INV_G = 1.0f / (float)G;
+  const float* part = P.partials + (size_t)u * P.splits * G * PSTRIDE;   // [split][head][4 + D]
   float* __restrict__ acc = P.acc + (size_t)u * P.k;
   int32_t* __restrict__ pos = P.pos + (size_t)u * P.k;
-  const float* __restrict__ ys = P.y_scratch + (size_t)u * (P.k + 1);
+  const float* __restrict__ ys = P.y_scratch + (size_t)u * G * (P.k + 1);   // [head][k + 1]
 
   // ---- independent of the streaming kernel: scores and positions of the first batch of entries, the new
   //      token's row, its own logit and adjusted logit (every warp computes these for itself: no hand-over)
@@ -99,56 +102,64 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
     kn_r[i] = c < D ? kn[c] : __float2half(0.f);
     vn_r[i] = c < D ? vn[c] : __float2half(0.f);
   }
-  float s = 0.f;
-  for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[c]), __half2float(kn[c]), s);
-  const float x_new = warp_sum(s) * P.scale;  // bias(p, p) = 0
-  float y_new = 0.f;
-  if (lane == 0) y_new = (x_new + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
-  y_new = __shfl_sync(0xffffffffu, y_new, 0);
+  float x_new[G], y_new[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float s = 0.f;
+    for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[g * D + c]), __half2float(kn[c]), s);
+    x_new[g] = warp_sum(s) * P.scale;  // bias(p, p) = 0
+    float yn = 0.f;
+    if (lane == 0) yn = (x_new[g] + noise_for(P, b, lh0 + g, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
+    y_new[g] = __shfl_sync(0xffffffffu, yn, 0);
+  }
 
   asm volatile("griddepcontrol.wait;" ::: "memory");   // the streaming kernel has finished; its writes are visible
 
   // ---- everything the streaming kernel produced is requested at once
+  if (G == 1) {
 #pragma unroll
-  for (int i = 0; i < BATCH; ++i) {
-    const int j = tid + i * NT;
-    yv[i] = j < len ? __ldcg(ys + j) : 0.f;
+    for (int i = 0; i < BATCH; ++i) {
+      const int j = tid + i * NT;
+      yv[i] = j < len ? __ldcg(ys + j) : 0.f;
+    }
   }
-  // (max, sum) pairs of both softmaxes: split `lane` and split `lane + 32`
-  float4 ps0 = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), ps1 = ps0;
-  if (lane < P.splits) ps0 = __ldcg(reinterpret_cast<const float4*>(part + (size_t)lane * PSTRIDE));
-  if (lane + 32 < P.splits) ps1 = __ldcg(reinterpret_cast<const float4*>(part + (size_t)(lane + 32) * PSTRIDE));
-  const float mx = warp_max(fmaxf(x_new, fmaxf(ps0.y > 0.f ? ps0.x : -INFINITY, ps1.y > 0.f ? ps1.x : -INFINITY)));
-  const float my = warp_max(fmaxf(y_new, fmaxf(ps0.w > 0.f ? ps0.z : -INFINITY, ps1.w > 0.f ? ps1.z : -INFINITY)));
-  const float w0 = ps0.y > 0.f ? fast_exp2((ps0.x - mx) * LOG2E) : 0.f;   // weight of split `lane` in the output
-  const float w1 = ps1.y > 0.f ? fast_exp2((ps1.x - mx) * LOG2E) : 0.f;
-  float lx = fmaf(ps0.y, w0, ps1.y * w1);
-  float ly = (ps0.w > 0.f ? ps0.w * fast_exp2((ps0.z - my) * LOG2E) : 0.f) + (ps1.w > 0.f ? ps1.w * fast_exp2((ps1.z - my) * LOG2E) : 0.f);
-  const float inv_lx = 1.f / (warp_sum(lx) + fast_exp2((x_new - mx) * LOG2E));
-  const float inv_ly = 1.f / (warp_sum(ly) + fast_exp2((y_new - my) * LOG2E));
+  float my[G], inv_ly[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    // (max, sum) pairs of both softmaxes: split `lane` and split `lane + 32`
+    float4 ps0 = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), ps1 = ps0;
+    if (lane < P.splits) ps0 = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)lane * G + g) * PSTRIDE));
+    if (lane + 32 < P.splits) ps1 = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(lane + 32) * G + g) * PSTRIDE));
+    const float mx = warp_max(fmaxf(x_new[g], fmaxf(ps0.y > 0.f ? ps0.x : -INFINITY, ps1.y > 0.f ? ps1.x : -INFINITY)));
+    my[g] = warp_max(fmaxf(y_new[g], fmaxf(ps0.w > 0.f ? ps0.z : -INFINITY, ps1.w > 0.f ? ps1.z : -INFINITY)));
+    const float w0 = ps0.y > 0.f ? fast_exp2((ps0.x - mx) * LOG2E) : 0.f;   // weight of split `lane` in the output
+    const float w1 = ps1.y > 0.f ? fast_exp2((ps1.x - mx) * LOG2E) : 0.f;
+    float lx = fmaf(ps0.y, w0, ps1.y * w1);
+    float ly = (ps0.w > 0.f ? ps0.w * fast_exp2((ps0.z - my[g]) * LOG2E) : 0.f) + (ps1.w > 0.f ? ps1.w * fast_exp2((ps1.z - my[g]) * LOG2E) : 0.f);
+    const float inv_lx = 1.f / (warp_sum(lx) + fast_exp2((x_new[g] - mx) * LOG2E));
+    inv_ly[g] = 1.f / (warp_sum(ly) + fast_exp2((y_new[g] - my[g]) * LOG2E));
 
-  // ---- attention output (Eq. 1): merged partial sums plus the new token's own value row
-  {
+    // ---- attention output of this head (Eq. 1): merged partial sums plus the new token's own value row
     float o[CPT];
 #pragma unroll
-    for (int i = 0; i < CPT; ++i) o[i] = fast_exp2((x_new - mx) * LOG2E) * __half2float(vn_r[i]);
+    for (int i = 0; i < CPT; ++i) o[i] = fast_exp2((x_new[g] - mx) * LOG2E) * __half2float(vn_r[i]);
 #pragma unroll 4
     for (int sp = 0; sp < P.splits; ++sp) {
       const float w = __shfl_sync(0xffffffffu, sp < 32 ? w0 : w1, sp & 31);
 #pragma unroll
       for (int i = 0; i < CPT; ++i) {
         const int c = tid + i * NT;
-        if (c < D) o[i] = fmaf(__ldcg(part + (size_t)sp * PSTRIDE + 4 + c), w, o[i]);
+        if (c < D) o[i] = fmaf(__ldcg(part + ((size_t)sp * G + g) * PSTRIDE + 4 + c), w, o[i]);
       }
     }
 #pragma unroll
     for (int i = 0; i < CPT; ++i) {
       const int c = tid + i * NT;
-      if (c < D) P.out[(size_t)u * D + c] = __float2half_rn(o[i] * inv_lx);
+      if (c < D) P.out[((size_t)u * G + g) * D + c] = __float2half_rn(o[i] * inv_lx);
     }
   }
 
-  // ---- score (Eq. 11), accumulation and the eviction candidate
+  // ---- score (Eq. 11; the mean over the group's heads), accumulation and the eviction candidate
   float* __restrict__ sc = P.score_opt ? P.score_opt + (size_t)u * (P.k + 1) : nullptr;
   unsigned long long best = ~0ull;
   int best_j = -1;
@@ -159,16 +170,36 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
       for (int i = 0; i < BATCH; ++i) {
         const int j = j0 + i * NT;
         const bool in = j < len;
-        yv[i] = in ? __ldcg(ys + j) : 0.f;
+        if (G == 1) yv[i] = in ? __ldcg(ys + j) : 0.f;
         av[i] = in ? acc[j] : 0.f;
         pv[i] = in ? pos[j] : 0x7fffffff;
       }
+    }
+    float zv[BATCH];
+    if (G == 1) {
+#pragma unroll
+      for (int i = 0; i < BATCH; ++i) zv[i] = fast_exp2((yv[i] - my[0]) * LOG2E) * inv_ly[0];
+    } else {
+#pragma unroll
+      for (int i = 0; i < BATCH; ++i) zv[i] = 0.f;
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+          const int j = j0 + i * NT;
+          yv[i] = j < len ? __ldcg(ys + (size_t)g * (P.k + 1) + j) : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) zv[i] = fmaf(fast_exp2((yv[i] - my[g]) * LOG2E), inv_ly[g], zv[i]);
+      }
+#pragma unroll
+      for (int i = 0; i < BATCH; ++i) zv[i] *= INV_G;
     }
 #pragma unroll
     for (int i = 0; i < BATCH; ++i) {
       const int j = j0 + i * NT;
       if (j < len) {
-        const float z = fast_exp2((yv[i] - my) * LOG2E) * inv_ly;
+        const float z = zv[i];
         const float a = av[i] + z;
         acc[j] = a;
         if (sc) sc[j] = z;
@@ -179,7 +210,10 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
       }
     }
   }
-  const float z_new = fast_exp2((y_new - my) * LOG2E) * inv_ly;
+  float z_new = 0.f;
+#pragma unroll
+  for (int g = 0; g < G; ++g) z_new = fmaf(fast_exp2((y_new[g] - my[g]) * LOG2E), inv_ly[g], z_new);
+  if (G > 1) z_new *= INV_G;
   if (sc && tid == 0) sc[len] = z_new;
   const unsigned long long key_new = evict_key(z_new, P.p);
 
@@ -263,7 +297,9 @@ __device__ __forceinline__ void dot8_mixed(float& acc, const uint4& kv, const ui
   }
 }
 
-template <int D, int NW, int NSTAGE, bool NEWPOS>
+// G query heads share the unit's cache: every K and V tile is fetched once and used for all G of them
+// (G logits per row, G pairs of running softmaxes, G output rows).
+template <int D, int NW, int NSTAGE, bool NEWPOS, int G>
 __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__ DecodeParams P) {
   constexpr int CPR = D / 8;          // 16-byte chunks per row
   constexpr int LPR = CPR;            // lanes that share one row in the value phase
@@ -271,11 +307,12 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   constexpr int NT = NW * 32;
   constexpr int TILE_BYTES = TILE_ROWS * D * 2;
   constexpr int PSTRIDE = 4 + D;
+  constexpr int ACC = G == 1 ? 4 : (G == 2 ? 2 : 1);   // independent accumulators per logit
 
   extern __shared__ __align__(128) unsigned char dyn_smem[];
-  __shared__ float sh_m[NW], sh_l[NW], sh_my[NW], sh_ly[NW];
-  __shared__ float sh_o[NW][D];
-  __shared__ __align__(16) __half sh_q[D];
+  __shared__ float sh_m[NW][G], sh_l[NW][G], sh_my[NW][G], sh_ly[NW][G];
+  __shared__ float sh_o[NW][G][D];
+  __shared__ __align__(16) __half sh_q[G][D];
 
   // Both kernels of a step are launched with programmatic stream serialization: this grid's CTAs may become
   // resident while the kernel before it in the stream is draining, and wait here until that kernel has
@@ -298,8 +335,11 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   const __half* Ku = P.K + (size_t)u * P.k * D;
   const __half* Vu = P.V + (size_t)u * P.k * D;
   const int32_t* pos_u = P.pos + (size_t)u * P.k;
-  const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
-  const float slope = (P.bias_mode == 1 && P.slopes) ? P.slopes[h] : 0.f;
+  const int Hkv = P.H / G;
+  const uint32_t b = (uint32_t)(u / Hkv), h0 = (uint32_t)(u % Hkv) * G, lh0 = (uint32_t)P.layer * P.H + h0;
+  float slope[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) slope[g] = (P.bias_mode == 1 && P.slopes) ? P.slopes[h0 + g] : 0.f;
 
   // warp-private ring of shared-memory slots filled by bulk async copies
   unsigned char* ring = dyn_smem + (size_t)warp * NSTAGE * TILE_BYTES;
@@ -324,14 +364,20 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   __syncwarp();
   for (int it = 0; it < NSTAGE && it < n_items; ++it) issue(it);
 
-  if (tid < D / 8)
-    reinterpret_cast<uint4*>(sh_q)[tid] = reinterpret_cast<const uint4*>(P.q + (size_t)u * D)[tid];
+  if (tid < G * D / 8)
+    reinterpret_cast<uint4*>(&sh_q[0][0])[tid] = reinterpret_cast<const uint4*>(P.q + (size_t)u * G * D)[tid];
+  if (G * D / 8 > NT && tid + NT < G * D / 8)   // eight heads of 256 features: a second round
+    reinterpret_cast<uint4*>(&sh_q[0][0])[tid + NT] = reinterpret_cast<const uint4*>(P.q + (size_t)u * G * D)[tid + NT];
   __syncthreads();
 
-  float m_x = -INFINITY, l_x = 0.f, m_y = -INFINITY, l_y = 0.f;  // l_* are per-lane partial sums
-  float o[8];
+  float m_x[G], l_x[G], m_y[G], l_y[G];  // l_* are per-lane partial sums
+  float o[G][8];
 #pragma unroll
-  for (int c = 0; c < 8; ++c) o[c] = 0.f;
+  for (int g = 0; g < G; ++g) {
+    m_x[g] = -INFINITY; l_x[g] = 0.f; m_y[g] = -INFINITY; l_y[g] = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) o[g][c] = 0.f;
+  }
   int pos_next = 0;
   // "New Pos": the bias counts places within the cache; the current token stands at place len
   const int32_t* place_u = NEWPOS ? P.place + (size_t)u * P.k : nullptr;
@@ -354,30 +400,43 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
       if (NEWPOS) place_next = (tb + lane < row_end) ? place_u[tb + lane] : 0;
     }
 
-    // ---- logits: lane r computes x of row tile_base + r.  Chunks are visited in a rotated
+    // ---- logits: lane r computes x of row tile_base + r (for each of the G heads).  Chunks are visited in a rotated
     //      order ((c + lane) mod CPR) so that the 16-byte reads of a quarter warp hit distinct banks.
-    float x_mine;
+    float x_mine[G];
     {
       const int it = 2 * ti;
       const bool ok = mbar_wait_bounded(bars + (it % NSTAGE), (uint32_t)((it / NSTAGE) & 1),
                                         ti == 0 ? P.first_wait_limit : DECODE_WAIT_LIMIT);
       if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       const unsigned char* krow = ring + (size_t)(it % NSTAGE) * TILE_BYTES + (size_t)lane * D * 2;
-      const unsigned char* qb = reinterpret_cast<const unsigned char*>(sh_q);
-      float part[4] = {0.f, 0.f, 0.f, 0.f};
+      float part[G][ACC];
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int a = 0; a < ACC; ++a) part[g][a] = 0.f;
 #pragma unroll
       for (int c0 = 0; c0 < CPR; c0 += 4) {
-        uint4 kv[4], qv[4];
+        uint4 kv[4];
+        int ch[4];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const int ch = (c0 + g + lane) & (CPR - 1);
-          kv[g] = *reinterpret_cast<const uint4*>(krow + ch * 16);
-          qv[g] = *reinterpret_cast<const uint4*>(qb + ch * 16);
+        for (int j = 0; j < 4; ++j) {
+          ch[j] = (c0 + j + lane) & (CPR - 1);
+          kv[j] = *reinterpret_cast<const uint4*>(krow + ch[j] * 16);
         }
 #pragma unroll
-        for (int g = 0; g < 4; ++g) dot8_mixed(part[g], kv[g], qv[g]);
+        for (int g = 0; g < G; ++g) {
+          const unsigned char* qb = reinterpret_cast<const unsigned char*>(&sh_q[g][0]);
+          uint4 qv[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) qv[j] = *reinterpret_cast<const uint4*>(qb + ch[j] * 16);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) dot8_mixed(part[g][j % ACC], kv[j], qv[j]);
+        }
       }
-      x_mine = (part[0] + part[1]) + (part[2] + part[3]);
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+        x_mine[g] = ACC == 4 ? (part[g][0] + part[g][1 % ACC]) + (part[g][2 % ACC] + part[g][3 % ACC])
+                             : (ACC == 2 ? part[g][0] + part[g][1 % ACC] : part[g][0]);
       __syncwarp();
       consumed = it + 1;
       if (it + NSTAGE < n_items) issue(it + NSTAGE);
@@ -385,25 +444,29 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
 
     // ---- per-row work: bias, noise, the two running softmaxes (warp-common maxima, per-lane sums)
     const bool valid = lane < rows;
-    float x = -INFINITY, y = -INFINITY;
-    if (valid) {
-      x = fmaf(x_mine, P.scale, -slope * (float)dist);
-      y = (x + noise_for(P, b, lh, (uint32_t)P.p, (uint32_t)pj)) * P.inv_tau;
-      P.y_scratch[(size_t)u * (P.k + 1) + tile_base + lane] = y;
-    }
-    const float mx_new = fmaxf(m_x, warp_max_redux(x));
-    const float my_new = fmaxf(m_y, warp_max_redux(y));
-    const float corr_x = fast_exp2((m_x - mx_new) * LOG2E);   // 0 on the first tile (m_x = -inf)
-    const float corr_y = fast_exp2((m_y - my_new) * LOG2E);
-    const float pr = valid ? fast_exp2((x - mx_new) * LOG2E) : 0.f;
-    const float ey = valid ? fast_exp2((y - my_new) * LOG2E) : 0.f;
-    const __half2 pr_h2 = __float2half2_rn(pr);
-    const uint32_t pr_pair = *reinterpret_cast<const uint32_t*>(&pr_h2);   // (p, p) as binary16, for the value phase
-    l_x = fmaf(l_x, corr_x, pr);
-    l_y = fmaf(l_y, corr_y, ey);
-    m_x = mx_new; m_y = my_new;
+    uint32_t pr_pair[G];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) o[c] *= corr_x;
+    for (int g = 0; g < G; ++g) {
+      float x = -INFINITY, y = -INFINITY;
+      if (valid) {
+        x = fmaf(x_mine[g], P.scale, -slope[g] * (float)dist);
+        y = (x + noise_for(P, b, lh0 + g, (uint32_t)P.p, (uint32_t)pj)) * P.inv_tau;
+        P.y_scratch[((size_t)u * G + g) * (P.k + 1) + tile_base + lane] = y;
+      }
+      const float mx_new = fmaxf(m_x[g], warp_max_redux(x));
+      const float my_new = fmaxf(m_y[g], warp_max_redux(y));
+      const float corr_x = fast_exp2((m_x[g] - mx_new) * LOG2E);   // 0 on the first tile (m_x = -inf)
+      const float corr_y = fast_exp2((m_y[g] - my_new) * LOG2E);
+      const float pr = valid ? fast_exp2((x - mx_new) * LOG2E) : 0.f;
+      const float ey = valid ? fast_exp2((y - my_new) * LOG2E) : 0.f;
+      const __half2 pr_h2 = __float2half2_rn(pr);
+      pr_pair[g] = *reinterpret_cast<const uint32_t*>(&pr_h2);   // (p, p) as binary16, for the value phase
+      l_x[g] = fmaf(l_x[g], corr_x, pr);
+      l_y[g] = fmaf(l_y[g], corr_y, ey);
+      m_x[g] = mx_new; m_y[g] = my_new;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) o[g][c] *= corr_x;
+    }
 
     // ---- value accumulation: LPR lanes share a row, each owns 8 columns
     {
@@ -415,15 +478,19 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
 #pragma unroll
       for (int i0 = 0; i0 < NLD; i0 += CH) {
         uint4 vv[CH];
-        uint32_t a[CH];
 #pragma unroll
         for (int i = 0; i < CH; ++i) {
           const int r = grp * LPR + i0 + i;
-          a[i] = __shfl_sync(0xffffffffu, pr_pair, r);
           vv[i] = r < rows ? *reinterpret_cast<const uint4*>(slot + (size_t)r * D * 2) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
-        for (int i = 0; i < CH; ++i) axpy8(o, a[i], vv[i]);
+        for (int g = 0; g < G; ++g) {
+          uint32_t a[CH];
+#pragma unroll
+          for (int i = 0; i < CH; ++i) a[i] = __shfl_sync(0xffffffffu, pr_pair[g], grp * LPR + i0 + i);
+#pragma unroll
+          for (int i = 0; i < CH; ++i) axpy8(o[g], a[i], vv[i]);
+        }
       }
       __syncwarp();
       consumed = it + 1;
@@ -440,60 +507,63 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
   }
 
   // ---- merge the lanes, then the warps of this CTA
-  l_x = warp_sum(l_x);
-  l_y = warp_sum(l_y);
 #pragma unroll
-  for (int off = LPR; off < 32; off <<= 1) {
+  for (int g = 0; g < G; ++g) {
+    l_x[g] = warp_sum(l_x[g]);
+    l_y[g] = warp_sum(l_y[g]);
 #pragma unroll
-    for (int c = 0; c < 8; ++c) o[c] += __shfl_xor_sync(0xffffffffu, o[c], off);
+    for (int off = LPR; off < 32; off <<= 1) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) o[g][c] += __shfl_xor_sync(0xffffffffu, o[g][c], off);
+    }
+    if (grp == 0) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) sh_o[warp][g][sub * 8 + c] = o[g][c];
+    }
+    if (lane == 0) { sh_m[warp][g] = m_x[g]; sh_l[warp][g] = l_x[g]; sh_my[warp][g] = m_y[g]; sh_ly[warp][g] = l_y[g]; }
   }
-  if (grp == 0) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) sh_o[warp][sub * 8 + c] = o[c];
-  }
-  if (lane == 0) { sh_m[warp] = m_x; sh_l[warp] = l_x; sh_my[warp] = m_y; sh_ly[warp] = l_y; }
   __syncthreads();
-  float* part = P.partials + ((size_t)u * P.splits + s) * PSTRIDE;
-  {
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float* part = P.partials + (((size_t)u * P.splits + s) * G + g) * PSTRIDE;
     float M = -INFINITY, MY = -INFINITY;
 #pragma unroll
-    for (int wi = 0; wi < NW; ++wi) { M = fmaxf(M, sh_m[wi]); MY = fmaxf(MY, sh_my[wi]); }
+    for (int wi = 0; wi < NW; ++wi) { M = fmaxf(M, sh_m[wi][g]); MY = fmaxf(MY, sh_my[wi][g]); }
     float sc[NW];
 #pragma unroll
-    for (int wi = 0; wi < NW; ++wi) sc[wi] = sh_l[wi] > 0.f ? fast_exp2((sh_m[wi] - M) * LOG2E) : 0.f;
+    for (int wi = 0; wi < NW; ++wi) sc[wi] = sh_l[wi][g] > 0.f ? fast_exp2((sh_m[wi][g] - M) * LOG2E) : 0.f;
     for (int c = tid; c < D; c += NT) {
       float acc_o = 0.f;
 #pragma unroll
-      for (int wi = 0; wi < NW; ++wi) acc_o = fmaf(sh_o[wi][c], sc[wi], acc_o);
+      for (int wi = 0; wi < NW; ++wi) acc_o = fmaf(sh_o[wi][g][c], sc[wi], acc_o);
       part[4 + c] = acc_o;
     }
     if (tid == 0) {
       float L = 0.f, LY = 0.f;
 #pragma unroll
       for (int wi = 0; wi < NW; ++wi) {
-        L = fmaf(sh_l[wi], sc[wi], L);
-        if (sh_ly[wi] > 0.f) LY = fmaf(sh_ly[wi], fast_exp2((sh_my[wi] - MY) * LOG2E), LY);
+        L = fmaf(sh_l[wi][g], sc[wi], L);
+        if (sh_ly[wi][g] > 0.f) LY = fmaf(sh_ly[wi][g], fast_exp2((sh_my[wi][g] - MY) * LOG2E), LY);
       }
       part[0] = M; part[1] = L; part[2] = MY; part[3] = LY;
     }
   }
-
 }
 
 // One CTA per unit, launched behind the streaming kernel as its programmatic dependent.
-template <int D>
-__global__ void __launch_bounds__(128, 8) decode_close_kernel(const __grid_constant__ DecodeParams P) {
+template <int D, int G>
+__global__ void __launch_bounds__(128, G == 1 ? 8 : 4) decode_close_kernel(const __grid_constant__ DecodeParams P) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // lets the next kernel's CTAs queue up behind this grid
   const int u = blockIdx.x;
   const int len = P.len[u];
   if (len < 0 || len > P.k) return;   // reported by the streaming kernel; nothing of the unit is written
-  combine_and_evict<D, 128>(P, u, len);
+  combine_and_evict<D, 128, G>(P, u, len);
 }
 
-template <int D, int NW, int NSTAGE>
+template <int D, int NW, int NSTAGE, int G>
 cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   constexpr size_t smem = (size_t)NW * NSTAGE * (TILE_ROWS * D * 2) + (size_t)NW * NSTAGE * 8;
-  auto kern = P.place ? decode_kernel<D, NW, NSTAGE, true> : decode_kernel<D, NW, NSTAGE, false>;
+  auto kern = P.place ? decode_kernel<D, NW, NSTAGE, true, G> : decode_kernel<D, NW, NSTAGE, false, G>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -515,7 +585,7 @@ cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   cfg.gridDim = dim3((unsigned)units);
   cfg.blockDim = dim3(128);
   cfg.dynamicSmemBytes = 0;
-  return cudaLaunchKernelEx(&cfg, decode_close_kernel<D>, P);
+  return cudaLaunchKernelEx(&cfg, decode_close_kernel<D, G>, P);
 }
 
 // One CTA per unit: place[j] = #{i : pos[i] < pos[j]} (positions of a unit are distinct).
@@ -559,29 +629,51 @@ void decode_plan(int units, int budget_k, int requested, int* splits_out, int* t
 
 // Template arguments <D, NW, NSTAGE> of the streaming kernel launch_decode picks for a shape (one table for the
 // launcher and for kf_describe_decode).
-static void decode_variant(int head_dim, int tiles_per_split, int* nw, int* nstage) {
-  *nw = (head_dim == 128 && tiles_per_split >= 16) ? 5 : 4;
+static void decode_variant(int head_dim, int tiles_per_split, int group, int* nw, int* nstage) {
+  *nw = (head_dim == 128 && tiles_per_split >= 16 && group == 1) ? 5 : 4;
   *nstage = head_dim == 64 ? 4 : 2;
 }
 
-int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos) {
+int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
+                    int group) {
   int nw = 4, nstage = 2;
-  decode_variant(head_dim, tiles_per_split, &nw, &nstage);
-  return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d> + decode_close_kernel<%d>; units=%d k=%d splits=%d tiles_per_split=%d group=1",
-                  head_dim, nw, nstage, new_pos ? 1 : 0, head_dim, units, budget_k, splits, tiles_per_split);
+  decode_variant(head_dim, tiles_per_split, group, &nw, &nstage);
+  if (group == 1)
+    return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d> + decode_close_kernel<%d>; units=%d k=%d splits=%d tiles_per_split=%d group=1",
+                    head_dim, nw, nstage, new_pos ? 1 : 0, head_dim, units, budget_k, splits, tiles_per_split);
+  return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d,%d> + decode_close_kernel<%d,%d>; units=%d k=%d splits=%d tiles_per_split=%d group=%d",
+                  head_dim, nw, nstage, new_pos ? 1 : 0, group, head_dim, group, units, budget_k, splits, tiles_per_split, group);
 }
 
-cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
-  if (P.splits < 1 || P.splits > MAX_SPLITS) return cudaErrorInvalidValue;
+bool decode_group_supported(int group) { return group == 1 || group == 2 || group == 4 || group == 8; }
+
+namespace {
+template <int G>
+cudaError_t launch_group(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
   int nw = 4, nstage = 2;
-  decode_variant(head_dim, P.tiles_per_split, &nw, &nstage);
+  decode_variant(head_dim, P.tiles_per_split, G, &nw, &nstage);
   switch (head_dim) {
-    case 64: return launch_one<64, 4, 4>(P, units, stream);
+    case 64: return launch_one<64, 4, 4, G>(P, units, stream);
     case 128:
       // long items (bandwidth-bound workloads): five warps and 80 KB of ring per CTA, two CTAs per SM, measured best;
       // short items (few units, latency-bound): four warps, three CTAs per SM
-      return nw == 5 ? launch_one<128, 5, 2>(P, units, stream) : launch_one<128, 4, 2>(P, units, stream);
-    case 256: return launch_one<256, 4, 2>(P, units, stream);
+      if constexpr (G == 1) {
+        if (nw == 5) return launch_one<128, 5, 2, 1>(P, units, stream);
+      }
+      return launch_one<128, 4, 2, G>(P, units, stream);
+    case 256: return launch_one<256, 4, 2, G>(P, units, stream);
+    default: return cudaErrorInvalidValue;
+  }
+}
+}  // namespace
+
+cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
+  if (P.splits < 1 || P.splits > MAX_SPLITS) return cudaErrorInvalidValue;
+  switch (P.group) {
+    case 1: return launch_group<1>(P, head_dim, units, stream);
+    case 2: return launch_group<2>(P, head_dim, units, stream);
+    case 4: return launch_group<4>(P, head_dim, units, stream);
+    case 8: return launch_group<8>(P, head_dim, units, stream);
     default: return cudaErrorInvalidValue;
   }
 }

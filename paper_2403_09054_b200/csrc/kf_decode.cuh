@@ -13,18 +13,19 @@ struct DecodeParams {
   int32_t* len;           // [units]     entries in use
   int32_t* place;         // [units][k]  place of each entry within the cache in position order, or null when the
                           //             bias uses the original positions (section 4.4.2)
-  const __half* q;        // [units][d]
+  const __half* q;        // [units][group][d]   (a unit is a cache: one (batch row, key/value head))
   const __half* knew;     // [units][d]
   const __half* vnew;     // [units][d]
-  __half* out;            // [units][d]
+  __half* out;            // [units][group][d]
   float* score_opt;       // [units][k+1] or null
-  float* y_scratch;       // [units][k+1] adjusted logits (x + zeta) / tau
-  float* partials;        // [units][splits][4 + d]
+  float* y_scratch;       // [units][group][k+1] adjusted logits (x + zeta) / tau
+  float* partials;        // [units][splits][group][4 + d]
   int* err;               // device error word
   const float* slopes;    // [H] ALiBi slopes or null
   int32_t k, w, p;        // budget, recent window, position of the query token
   int32_t splits, tiles_per_split;
-  int32_t H, layer, noise_mode, bias_mode;
+  int32_t H, layer, noise_mode, bias_mode;   // H = query heads
+  int32_t group;          // query heads per key/value head (H / group caches per batch row)
   float scale, inv_tau, noise_const, noise_mu, noise_sigma;
   uint32_t first_wait_limit;   // polls the streaming kernel grants its first tile (DECODE_WAIT_LIMIT; 0 in the self-test
                                // that makes a wait run out: the warp gives up at once, then drains with the full limit)
@@ -43,7 +44,9 @@ int decode_max_splits();
 void decode_plan(int units, int budget_k, int requested, int* splits, int* tiles_per_split);
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 // Names the kernels (with their template arguments) and the split plan of a layer call of this shape; snprintf semantics.
-int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos);
+int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
+                    int group);
+bool decode_group_supported(int group);   // query heads per key/value head the generation kernels are built for
 
 // Reorders every unit's entries of one layer into ascending position, in place (see kf_compact.cu).  `place` may be
 // null; `dst_scratch` is [units][k] int32 of scratch.  Budgets above compact_max_k() are refused (cudaErrorInvalidValue).

@@ -8,11 +8,12 @@
 namespace kf {
 
 struct PrefillParams {
-  const __half* Q;     // [units][n][d]
-  const __half* K;     // [units][n][d]
-  float* acc_full;     // [units][n] f_theta before pruning (zeroed by the caller)
+  const __half* Q;     // [units][n][d]            a unit here is a (batch row, query head)
+  const __half* K;     // [units / group][n][d]    query heads of a group read the same keys
+  float* acc_full;     // [units][n] f_theta of each query head before pruning (zeroed by the caller)
   const float* slopes; // [H] or null
   int* err;
+  int32_t group;       // query heads per key/value head
   int32_t n, H, layer, noise_mode, bias_mode;
   float scale, inv_tau, noise_const, noise_mu, noise_sigma;
   PhiloxKeys pk;
@@ -49,7 +50,8 @@ struct PrefillTcParams {
   const float* slopes; // [H] or null
   int* err;
   int32_t n, nblk, H, layer;
-  int32_t units;       // (batch row, head) pairs of the call
+  int32_t units;       // (batch row, query head) pairs of the call
+  int32_t group;       // query heads per key/value head: unit u reads the keys of cache u / group
   float a_scale;       // logit scale * log2(e) / tau
   float ax;            // logit scale * log2(e)
   float c1;            // log2(e) / tau
@@ -61,8 +63,9 @@ struct PrefillTcParams {
 
 // What the caller of the tensor-core scoring provides.
 struct PrefillTcArgs {
-  const __half* Q;     // [units][n][d]
-  const __half* K;
+  const __half* Q;     // [units][n][d]           units = (batch row, query head) pairs
+  const __half* K;     // [units / group][n][d]
+  int32_t group;       // query heads per key/value head
   float* lse2;         // scratch, prefill_tc_lse_floats(units, n) floats
   float* lse_x;        // null, or a second such array: receives the plain softmax statistics of the prompt rows
   float* acc_full;     // [units][n], fully overwritten
@@ -75,9 +78,10 @@ struct PrefillTcArgs {
 
 // Causal attention output of the prompt (see kf_prefill_attend.cu).
 struct PrefillAttendArgs {
-  const __half* Q;     // [units][n][d]
-  const __half* K;
-  const __half* V;
+  const __half* Q;     // [units][n][d]           units = (batch row, query head) pairs
+  const __half* K;     // [units / group][n][d]
+  const __half* V;     // [units / group][n][d]
+  int32_t group;       // query heads per key/value head
   __half* out;         // [units][n][d]
   const float* lse_x;  // null, or the rows' log2-domain log-sum-exp from the scoring sweep (skips the statistics phase)
   const float* slopes; // [H] or null
@@ -91,6 +95,9 @@ size_t prefill_tc_lse_floats(int units, int n_max);
 cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int units, cudaStream_t stream);
 cudaError_t launch_prefill_score_simt(const PrefillParams& P, int head_dim, int units, cudaStream_t stream);
 cudaError_t launch_prefill_select(const SelectParams& P, int units, cudaStream_t stream);
+// dst[c][j] = mean over r < group of src[c * group + r][j]: the prompt scores of a cache from those of its query heads
+// (a fixed summation order, r ascending).
+cudaError_t launch_group_mean(const float* src, float* dst, int caches, int group, int n, cudaStream_t stream);
 cudaError_t launch_prefill_gather(const GatherParams& P, int head_dim, int units, cudaStream_t stream);
 
 }  // namespace kf

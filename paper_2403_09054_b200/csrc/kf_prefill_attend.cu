@@ -31,6 +31,7 @@ struct AttendParams {
   const float* slopes;         // [H] or null
   int* err;
   int32_t n, nblk, H;
+  int32_t group;               // query heads per key/value head: unit u reads the keys and values of cache u / group
   float a_scale;               // logit scale * log2(e)
 };
 
@@ -121,14 +122,14 @@ __global__ void __launch_bounds__(at_threads(NG), 1) prefill_attend(const __grid
           if (kit >= KST) ok = wait_bar(k_empty + s, (uint32_t)((kit / KST - 1) & 1), abort_flag);
           if (!ok) break;
           mbar_expect_tx(k_full + s, KOP_BYTES);
-          for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sK + (size_t)s * KOP_BYTES + kc * KBOX, &P.tmK, kc * 64, t * BN, u, k_full + s);
+          for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sK + (size_t)s * KOP_BYTES + kc * KBOX, &P.tmK, kc * 64, t * BN, u / P.group, k_full + s);
           ++kit;
           if (pass == 1) {
             const int sv = vit % VST;
             if (vit >= VST) ok = wait_bar(v_empty + sv, (uint32_t)((vit / VST - 1) & 1), abort_flag);
             if (!ok) break;
             mbar_expect_tx(v_full + sv, KOP_BYTES);
-            for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sV + (size_t)sv * KOP_BYTES + kc * KBOX, &P.tmV, kc * 64, t * BN, u, v_full + sv);
+            for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sV + (size_t)sv * KOP_BYTES + kc * KBOX, &P.tmV, kc * 64, t * BN, u / P.group, v_full + sv);
             ++vit;
           }
         }
@@ -381,8 +382,9 @@ cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int 
   AttendParams P{};
   const int bn = head_dim == 256 ? 64 : 128;   // key / value rows per tile
   if (!make_operand_map(&P.tmQ, a.Q, units, a.n, head_dim, 128)) return cudaErrorNotSupported;
-  if (!make_operand_map(&P.tmK, a.K, units, a.n, head_dim, bn)) return cudaErrorNotSupported;
-  if (!make_operand_map(&P.tmV, a.V, units, a.n, head_dim, bn)) return cudaErrorNotSupported;
+  if (a.group < 1 || units % a.group != 0) return cudaErrorInvalidValue;
+  if (!make_operand_map(&P.tmK, a.K, units / a.group, a.n, head_dim, bn)) return cudaErrorNotSupported;
+  if (!make_operand_map(&P.tmV, a.V, units / a.group, a.n, head_dim, bn)) return cudaErrorNotSupported;
   P.out = a.out;
   P.lse_in = a.lse_x;
   P.slopes = a.slopes;
@@ -390,6 +392,7 @@ cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int 
   P.n = a.n;
   P.nblk = (a.n + 127) / 128;
   P.H = a.H;
+  P.group = a.group;
   P.a_scale = a.scale * LOG2E;
   const bool alibi = a.bias_mode == 1 && a.slopes != nullptr;
   switch (head_dim) {

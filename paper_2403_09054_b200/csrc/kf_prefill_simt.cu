@@ -4,6 +4,8 @@
 //   prefill_gather     : copy the kept K/V rows, positions and scores into the k-slot cache
 #include "kf_prefill.cuh"
 
+#include <algorithm>
+
 namespace kf {
 
 namespace {
@@ -36,7 +38,7 @@ __global__ void __launch_bounds__(NTH) prefill_score_simt(const __grid_constant_
   const uint32_t b = (uint32_t)(u / P.H), h = (uint32_t)(u % P.H), lh = (uint32_t)P.layer * P.H + h;
   const float slope = (P.bias_mode == 1 && P.slopes) ? P.slopes[h] : 0.f;
   const __half* Qu = P.Q + (size_t)u * n * D;
-  const __half* Ku = P.K + (size_t)u * n * D;
+  const __half* Ku = P.K + (size_t)(u / P.group) * n * D;   // the keys of this query head's cache
   float* acc_u = P.acc_full + (size_t)u * n;
 
   for (int e = tid; e < BM * D; e += NTH) {
@@ -281,6 +283,24 @@ cudaError_t launch_prefill_score_simt(const PrefillParams& P, int head_dim, int 
     default:
       return cudaErrorInvalidValue;
   }
+  return cudaGetLastError();
+}
+
+namespace {
+__global__ void __launch_bounds__(256) group_mean_kernel(const float* __restrict__ src, float* __restrict__ dst, int group, int n) {
+  const int c = blockIdx.y;
+  const float inv = 1.0f / (float)group;
+  for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
+    float s = 0.f;
+    for (int r = 0; r < group; ++r) s += src[((size_t)c * group + r) * n + j];
+    dst[(size_t)c * n + j] = s * inv;
+  }
+}
+}  // namespace
+
+cudaError_t launch_group_mean(const float* src, float* dst, int caches, int group, int n, cudaStream_t stream) {
+  dim3 grid((unsigned)std::min((n + 255) / 256, 64), (unsigned)caches);
+  group_mean_kernel<<<grid, 256, 0, stream>>>(src, dst, group, n);
   return cudaGetLastError();
 }
 

@@ -187,7 +187,9 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
         // the resident block may be replaced once the MMAs of the previous item have read it
         if (k > 0 && !wait_bar(r_empty, (uint32_t)((k - 1) & 1), abort_flag)) { ok = false; break; }
         mbar_expect_tx(r_full, OP_BYTES);
-        for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sR + kc * TC_BOX_BYTES, mapR, kc * 64, Rb * TC_BM, u, r_full);
+        // unit u is a (batch row, query head); its keys are those of cache u / group
+        const int uR = SWEEP2 ? u / P.group : u, uS = SWEEP2 ? u : u / P.group;
+        for (int kc = 0; kc < KCH; ++kc) tma_load_3d(sR + kc * TC_BOX_BYTES, mapR, kc * 64, Rb * TC_BM, uR, r_full);
         issued_slot[1] = k + 1;
         const int t_begin = SWEEP2 ? Rb : 0, n_tiles = tiles_of(Rb);
         for (int it = 0; it < n_tiles; ++it, ++gt) {
@@ -195,7 +197,7 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
           if (gt >= NST && !wait_bar(s_empty + s, (uint32_t)((gt / NST - 1) & 1), abort_flag)) { ok = false; break; }
           mbar_expect_tx(s_full + s, OP_BYTES);
           unsigned char* dst = sS + (size_t)s * OP_BYTES;
-          for (int kc = 0; kc < KCH; ++kc) tma_load_3d(dst + kc * TC_BOX_BYTES, mapS, kc * 64, (t_begin + it) * TC_BN, u, s_full + s);
+          for (int kc = 0; kc < KCH; ++kc) tma_load_3d(dst + kc * TC_BOX_BYTES, mapS, kc * 64, (t_begin + it) * TC_BN, uS, s_full + s);
         }
       }
       if (!ok) {
@@ -620,7 +622,8 @@ cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int un
   if (a.n < 1 || units < 1 || units > 65535) return cudaErrorInvalidValue;
   PrefillTcParams P{};
   if (!make_operand_map(&P.tmQ, a.Q, units, a.n, head_dim)) return cudaErrorNotSupported;
-  if (!make_operand_map(&P.tmK, a.K, units, a.n, head_dim)) return cudaErrorNotSupported;
+  if (a.group < 1 || units % a.group != 0) return cudaErrorInvalidValue;
+  if (!make_operand_map(&P.tmK, a.K, units / a.group, a.n, head_dim)) return cudaErrorNotSupported;
   P.lse2 = a.lse2;
   P.lse_x = a.lse_x;
   P.ax = a.scale * LOG2E;
@@ -630,6 +633,7 @@ cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int un
   P.n = a.n;
   P.nblk = (a.n + TC_BM - 1) / TC_BM;
   P.units = units;
+  P.group = a.group;
   P.H = a.H;
   P.layer = a.layer;
   P.inv_tau = a.inv_tau;

@@ -30,6 +30,7 @@ def oracle_params(wl: W.Workload, noise_mode=ko.NOISE_GUMBEL, logit_scale=0.0, p
     return ko.Params(head_dim=wl.head_dim, n_heads=wl.n_heads, budget_k=wl.budget_k, recent_w=wl.recent_w,
                      gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end,
                      noise_seed=wl.noise_seed, noise_mode=noise_mode, logit_scale=logit_scale, pos_mode=pos_mode,
+                     n_kv_heads=wl.n_kv_heads,
                      bias_mode=1 if wl.positional == "alibi" else 0,
                      alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None)
 
@@ -39,7 +40,7 @@ def make_gpu(wl: W.Workload, noise_mode=kf.KF_NOISE_GUMBEL, max_prompt_len=None,
     (see check_guards): the kernels and their launch shapes are the same with and without them."""
     kw.setdefault("debug_canaries", 1)
     return kf.Keyformer(n_layers=wl.n_layers, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
-                        budget_k=wl.budget_k, recent_w=wl.recent_w,
+                        n_kv_heads=wl.n_kv_heads, budget_k=wl.budget_k, recent_w=wl.recent_w,
                         max_prompt_len=max_prompt_len or wl.prompt_len, gen_len_T=wl.gen_len_T,
                         tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
                         noise_mode=noise_mode,
@@ -79,7 +80,7 @@ class LockStep:
         self.pos_mode = pos_mode
         self.units = np.ascontiguousarray(units, dtype=np.int32).reshape(-1, 3)
         assert (self.units[:, 0] == layer).all()
-        self.flat = torch.as_tensor(self.units[:, 1] * wl.n_heads + self.units[:, 2], dtype=torch.long)
+        self.flat = torch.as_tensor(self.units[:, 1] * wl.kv_heads + self.units[:, 2], dtype=torch.long)
         self.P = oracle_params(wl, noise_mode, logit_scale, pos_mode)
         self.st = ko.State(self.P, self.units)
         self.adoptions = 0
@@ -89,9 +90,16 @@ class LockStep:
 
     # ------------------------------------------------------------------ helpers
     def _rows(self, t: torch.Tensor) -> np.ndarray:
-        """[B, H, ...] device tensor -> numpy rows of the sampled units."""
-        flat = t.reshape(self.wl.batch * self.wl.n_heads, *t.shape[2:])
+        """[B, Hkv, ...] device tensor (one entry per cache) -> numpy rows of the sampled units."""
+        flat = t.reshape(self.wl.batch * self.wl.kv_heads, *t.shape[2:])
         return flat[self.flat.to(t.device)].cpu().numpy()
+
+    def _qrows(self, t: torch.Tensor) -> np.ndarray:
+        """[B, H, ...] device tensor (one entry per query head) -> numpy [U, ...] of the sampled units, or
+        [U, g, ...] when g query heads share a cache (the heads of a group are consecutive)."""
+        g = self.wl.group
+        flat = t.reshape(self.wl.batch * self.wl.kv_heads, g, *t.shape[2:])[self.flat.to(t.device)].cpu().numpy()
+        return flat[:, 0] if g == 1 else flat
 
     def gpu_state(self, rows=True):
         K, V, pos, acc, ln = self.gpu.kf_view_state(self.layer)
@@ -105,7 +113,7 @@ class LockStep:
         wl, gpu = self.wl, self.gpu
         n = q.shape[-2]
         self.n = n
-        score = torch.empty(wl.batch, wl.n_heads, n, dtype=torch.float32, device=q.device)
+        score = torch.empty(wl.batch, wl.kv_heads, n, dtype=torch.float32, device=q.device)
         gpu.kf_prefill_score_prune(self.layer, q, k, v, score_out=score)
         assert gpu.kf_poll_error() == 0
         # every unit of the layer, sampled by the oracle or not: each of the n softmax rows adds 1 to the scores,
@@ -120,8 +128,8 @@ class LockStep:
         n_rec = min(w_, L_all)
         if n_rec > 0:
             assert torch.equal(pos_all[..., L_all - n_rec:L_all].long(),
-                               torch.arange(n - n_rec, n, device=pos_all.device).expand(wl.batch, wl.n_heads, n_rec))
-        Qs, Ks, Vs = self._rows(q), self._rows(k), self._rows(v)
+                               torch.arange(n - n_rec, n, device=pos_all.device).expand(wl.batch, wl.kv_heads, n_rec))
+        Qs, Ks, Vs = self._qrows(q), self._rows(k), self._rows(v)
         acc_ref = self.st.prefill_score(Qs, Ks)
         acc_gpu = self._rows(score).astype(np.float64)
         err = np.abs(acc_gpu - acc_ref) - SCORE_RTOL * np.abs(acc_ref)
@@ -156,7 +164,7 @@ class LockStep:
         U = len(self.units)
         _, _, pos_before, _, len_before = self.gpu_state(rows=False)
         out = torch.empty(wl.batch, wl.n_heads, wl.head_dim, dtype=torch.float16, device=q.device)
-        score = torch.zeros(wl.batch, wl.n_heads, wl.budget_k + 1, dtype=torch.float32, device=q.device)
+        score = torch.zeros(wl.batch, wl.kv_heads, wl.budget_k + 1, dtype=torch.float32, device=q.device)
         len_all_before = self.gpu.kf_view_state(self.layer)[4].clone()
         self.gpu.kf_decode_step(self.layer, step, q, knew, vnew, out, score_out=score)
         assert self.gpu.kf_poll_error() == 0
@@ -190,8 +198,8 @@ class LockStep:
         wl = self.wl
         kk, w = wl.budget_k, wl.recent_w
         U = len(self.units)
-        out_ref, z_ref = self.st.decode_score(step, self._rows(q), self._rows(knew), self._rows(vnew))
-        out_gpu = self._rows(out).astype(np.float64)
+        out_ref, z_ref = self.st.decode_score(step, self._qrows(q), self._rows(knew), self._rows(vnew))
+        out_gpu = self._qrows(out).astype(np.float64)
         z_gpu = self._rows(score).astype(np.float64)
         Kc, Vc, pos_after, acc_after, len_after = self.gpu_state(rows=check_state)
         p = self.n + step - 1
@@ -199,10 +207,10 @@ class LockStep:
         own = np.full(U, -1, dtype=np.int32)
         for u in range(U):
             tag = f"step {step} unit {self.units[u]}"
-            scale = np.abs(out_ref[u]).max()
-            oerr = np.abs(out_gpu[u] - out_ref[u]).max()
-            self.max_out_err = max(self.max_out_err, oerr / scale)
-            assert oerr <= OUT_RTOL * scale, f"{tag}: attention output off by {oerr:.3e} (scale {scale:.3e})"
+            scale = np.abs(out_ref[u]).max(axis=-1)               # per query head of the unit
+            oerr = np.abs(out_gpu[u] - out_ref[u]).max(axis=-1)
+            self.max_out_err = max(self.max_out_err, float((oerr / scale).max()))
+            assert (oerr <= OUT_RTOL * scale).all(), f"{tag}: attention output off by {oerr.max():.3e} (scale {scale.min():.3e})"
             L = int(len_before[u])
             m = L + 1
             assert int(self.st.len[u]) == m

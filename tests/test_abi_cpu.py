@@ -108,3 +108,13 @@ def test_guard_blocks_enlarge_the_workspace():
     base, dbg = kf.kf_workspace_bytes(_cfg()), kf.kf_workspace_bytes(_cfg(debug_canaries=1))
     assert dbg - base == 14 * 256                        # one guard behind each of the 14 sub-buffers (no places)
     assert kf.kf_workspace_bytes(_cfg(debug_canaries=2)) == 0 and kf.kf_workspace_bytes(_cfg(debug_fail_first_wait=3)) == 0
+
+
+def test_unsupported_group_sizes_are_rejected():
+    for hkv in (3, 5, 7):           # 12 / 5, 12 / 7 do not divide; 12 / 3 = 4 is fine
+        cfg = kf.make_config(n_layers=1, batch=1, n_heads=12, n_kv_heads=hkv, head_dim=64, budget_k=8, recent_w=2,
+                             max_prompt_len=16, gen_len_T=4)[0]
+        assert (kf.kf_workspace_bytes(cfg) > 0) == (hkv == 3)
+    cfg = kf.make_config(n_layers=1, batch=1, n_heads=32, n_kv_heads=1, head_dim=64, budget_k=8, recent_w=2,
+                         max_prompt_len=16, gen_len_T=4)[0]
+    assert kf.kf_workspace_bytes(cfg) == 0              # 32 query heads on one cache: more than the kernels are built for

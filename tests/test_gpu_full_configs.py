@@ -46,6 +46,15 @@ def test_config4_cerebras_three_layers_sampled_units_all_steps():
     _report("c4_cerebras", r)
 
 
+def test_config4_cerebras_with_shared_key_value_heads_sampled_units_all_steps():
+    """The Cerebras-shaped model with its 32 query heads on 8 key/value heads (section 6), 24 caches of three layers,
+    all 256 steps."""
+    wl = W.get_config("c4_cerebras_gqa8")
+    r = lockstep.run_workload(wl, units_per_layer=8, layers=[0, wl.n_layers // 2 - 1, wl.n_layers - 1], check_state_every=64)
+    assert r["units"] == 24 and r["steps"] == 256
+    _report("c4_cerebras_gqa8", r)
+
+
 @pytest.mark.parametrize("name", ["c5_prefill_1k", "c5_prefill_2k", "c5_prefill_4k", "c5_prefill_8k"])
 def test_config5_prefill_sweep(name):
     base = W.get_config(name)

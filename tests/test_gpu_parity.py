@@ -437,3 +437,53 @@ def test_misaligned_pointers_are_rejected_on_the_host():
     assert gpu.kf_launch_count() == launches + 4                        # only the accepted prompt call launched
     gpu.kf_decode_step(0, 1, q, kn, vn, out)
     lockstep.check_guards(gpu)
+
+
+# ------------------------------------------------------------------ query heads sharing a key/value head (section 6)
+@pytest.mark.parametrize("impl", [kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_SIMT])
+@pytest.mark.parametrize("d,g", [(64, 2), (128, 4), (256, 8), (128, 8), (64, 4)])
+def test_shared_key_value_heads(d, g, impl):
+    """One cache and one accumulated score per key/value head; every query head of the group has its own logits,
+    noise and softmax; the accumulated score receives the group's mean.  Prompt phase plus generation, in lock
+    step with the oracle (several splits, a ragged last tile)."""
+    wl = _wl(head_dim=d, n_heads=3 * g, n_kv_heads=3, prompt_len=211, budget_k=150, recent_w=20, gen_len_T=10)
+    r = lockstep.run_workload(wl, gpu_kwargs=dict(prefill_impl=impl))
+    assert r["steps"] == 10 and r["units"] == 2 * 3
+
+
+@pytest.mark.parametrize("pos_mode", [0, 1])
+def test_shared_key_value_heads_with_alibi_slopes_per_query_head(pos_mode):
+    wl = W.get_config("c3_mpt").scaled(n_heads=8, n_kv_heads=2, batch=2, prompt_len=300, budget_k=128, recent_w=32, gen_len_T=12)
+    lockstep.run_workload(wl, pos_mode=pos_mode)
+
+
+@pytest.mark.parametrize("noise", ["none", "const", "gauss"])
+def test_shared_key_value_heads_other_adjustments(noise):
+    lockstep.run_workload(_wl(head_dim=128, n_heads=4, n_kv_heads=1, prompt_len=140, budget_k=60, recent_w=12), noise=noise)
+
+
+def test_multi_query_attention_filling_cache_and_window_edge_cases():
+    """All query heads on one cache (MQA); a prompt shorter than the budget (the cache fills during generation),
+    then no recent window, then window = budget."""
+    for n, k, w in ((30, 48, 8), (90, 33, 0), (90, 32, 32)):
+        lockstep.run_workload(_wl(head_dim=64, n_heads=8, n_kv_heads=1, prompt_len=n, budget_k=k, recent_w=w, gen_len_T=24))
+
+
+def test_shared_key_value_heads_many_splits_and_host_buffers():
+    wl = _wl(batch=1, head_dim=128, n_heads=8, n_kv_heads=2, prompt_len=2300, budget_k=2100, recent_w=100, gen_len_T=3)
+    lockstep.run_workload(wl, gpu_kwargs=dict(decode_splits=17))
+    a, b = lockstep.make_gpu(wl), lockstep.make_gpu(wl)
+    Q, K, V = W.make_prompt(wl, 0, DEV)
+    a.kf_prefill_score_prune(0, Q, K, V)
+    b.kf_prefill_score_prune(0, Q, K, V)
+    for s in range(1, 4):
+        q, kn, vn = W.make_step(wl, 0, s, DEV)
+        out_a = torch.empty_like(q)
+        a.kf_decode_step(0, s, q, kn, vn, out_a)
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, kn, vn))
+        out_b = torch.empty_like(hq).pin_memory()
+        b.kf_decode_step_host(0, s, hq, hk, hv, out_b, wait=True)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a.cpu(), out_b)
+    lockstep.check_guards(a)
+    lockstep.check_guards(b)

@@ -20,8 +20,9 @@ def _check(wl, units=None):
     gpu.kf_prefill_attend(q, k, v, out)
     assert gpu.kf_poll_error() == 0
     lbh = W.unit_list(wl, 0) if units is None else W.sample_units(wl, units, seed=3, layer=0)
-    flat = torch.as_tensor(lbh[:, 1] * wl.n_heads + lbh[:, 2], dtype=torch.long, device=DEV)
-    rows = lambda t: t.reshape(wl.batch * wl.n_heads, wl.prompt_len, wl.head_dim)[flat].cpu().numpy()
+    flat = torch.as_tensor(lbh[:, 1] * wl.kv_heads + lbh[:, 2], dtype=torch.long, device=DEV)
+    # one entry per cache; tensors with one entry per query head give [U, g, n, d] when g heads share a cache
+    rows = lambda t: t.reshape(wl.batch * wl.kv_heads, -1, wl.prompt_len, wl.head_dim)[flat].squeeze(1).cpu().numpy()
     st = ko.State(lockstep.oracle_params(wl), lbh)
     ref = st.prefill_attend(rows(q), rows(k), rows(v))
     got = rows(out).astype(np.float64)
@@ -73,3 +74,10 @@ def test_attend_and_score_in_one_call_match_the_separate_calls(d, positional):
 def test_prompt_attention_gptj_shape_sampled_units():
     wl = W.get_config("c2_gptj").scaled(n_heads=4, prompt_len=1100, budget_k=512, recent_w=128)
     _check(wl, units=2)
+
+
+@pytest.mark.parametrize("d,g,positional", [(128, 4, "none"), (64, 2, "alibi"), (256, 8, "rotary")])
+def test_prompt_attention_with_shared_key_value_heads(d, g, positional):
+    """g query heads read the keys and values of one cache (section 6: MQA / GQA)."""
+    _check(W.Workload("attend_gqa", 1, 2, 2 * g, d, 333, 100, 10, 0, data_seed=6, positional=positional, rotary_dims=32,
+                      n_kv_heads=2))
