@@ -52,6 +52,11 @@ extern "C" {
 #define KF_PREFILL_TENSOR 0 /* tcgen05 tensor cores, accumulators in tensor memory (default) */
 #define KF_PREFILL_SIMT   1 /* CUDA cores; scores are summed with floating-point atomics     */
 
+/* Which streaming kernel kf_decode_step uses. */
+#define KF_DECODE_AUTO       0 /* tensor cores where several query heads share a cache and head_dim is 128, else CUDA cores */
+#define KF_DECODE_CUDA_CORES 1 /* lane-per-row mixed-precision fma (every shape)                                          */
+#define KF_DECODE_TENSOR     2 /* tcgen05 logits and value sums, accumulators in tensor memory (head_dim 128 only)        */
+
 #define KF_BIAS_NONE  0
 #define KF_BIAS_ALIBI 1     /* x_ij += -slope_h * (i - j); which i and j is chosen by pos_mode */
 
@@ -95,6 +100,7 @@ typedef struct kf_config {
                               accumulates the mean of their scores.  Caches are then per (layer, batch row, key/value
                               head): wherever a shape below says [B][H] for K, V, k_new, v_new, scores, positions or entry
                               counts read [B][Hkv]; q and out stay [B][H].                                         */
+  int32_t decode_impl;     /* KF_DECODE_*                                                                              */
   int32_t debug_canaries;  /* 1: a 256-byte guard of a known pattern follows every sub-buffer of the workspace
                               (kf_workspace_bytes grows accordingly); kf_check_canaries verifies them.  0: none */
   int32_t debug_fail_first_wait; /* self-test of the error path: 1 makes every warp of the generation kernel give up

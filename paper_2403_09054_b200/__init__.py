@@ -4,4 +4,4 @@ from .binding import (Keyformer, KeyformerError, kf_config, make_config, kf_work
                       LIB, LIB_PATH, EXPORTS,
                       KF_OK, KF_EINVAL, KF_ENOSPC, KF_ESTATE, KF_ECUDA, KF_ETIMEOUT, KF_EBOUNDS,
                       KF_NOISE_GUMBEL, KF_NOISE_NONE, KF_NOISE_CONST, KF_NOISE_GAUSS, KF_BIAS_NONE, KF_BIAS_ALIBI, KF_PREFILL_TENSOR, KF_PREFILL_SIMT,
-                      KF_POS_ORIGINAL, KF_POS_NEW)
+                      KF_POS_ORIGINAL, KF_POS_NEW, KF_DECODE_AUTO, KF_DECODE_CUDA_CORES, KF_DECODE_TENSOR)

@@ -52,8 +52,21 @@ bool config_ok(const kf_config* c) {
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
   if (c->n_kv_heads < 0 || c->n_kv_heads > c->n_heads) return false;
   if (c->n_kv_heads > 0 && (c->n_heads % c->n_kv_heads != 0 || !kf::decode_group_supported(c->n_heads / c->n_kv_heads))) return false;
+  if (c->decode_impl < KF_DECODE_AUTO || c->decode_impl > KF_DECODE_TENSOR) return false;
+  if (c->decode_impl == KF_DECODE_TENSOR &&
+      !kf::decode_tc_supported(c->head_dim, c->n_kv_heads > 0 ? c->n_heads / c->n_kv_heads : 1)) return false;
   if (c->debug_canaries < 0 || c->debug_canaries > 1 || c->debug_fail_first_wait < 0 || c->debug_fail_first_wait > 1) return false;
   return true;
+}
+
+// Which streaming kernel the generation step uses: the tensor-core one where it is built (head_dim 128) and pays
+// (several query heads per cache), unless the configuration asks for one of them.
+bool decode_uses_tensor_cores(const kf_config* c) {
+  const int hkv = c->n_kv_heads > 0 ? c->n_kv_heads : c->n_heads;
+  const int group = c->n_heads / hkv;
+  if (c->decode_impl == KF_DECODE_CUDA_CORES) return false;
+  if (c->decode_impl == KF_DECODE_TENSOR) return true;
+  return group >= 2 && kf::decode_tc_supported(c->head_dim, group);
 }
 
 Layout make_layout(const kf_config* c) {
@@ -108,6 +121,10 @@ struct kf_ctx {
   std::vector<int32_t> n_prompt;   // per layer, -1 before prefill
   std::vector<int32_t> last_step;  // per layer
   int64_t launches;
+  // tensor-core generation kernel: TMA maps of every layer's cache (built on first use; they depend on addresses only)
+  bool decode_tc = false;
+  std::vector<CUtensorMap> tmK, tmV;
+  std::vector<char> tm_ready;
   // kf_decode_step_host: copy streams and events (created on first use), two staging sets used alternately
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
   cudaEvent_t in_done[2] = {nullptr, nullptr}, kernel_done[2] = {nullptr, nullptr}, out_done[2] = {nullptr, nullptr};
@@ -141,6 +158,10 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
   ctx->n_prompt.assign(cfg->n_layers, -1);
   ctx->last_step.assign(cfg->n_layers, 0);
   ctx->launches = 0;
+  ctx->decode_tc = decode_uses_tensor_cores(cfg);
+  ctx->tmK.resize(cfg->n_layers);
+  ctx->tmV.resize(cfg->n_layers);
+  ctx->tm_ready.assign(cfg->n_layers, 0);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(ctx->ws + lay.acc, 0, lay.y_scratch - lay.acc, st);  // acc, pos, len
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws + lay.err, 0, lay.slopes - lay.err, st);  // error word
@@ -332,7 +353,15 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.noise_mu = c.noise_mu; P.noise_sigma = c.noise_sigma;
   P.first_wait_limit = c.debug_fail_first_wait ? 0u : kf::DECODE_WAIT_LIMIT;
   P.pk = ctx->pk;
-  if (kf::launch_decode(P, c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+  if (ctx->decode_tc) {
+    if (!ctx->tm_ready[layer]) {
+      if (!kf::decode_tc_cache_maps(&ctx->tmK[layer], &ctx->tmV[layer], P.K, P.V, L.units, c.budget_k, c.head_dim)) return KF_ECUDA;
+      ctx->tm_ready[layer] = 1;
+    }
+    if (kf::launch_decode_tc(P, ctx->tmK[layer], ctx->tmV[layer], c.head_dim, L.units, st) != cudaSuccess) return KF_ECUDA;
+  } else if (kf::launch_decode(P, c.head_dim, L.units, st) != cudaSuccess) {
+    return KF_ECUDA;
+  }
   ctx->launches += 2;   // streaming kernel + closing kernel
   ctx->last_step[layer] = step;
   return KF_OK;
@@ -589,7 +618,7 @@ int kf_describe_decode(const kf_ctx* ctx, char* buf, size_t n) {
   int splits = 1, tps = 4;
   kf::decode_plan(ctx->lay.units, ctx->cfg.budget_k, ctx->cfg.decode_splits, &splits, &tps);
   const int len = kf::decode_describe(buf, n, ctx->cfg.head_dim, ctx->lay.units, ctx->cfg.budget_k, splits, tps,
-                                      ctx->cfg.pos_mode == KF_POS_NEW, ctx->lay.group);
+                                      ctx->cfg.pos_mode == KF_POS_NEW, ctx->lay.group, ctx->decode_tc);
   return len < 0 ? KF_EINVAL : len;
 }
 

@@ -42,14 +42,6 @@ __device__ __forceinline__ void axpy8(float (&o)[8], uint32_t pp, const uint4& v
   }
 }
 
-__device__ __forceinline__ float noise_for(const DecodeParams& P, uint32_t b, uint32_t lh, uint32_t i, uint32_t j) {
-  if (P.noise_mode == 0) return gumbel_from_word(noise_word(P.pk, b, lh, i, j));
-  if (P.noise_mode == 2) return P.noise_const;
-  if (P.noise_mode == 3)
-    return fmaf(P.noise_sigma, gauss_from_words(noise_word(P.pk, b, lh, i, j), noise_word(P.pk, b | GAUSS_PLANE, lh, i, j)), P.noise_mu);
-  return 0.f;
-}
-
 __device__ __forceinline__ unsigned long long evict_key(float a, int pos) {
   // smallest key = smallest accumulated score; equal scores: the higher position leaves
   return ((unsigned long long)__float_as_uint(a) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)pos);
@@ -560,6 +552,22 @@ __global__ void __launch_bounds__(128, G == 1 ? 8 : 4) decode_close_kernel(const
   combine_and_evict<D, 128, G>(P, u, len);
 }
 
+// The closing kernel behind whichever streaming kernel ran, as its programmatic dependent.
+template <int D, int G>
+cudaError_t launch_close(const DecodeParams& P, int units, cudaStream_t stream) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)units);
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_close_kernel<D, G>, P);
+}
+
 template <int D, int NW, int NSTAGE, int G>
 cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   constexpr size_t smem = (size_t)NW * NSTAGE * (TILE_ROWS * D * 2) + (size_t)NW * NSTAGE * 8;
@@ -582,10 +590,7 @@ cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   cfg.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, P);
   if (e != cudaSuccess) return e;
-  cfg.gridDim = dim3((unsigned)units);
-  cfg.blockDim = dim3(128);
-  cfg.dynamicSmemBytes = 0;
-  return cudaLaunchKernelEx(&cfg, decode_close_kernel<D, G>, P);
+  return launch_close<D, G>(P, units, stream);
 }
 
 // One CTA per unit: place[j] = #{i : pos[i] < pos[j]} (positions of a unit are distinct).
@@ -635,7 +640,10 @@ static void decode_variant(int head_dim, int tiles_per_split, int group, int* nw
 }
 
 int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
-                    int group) {
+                    int group, bool tensor_cores) {
+  if (tensor_cores)
+    return snprintf(buf, n, "decode_tc_kernel<%d,%d> + decode_close_kernel<%d,%d>; units=%d k=%d splits=%d tiles_per_split=%d group=%d",
+                    head_dim, group, head_dim, group, units, budget_k, splits, tiles_per_split, group);
   int nw = 4, nstage = 2;
   decode_variant(head_dim, tiles_per_split, group, &nw, &nstage);
   if (group == 1)
@@ -666,6 +674,17 @@ cudaError_t launch_group(const DecodeParams& P, int head_dim, int units, cudaStr
   }
 }
 }  // namespace
+
+cudaError_t launch_decode_close(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
+  if (head_dim != 128) return cudaErrorInvalidValue;   // the tensor-core streaming kernel is built for head_dim 128
+  switch (P.group) {
+    case 1: return launch_close<128, 1>(P, units, stream);
+    case 2: return launch_close<128, 2>(P, units, stream);
+    case 4: return launch_close<128, 4>(P, units, stream);
+    case 8: return launch_close<128, 8>(P, units, stream);
+    default: return cudaErrorInvalidValue;
+  }
+}
 
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
   if (P.splits < 1 || P.splits > MAX_SPLITS) return cudaErrorInvalidValue;

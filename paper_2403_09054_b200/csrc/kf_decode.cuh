@@ -1,6 +1,8 @@
 // Launch interface of the generation-phase kernel (see kf_decode.cu).
 #pragma once
 
+#include <cuda.h>
+
 #include "kf_common.cuh"
 
 namespace kf {
@@ -34,6 +36,17 @@ struct DecodeParams {
 
 constexpr uint32_t DECODE_WAIT_LIMIT = 1u << 22;   // polls of a bounded wait in the generation kernels
 
+#ifdef __CUDACC__
+// zeta of Eq. 4 for logit (query position i, key position j) of (batch b, layer * H + head lh), by adjustment mode.
+__device__ __forceinline__ float noise_for(const DecodeParams& P, uint32_t b, uint32_t lh, uint32_t i, uint32_t j) {
+  if (P.noise_mode == 0) return gumbel_from_word(noise_word(P.pk, b, lh, i, j));
+  if (P.noise_mode == 2) return P.noise_const;
+  if (P.noise_mode == 3)
+    return fmaf(P.noise_sigma, gauss_from_words(noise_word(P.pk, b, lh, i, j), noise_word(P.pk, b | GAUSS_PLANE, lh, i, j)), P.noise_mu);
+  return 0.f;
+}
+#endif
+
 // Size of the built-in scratch block used by kf_decode_step_static (16 MiB per GPU).
 constexpr size_t STATIC_SCRATCH_BYTES = (size_t)16 << 20;
 
@@ -45,7 +58,16 @@ void decode_plan(int units, int budget_k, int requested, int* splits, int* tiles
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 // Names the kernels (with their template arguments) and the split plan of a layer call of this shape; snprintf semantics.
 int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
-                    int group);
+                    int group, bool tensor_cores);
+// Tensor-core streaming kernel for query heads sharing a cache (see kf_decode_tc.cu), followed by the same closing kernel.
+// `tmK`, `tmV`: TMA maps of the layer's cache built by decode_tc_cache_maps (they depend on the cache addresses only).
+bool decode_tc_supported(int head_dim, int group);
+bool decode_tc_cache_maps(CUtensorMap* tmK, CUtensorMap* tmV, const __half* K, const __half* V, int units, int budget_k, int head_dim);
+cudaError_t launch_decode_tc(const DecodeParams& P, const CUtensorMap& tmK, const CUtensorMap& tmV, int head_dim, int units,
+                             cudaStream_t stream);
+
+// Closing kernel alone (merge, normalise, accumulate, evict, replace), behind a streaming kernel launched elsewhere.
+cudaError_t launch_decode_close(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 bool decode_group_supported(int group);   // query heads per key/value head the generation kernels are built for
 
 // Reorders every unit's entries of one layer into ascending position, in place (see kf_compact.cu).  `place` may be

@@ -118,3 +118,9 @@ def test_unsupported_group_sizes_are_rejected():
     cfg = kf.make_config(n_layers=1, batch=1, n_heads=32, n_kv_heads=1, head_dim=64, budget_k=8, recent_w=2,
                          max_prompt_len=16, gen_len_T=4)[0]
     assert kf.kf_workspace_bytes(cfg) == 0              # 32 query heads on one cache: more than the kernels are built for
+
+
+def test_tensor_core_generation_kernel_is_refused_where_it_is_not_built():
+    assert kf.kf_workspace_bytes(_cfg(decode_impl=kf.KF_DECODE_TENSOR)) > 0                 # head_dim 128
+    assert kf.kf_workspace_bytes(_cfg(decode_impl=kf.KF_DECODE_TENSOR, head_dim=64)) == 0
+    assert kf.kf_workspace_bytes(_cfg(decode_impl=3)) == 0

@@ -487,3 +487,72 @@ def test_shared_key_value_heads_many_splits_and_host_buffers():
         assert torch.equal(out_a.cpu(), out_b)
     lockstep.check_guards(a)
     lockstep.check_guards(b)
+
+
+# ------------------------------------------------------------------ tensor-core streaming kernel of the generation step
+@pytest.mark.parametrize("g", [1, 2, 4, 8])
+def test_tensor_core_generation_kernel_in_lock_step(g):
+    """tcgen05 logits and value sums (head_dim 128): several splits, a ragged last tile, items of several tiles."""
+    wl = _wl(head_dim=128, n_heads=2 * g, n_kv_heads=2, prompt_len=900, budget_k=700, recent_w=60, gen_len_T=8)
+    for splits in (0, 1, 2):
+        gpu_kwargs = dict(decode_impl=kf.KF_DECODE_TENSOR, decode_splits=splits)
+        r = lockstep.run_workload(wl, gpu_kwargs=gpu_kwargs)
+        assert r["steps"] == 8
+    gpu = lockstep.make_gpu(wl, decode_impl=kf.KF_DECODE_TENSOR)
+    assert gpu.kf_describe_decode().startswith(f"decode_tc_kernel<128,{g}>")
+    assert lockstep.make_gpu(wl, decode_impl=kf.KF_DECODE_CUDA_CORES).kf_describe_decode().startswith("decode_kernel<128")
+
+
+@pytest.mark.parametrize("pos_mode,noise", [(0, "gumbel"), (1, "gumbel"), (0, "none"), (0, "gauss")])
+def test_tensor_core_generation_kernel_alibi_positions_and_adjustments(pos_mode, noise):
+    wl = W.get_config("c3_mpt").scaled(n_heads=8, n_kv_heads=2, batch=2, prompt_len=500, budget_k=300, recent_w=64, gen_len_T=10)
+    lockstep.run_workload(wl, pos_mode=pos_mode, noise=noise, gpu_kwargs=dict(decode_impl=kf.KF_DECODE_TENSOR))
+
+
+@pytest.mark.parametrize("scale", [1.0, 3.0])
+def test_tensor_core_generation_kernel_moves_its_reference_exponent(scale):
+    """Logits tens of units apart: a later tile of an item exceeds the first tile's maximum by far more than 2^8, so
+    the output accumulator is rescaled in tensor memory (one item of six tiles per cache)."""
+    wl = _wl(head_dim=128, n_heads=4, n_kv_heads=1, batch=3, prompt_len=800, budget_k=700, recent_w=50, gen_len_T=6)
+    lockstep.run_workload(wl, logit_scale=scale, gpu_kwargs=dict(decode_impl=kf.KF_DECODE_TENSOR, decode_splits=1))
+
+
+def test_tensor_core_generation_kernel_ignores_what_lies_beyond_the_entry_count():
+    """A cache that is still filling: the slots past the entry count hold NaN patterns (as uninitialised memory
+    may); they must not leak into the output through a zero weight."""
+    wl = _wl(head_dim=128, n_heads=4, n_kv_heads=2, prompt_len=70, budget_k=200, recent_w=16, gen_len_T=20)
+    gpu = lockstep.make_gpu(wl, decode_impl=kf.KF_DECODE_TENSOR)
+    K, V = gpu.kf_view_state(0)[:2]
+    K.fill_(float("nan"))
+    V.fill_(float("nan"))
+    ls = lockstep.LockStep(wl, gpu, 0, W.unit_list(wl, 0))
+    ls.prefill(*W.make_prompt(wl, 0, DEV))
+    for s in range(1, 21):
+        ls.decode_step(s, *W.make_step(wl, 0, s, DEV))
+    lockstep.check_guards(gpu)
+    gpu.kf_destroy()
+
+
+def test_tensor_core_and_cuda_core_generation_kernels_agree():
+    wl = _wl(head_dim=128, n_heads=8, n_kv_heads=2, prompt_len=600, budget_k=400, recent_w=40, gen_len_T=5)
+    Q, K, V = W.make_prompt(wl, 0, DEV)
+    outs = []
+    for impl in (kf.KF_DECODE_TENSOR, kf.KF_DECODE_CUDA_CORES):
+        gpu = lockstep.make_gpu(wl, decode_impl=impl)
+        gpu.kf_prefill_score_prune(0, Q, K, V)
+        res = []
+        for s in range(1, 6):
+            q, kn, vn = W.make_step(wl, 0, s, DEV)
+            out = torch.empty_like(q)
+            sc = torch.zeros(wl.batch, wl.kv_heads, wl.budget_k + 1, device=DEV)
+            gpu.kf_decode_step(0, s, q, kn, vn, out, score_out=sc)
+            res.append((out, sc))
+        torch.cuda.synchronize()
+        res.append(tuple(t.clone() for t in gpu.kf_view_state(0)[2:]))
+        lockstep.check_guards(gpu)
+        outs.append(res)
+    for (oa, sa), (ob, sb) in zip(outs[0][:5], outs[1][:5]):
+        scale = ob.float().abs().amax(dim=-1, keepdim=True)
+        assert ((oa.float() - ob.float()).abs() <= 2e-3 * scale).all()
+        assert torch.allclose(sa, sb, rtol=1e-3, atol=1e-7)
+    assert torch.equal(outs[0][5][0], outs[1][5][0])        # the same entries were kept
