@@ -616,7 +616,11 @@ int kf_check_canaries(kf_ctx* ctx, void* stream, int32_t* first_bad) {
 int kf_describe_decode(const kf_ctx* ctx, char* buf, size_t n) {
   if (!ctx || !buf || n == 0) return KF_EINVAL;
   int splits = 1, tps = 4;
-  kf::decode_plan(ctx->lay.units, ctx->cfg.budget_k, ctx->cfg.decode_splits, &splits, &tps);
+  if (ctx->decode_tc) {
+    if (kf::decode_tc_plan(ctx->lay.units, ctx->cfg.budget_k, &tps, &splits) != cudaSuccess) return KF_ECUDA;
+  } else {
+    kf::decode_plan(ctx->lay.units, ctx->cfg.budget_k, ctx->cfg.decode_splits, &splits, &tps);
+  }
   const int len = kf::decode_describe(buf, n, ctx->cfg.head_dim, ctx->lay.units, ctx->cfg.budget_k, splits, tps,
                                       ctx->cfg.pos_mode == KF_POS_NEW, ctx->lay.group, ctx->decode_tc);
   return len < 0 ? KF_EINVAL : len;

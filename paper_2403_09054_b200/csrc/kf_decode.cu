@@ -47,6 +47,76 @@ __device__ __forceinline__ unsigned long long evict_key(float a, int pos) {
   return ((unsigned long long)__float_as_uint(a) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)pos);
 }
 
+// The eviction decision and the replacement, common to every form of the closing stage: `best` / `best_j` are the
+// thread's smallest eviction key (accumulated score, inverted position) among its non-recent entries and its slot,
+// z_new the new token's own score, kn_r / vn_r the thread's columns of the new token's row.
+template <int D, int NT, int CPT>
+__device__ __forceinline__ void evict_and_replace(const DecodeParams& P, int u, int len, unsigned long long best, int best_j,
+                                                  float z_new, const __half (&kn_r)[CPT], const __half (&vn_r)[CPT]) {
+  __shared__ unsigned long long sh_key[NT / 32];
+  __shared__ int sh_j[NT / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int BATCH = 8;
+  float* __restrict__ acc = P.acc + (size_t)u * P.k;
+  int32_t* __restrict__ pos = P.pos + (size_t)u * P.k;
+  const unsigned long long key_new = evict_key(z_new, P.p);
+  int slot;   // where the new token's row goes
+  if (len < P.k) {  // cache not full yet: append
+    slot = len;
+    if (tid == 0) P.len[u] = len + 1;
+  } else {
+    // smallest key over the CTA: warp minimum by shuffles, the owning lane publishes it with its slot
+    const unsigned long long mine = best;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other < best ? other : best;
+    }
+    if (best == ~0ull ? lane == 0 : mine == best) { sh_key[warp] = best; sh_j[warp] = best_j; }   // keys are unique
+    __syncthreads();
+    best = sh_key[0];
+    slot = sh_j[0];
+#pragma unroll
+    for (int wi = 1; wi < NT / 32; ++wi)
+      if (sh_key[wi] < best) { best = sh_key[wi]; slot = sh_j[wi]; }
+    if (P.w == 0 && key_new < best) return;  // the new token itself has the lowest score: it is not stored
+    if (best == ~0ull || slot < 0 || slot >= len) {  // cannot happen for 0 <= w <= k; flag it instead of guessing
+      if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
+      return;
+    }
+  }
+  if (P.place) {
+    // the entries behind the one that leaves move up one place; the new token takes the last place
+    int32_t* __restrict__ place = P.place + (size_t)u * P.k;
+    if (len >= P.k) {
+      const int pos_out = (int)(0xffffffffu - (uint32_t)best);   // the key's low word is 2^32 - 1 - position
+      for (int j0 = tid; j0 < len; j0 += NT * BATCH) {   // loads of a batch first, so that they overlap
+        int pp[BATCH], pl[BATCH];
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+          const int j = j0 + i * NT;
+          pp[i] = j < len ? pos[j] : -1;
+          pl[i] = j < len ? place[j] : 0;
+        }
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+          const int j = j0 + i * NT;
+          if (j != slot && pp[i] > pos_out) place[j] = pl[i] - 1;   // pp = -1 beyond the end never passes
+        }
+      }
+    }
+    if (tid == 0) place[slot] = len < P.k ? len : P.k - 1;
+  }
+  if (tid == 0) { pos[slot] = P.p; acc[slot] = z_new; }
+  __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + slot) * D;
+  __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + slot) * D;
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    const int c = tid + i * NT;
+    if (c < D) { Kr[c] = kn_r[i]; Vr[c] = vn_r[i]; }
+  }
+}
+
 // Closing a unit: merge splits, normalise, accumulate, evict, replace.  Everything that does not depend on the
 // streaming kernel (scores and positions of the entries, the new token's own logit) is requested before
 // `griddepcontrol.wait`, i.e. while the streaming kernel's last CTAs are still running.
@@ -54,8 +124,6 @@ __device__ __forceinline__ unsigned long long evict_key(float a, int pos) {
 // adjusted logits and output row; the score added to f_theta is the mean of the heads' softmaxes (Eq. 11).
 template <int D, int NT, int G>
 __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
-  __shared__ unsigned long long sh_key[NT / 32];
-  __shared__ int sh_j[NT / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int Hkv = P.H / G;
   const uint32_t b = (uint32_t)(u / Hkv), h0 = (uint32_t)(u % Hkv) * G, lh0 = (uint32_t)P.layer * P.H + h0;
@@ -207,63 +275,137 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   for (int g = 0; g < G; ++g) z_new = fmaf(fast_exp2((y_new[g] - my[g]) * LOG2E), inv_ly[g], z_new);
   if (G > 1) z_new *= INV_G;
   if (sc && tid == 0) sc[len] = z_new;
-  const unsigned long long key_new = evict_key(z_new, P.p);
+  evict_and_replace<D, NT, CPT>(P, u, len, best, best_j, z_new, kn_r, vn_r);
+}
 
-  int slot;   // where the new token's row goes
-  if (len < P.k) {  // cache not full yet: append
-    slot = len;
-    if (tid == 0) P.len[u] = len + 1;
-  } else {
-    // smallest key over the CTA: warp minimum by shuffles, the owning lane publishes it with its slot
-    const unsigned long long mine = best;
+// The closing stage for G > 1 query heads on one cache, with NT = 128 * min(G, 4) threads so that the heads are worked on
+// side by side instead of one after the other: warp n merges the split statistics of head n and leaves them in shared
+// memory; then every thread owns one (head, column) of the outputs and a few entries of the score update, all of whose
+// loads are issued together.
+template <int D, int NT, int G>
+__device__ void combine_and_evict_group(const DecodeParams& P, int u, int len) {
+  static_assert(G > 1 && NT >= 32 * G && NT >= D, "one warp per head for the statistics, one thread per column of the new row");
+  __shared__ float sh_mx[G], sh_inv_lx[G], sh_my[G], sh_inv_ly[G], sh_xnew[G], sh_ynew[G];
+  __shared__ float sh_w[G][MAX_SPLITS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Hkv = P.H / G;
+  const uint32_t b = (uint32_t)(u / Hkv), h0 = (uint32_t)(u % Hkv) * G, lh0 = (uint32_t)P.layer * P.H + h0;
+  const __half* q = P.q + (size_t)u * G * D;
+  const __half* kn = P.knew + (size_t)u * D;
+  const __half* vn = P.vnew + (size_t)u * D;
+  constexpr int PSTRIDE = 4 + D;
+  constexpr float INV_G = 1.0f / (float)G;
+  const float* part = P.partials + (size_t)u * P.splits * G * PSTRIDE;   // [split][head][4 + D]
+  float* __restrict__ acc = P.acc + (size_t)u * P.k;
+  int32_t* __restrict__ pos = P.pos + (size_t)u * P.k;
+  const float* __restrict__ ys = P.y_scratch + (size_t)u * G * (P.k + 1);   // [head][k + 1]
+
+  // ---- independent of the streaming kernel
+  constexpr int BATCH = 4;
+  float av[BATCH];
+  int pv[BATCH];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-      best = other < best ? other : best;
-    }
-    if (best == ~0ull ? lane == 0 : mine == best) { sh_key[warp] = best; sh_j[warp] = best_j; }   // keys are unique
-    __syncthreads();
-    best = sh_key[0];
-    slot = sh_j[0];
-#pragma unroll
-    for (int wi = 1; wi < NT / 32; ++wi)
-      if (sh_key[wi] < best) { best = sh_key[wi]; slot = sh_j[wi]; }
-    if (P.w == 0 && key_new < best) return;  // the new token itself has the lowest score: it is not stored
-    if (best == ~0ull || slot < 0 || slot >= len) {  // cannot happen for 0 <= w <= k; flag it instead of guessing
-      if (tid == 0) atomicExch(P.err, ERR_BOUNDS);
-      return;
-    }
+  for (int i = 0; i < BATCH; ++i) {
+    const int j = tid + i * NT;
+    const bool in = j < len;
+    av[i] = in ? acc[j] : 0.f;
+    pv[i] = in ? pos[j] : 0x7fffffff;
   }
-  if (P.place) {
-    // the entries behind the one that leaves move up one place; the new token takes the last place
-    int32_t* __restrict__ place = P.place + (size_t)u * P.k;
-    if (len >= P.k) {
-      const int pos_out = (int)(0xffffffffu - (uint32_t)best);   // the key's low word is 2^32 - 1 - position
-      for (int j0 = tid; j0 < len; j0 += NT * BATCH) {   // loads of a batch first, so that they overlap
-        int pp[BATCH], pl[BATCH];
+  for (int line = tid + (NT * BATCH) / 32; line * 32 < len; line += NT) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(acc + line * 32));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(pos + line * 32));
+  }
+  __half kn_r[1], vn_r[1];
+  kn_r[0] = tid < D ? kn[tid] : __float2half(0.f);
+  vn_r[0] = tid < D ? vn[tid] : __float2half(0.f);
+  float x_new = 0.f, y_new = 0.f;
+  if (warp < G) {   // warp n: head n's logit of the new token against itself
+    float s = 0.f;
+    for (int c = lane; c < D; c += 32) s = fmaf(__half2float(q[warp * D + c]), __half2float(kn[c]), s);
+    x_new = warp_sum(s) * P.scale;  // bias(p, p) = 0
+    if (lane == 0) y_new = (x_new + noise_for(P, b, lh0 + warp, (uint32_t)P.p, (uint32_t)P.p)) * P.inv_tau;
+    y_new = __shfl_sync(0xffffffffu, y_new, 0);
+  }
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the streaming kernel has finished; its writes are visible
+
+  if (warp < G) {
+    const int g = warp;
+    float4 ps0 = make_float4(-INFINITY, 0.f, -INFINITY, 0.f), ps1 = ps0;
+    if (lane < P.splits) ps0 = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)lane * G + g) * PSTRIDE));
+    if (lane + 32 < P.splits) ps1 = __ldcg(reinterpret_cast<const float4*>(part + ((size_t)(lane + 32) * G + g) * PSTRIDE));
+    const float mx = warp_max(fmaxf(x_new, fmaxf(ps0.y > 0.f ? ps0.x : -INFINITY, ps1.y > 0.f ? ps1.x : -INFINITY)));
+    const float my = warp_max(fmaxf(y_new, fmaxf(ps0.w > 0.f ? ps0.z : -INFINITY, ps1.w > 0.f ? ps1.z : -INFINITY)));
+    const float w0 = ps0.y > 0.f ? fast_exp2((ps0.x - mx) * LOG2E) : 0.f;
+    const float w1 = ps1.y > 0.f ? fast_exp2((ps1.x - mx) * LOG2E) : 0.f;
+    const float lx = fmaf(ps0.y, w0, ps1.y * w1);
+    const float ly = (ps0.w > 0.f ? ps0.w * fast_exp2((ps0.z - my) * LOG2E) : 0.f) + (ps1.w > 0.f ? ps1.w * fast_exp2((ps1.z - my) * LOG2E) : 0.f);
+    const float inv_lx = 1.f / (warp_sum(lx) + fast_exp2((x_new - mx) * LOG2E));
+    const float inv_ly = 1.f / (warp_sum(ly) + fast_exp2((y_new - my) * LOG2E));
+    sh_w[g][lane] = w0;
+    sh_w[g][lane + 32] = w1;
+    if (lane == 0) { sh_mx[g] = mx; sh_inv_lx[g] = inv_lx; sh_my[g] = my; sh_inv_ly[g] = inv_ly; sh_xnew[g] = x_new; sh_ynew[g] = y_new; }
+  }
+  __syncthreads();
+
+  // ---- attention outputs (Eq. 1): one (head, column) per thread and round
+  for (int idx = tid; idx < G * D; idx += NT) {
+    const int g = idx / D, c = idx % D;
+    float o = fast_exp2((sh_xnew[g] - sh_mx[g]) * LOG2E) * __half2float(vn[c]);
+    const float* col = part + (size_t)g * PSTRIDE + 4 + c;
+#pragma unroll 8
+    for (int sp = 0; sp < P.splits; ++sp) o = fmaf(__ldcg(col + (size_t)sp * G * PSTRIDE), sh_w[g][sp], o);
+    P.out[((size_t)u * G + g) * D + c] = __float2half_rn(o * sh_inv_lx[g]);
+  }
+
+  // ---- score (Eq. 11; the mean over the group's heads), accumulation and the eviction candidate
+  float my[G], inv_ly[G];
 #pragma unroll
-        for (int i = 0; i < BATCH; ++i) {
-          const int j = j0 + i * NT;
-          pp[i] = j < len ? pos[j] : -1;
-          pl[i] = j < len ? place[j] : 0;
-        }
+  for (int g = 0; g < G; ++g) { my[g] = sh_my[g]; inv_ly[g] = sh_inv_ly[g] * INV_G; }
+  float* __restrict__ sc = P.score_opt ? P.score_opt + (size_t)u * (P.k + 1) : nullptr;
+  unsigned long long best = ~0ull;
+  int best_j = -1;
+  const int cutoff = P.p - P.w;  // entries with pos <= cutoff are outside the recent window
+  for (int j0 = tid; j0 < len; j0 += NT * BATCH) {
+    if (j0 != tid) {
 #pragma unroll
-        for (int i = 0; i < BATCH; ++i) {
-          const int j = j0 + i * NT;
-          if (j != slot && pp[i] > pos_out) place[j] = pl[i] - 1;   // pp = -1 beyond the end never passes
+      for (int i = 0; i < BATCH; ++i) {
+        const int j = j0 + i * NT;
+        const bool in = j < len;
+        av[i] = in ? acc[j] : 0.f;
+        pv[i] = in ? pos[j] : 0x7fffffff;
+      }
+    }
+    float yv[G][BATCH];
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+      for (int i = 0; i < BATCH; ++i) {
+        const int j = j0 + i * NT;
+        yv[g][i] = j < len ? __ldcg(ys + (size_t)g * (P.k + 1) + j) : 0.f;
+      }
+#pragma unroll
+    for (int i = 0; i < BATCH; ++i) {
+      const int j = j0 + i * NT;
+      if (j < len) {
+        float z = 0.f;
+#pragma unroll
+        for (int g = 0; g < G; ++g) z = fmaf(fast_exp2((yv[g][i] - my[g]) * LOG2E), inv_ly[g], z);
+        const float a = av[i] + z;
+        acc[j] = a;
+        if (sc) sc[j] = z;
+        if (pv[i] <= cutoff) {
+          const unsigned long long key = evict_key(a, pv[i]);
+          if (key < best) { best = key; best_j = j; }
         }
       }
     }
-    if (tid == 0) place[slot] = len < P.k ? len : P.k - 1;
   }
-  if (tid == 0) { pos[slot] = P.p; acc[slot] = z_new; }
-  __half* Kr = const_cast<__half*>(P.K) + ((size_t)u * P.k + slot) * D;
-  __half* Vr = const_cast<__half*>(P.V) + ((size_t)u * P.k + slot) * D;
+  float z_new = 0.f;
 #pragma unroll
-  for (int i = 0; i < CPT; ++i) {
-    const int c = tid + i * NT;
-    if (c < D) { Kr[c] = kn_r[i]; Vr[c] = vn_r[i]; }
-  }
+  for (int g = 0; g < G; ++g) z_new = fmaf(fast_exp2((sh_ynew[g] - my[g]) * LOG2E), inv_ly[g], z_new);
+  if (sc && tid == 0) sc[len] = z_new;
+  evict_and_replace<D, NT, 1>(P, u, len, best, best_j, z_new, kn_r, vn_r);
 }
 
 // Warp-wide maximum in one instruction (f32 redux is an sm_100a feature).
@@ -543,13 +685,16 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
 }
 
 // One CTA per unit, launched behind the streaming kernel as its programmatic dependent.
+__host__ __device__ constexpr int close_threads(int d, int g) { return g == 1 ? 128 : (128 * (g < 4 ? g : 4) < d ? d : 128 * (g < 4 ? g : 4)); }
+
 template <int D, int G>
-__global__ void __launch_bounds__(128, G == 1 ? 8 : 4) decode_close_kernel(const __grid_constant__ DecodeParams P) {
+__global__ void __launch_bounds__(close_threads(D, G), G == 1 ? 8 : (G == 8 ? 1 : 2)) decode_close_kernel(const __grid_constant__ DecodeParams P) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // lets the next kernel's CTAs queue up behind this grid
   const int u = blockIdx.x;
   const int len = P.len[u];
   if (len < 0 || len > P.k) return;   // reported by the streaming kernel; nothing of the unit is written
-  combine_and_evict<D, 128, G>(P, u, len);
+  if constexpr (G == 1) combine_and_evict<D, 128, 1>(P, u, len);
+  else combine_and_evict_group<D, close_threads(D, G), G>(P, u, len);
 }
 
 // The closing kernel behind whichever streaming kernel ran, as its programmatic dependent.
@@ -560,7 +705,7 @@ cudaError_t launch_close(const DecodeParams& P, int units, cudaStream_t stream) 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)units);
-  cfg.blockDim = dim3(128);
+  cfg.blockDim = dim3(close_threads(D, G));
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
   cfg.attrs = attr;
@@ -642,8 +787,8 @@ static void decode_variant(int head_dim, int tiles_per_split, int group, int* nw
 int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
                     int group, bool tensor_cores) {
   if (tensor_cores)
-    return snprintf(buf, n, "decode_tc_kernel<%d,%d> + decode_close_kernel<%d,%d>; units=%d k=%d splits=%d tiles_per_split=%d group=%d",
-                    head_dim, group, head_dim, group, units, budget_k, splits, tiles_per_split, group);
+    return snprintf(buf, n, "decode_tc_kernel<%d,%d> + decode_close_kernel<%d,%d>; units=%d k=%d ctas=%d pieces=%d group=%d",
+                    head_dim, group, head_dim, group, units, budget_k, tiles_per_split, splits, group);
   int nw = 4, nstage = 2;
   decode_variant(head_dim, tiles_per_split, group, &nw, &nstage);
   if (group == 1)

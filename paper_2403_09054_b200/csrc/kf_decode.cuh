@@ -57,14 +57,17 @@ int decode_max_splits();
 void decode_plan(int units, int budget_k, int requested, int* splits, int* tiles_per_split);
 cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
 // Names the kernels (with their template arguments) and the split plan of a layer call of this shape; snprintf semantics.
+// For the tensor-core kernel `splits` = partials per cache and `tiles_per_split` = CTAs of the launch.
 int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
                     int group, bool tensor_cores);
 // Tensor-core streaming kernel for query heads sharing a cache (see kf_decode_tc.cu), followed by the same closing kernel.
 // `tmK`, `tmV`: TMA maps of the layer's cache built by decode_tc_cache_maps (they depend on the cache addresses only).
 bool decode_tc_supported(int head_dim, int group);
 bool decode_tc_cache_maps(CUtensorMap* tmK, CUtensorMap* tmV, const __half* K, const __half* V, int units, int budget_k, int head_dim);
-cudaError_t launch_decode_tc(const DecodeParams& P, const CUtensorMap& tmK, const CUtensorMap& tmV, int head_dim, int units,
+cudaError_t launch_decode_tc(DecodeParams P, const CUtensorMap& tmK, const CUtensorMap& tmV, int head_dim, int units,
                              cudaStream_t stream);
+// CTAs of a tensor-core launch and the partials it leaves per cache (needs the current device's SM count).
+cudaError_t decode_tc_plan(int units, int budget_k, int* ctas, int* pieces);
 
 // Closing kernel alone (merge, normalise, accumulate, evict, replace), behind a streaming kernel launched elsewhere.
 cudaError_t launch_decode_close(const DecodeParams& P, int head_dim, int units, cudaStream_t stream);
