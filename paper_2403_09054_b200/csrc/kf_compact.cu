@@ -10,11 +10,11 @@
 // window, slot = place.
 //
 // Two launches.  compact_rank_kernel, one CTA per unit: the rank of every entry among the positions of its unit
-// (counted in shared memory) is its destination slot.  compact_move_kernel, one warp per unit: the permutation is
-// applied cycle by cycle, a row travelling through the registers of the warp (each lane holds 1/32 of a K row and
-// of a V row), so no staging buffer is needed; the rows of the next destinations are requested in batches before
-// any of them is overwritten, so the walk pays one memory latency per batch rather than per row, and a warp
-// per unit keeps enough units resident to fill the memory system.
+// (a sort in shared memory, then a bisection per entry) is its destination slot.  compact_move_kernel, one CTA of eight warps per unit: the
+// permutation is applied cycle by cycle, a row travelling through the registers of a warp (each lane holds 1/32 of a
+// K row and of a V row), so no staging buffer is needed.  Long cycles are cut into segments that the warps walk at
+// the same time (see the kernel), and within a segment the rows of the next destinations are requested in batches
+// before any of them is overwritten, so a walk pays one memory latency per batch rather than per row.
 #include "kf_decode.cuh"
 
 namespace kf {
@@ -22,7 +22,7 @@ namespace kf {
 namespace {
 
 constexpr int CP_THREADS = 256;
-constexpr int CP_MAX_K = 16384;   // one int32 per slot and warp in shared memory
+constexpr int CP_MAX_K = 16384;   // one int32 per slot in shared memory
 __host__ __device__ constexpr int cp_ahead(int d) { return d == 256 ? 8 : 16; }   // rows in flight per warp
 
 template <int D> struct RowPart;   // what one lane holds of a row of D binary16 values
@@ -30,53 +30,88 @@ template <> struct RowPart<64> { using type = uint32_t; };
 template <> struct RowPart<128> { using type = uint2; };
 template <> struct RowPart<256> { using type = uint4; };
 
+// dst[j] = number of the unit's positions smaller than pos[j] (positions of a unit are distinct): the positions are
+// sorted in shared memory (bitonic network, padded to a power of two with the largest value) and every entry finds
+// its own position in the sorted array by bisection.
 __global__ void __launch_bounds__(CP_THREADS) compact_rank_kernel(const int32_t* __restrict__ pos, const int32_t* __restrict__ len,
-                                                                  int32_t* __restrict__ dst, int k) {
+                                                                  int32_t* __restrict__ dst, int k, int n_pow2) {
   extern __shared__ __align__(16) int32_t cp_smem[];
-  int32_t* spos = cp_smem;
+  int32_t* key = cp_smem;
   const int u = blockIdx.x, tid = threadIdx.x;
   const int n = min(len[u], k);
   const int32_t* pos_u = pos + (size_t)u * k;
-  const int n4 = (n + 3) & ~3;   // padded with the largest value, which counts for nobody
-  for (int j = tid; j < n4; j += CP_THREADS) spos[j] = j < n ? pos_u[j] : 0x7fffffff;
+  int np = 1;
+  while (np < n) np <<= 1;          // the network only has to cover this unit's entries (np <= n_pow2)
+  for (int j = tid; j < np; j += CP_THREADS) key[j] = j < n ? pos_u[j] : 0x7fffffff;
+  for (int size = 2; size <= np; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      __syncthreads();
+      for (int p = tid; p < (np >> 1); p += CP_THREADS) {
+        const int i = ((p & ~(stride - 1)) << 1) | (p & (stride - 1));   // lower index of the pair
+        const int j = i | stride;
+        const bool up = (i & size) == 0;
+        const int a = key[i], b = key[j];
+        if ((a > b) == up) { key[i] = b; key[j] = a; }
+      }
+    }
+  }
   __syncthreads();
   for (int j = tid; j < n; j += CP_THREADS) {
-    const int pj = spos[j];
-    int c = 0;
-    for (int i = 0; i < n4; i += 4) {   // positions of a unit are distinct
-      const int4 q = *reinterpret_cast<const int4*>(spos + i);
-      c += (q.x < pj ? 1 : 0) + (q.y < pj ? 1 : 0) + (q.z < pj ? 1 : 0) + (q.w < pj ? 1 : 0);
+    const int pj = pos_u[j];
+    int lo = 0, hi = n;             // first index whose key is not below pj
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (key[mid] < pj) lo = mid + 1; else hi = mid;
     }
-    dst[(size_t)u * k + j] = c;
+    dst[(size_t)u * k + j] = lo;
   }
+  (void)n_pow2;
 }
 
+// One CTA of CP_WARPS warps per unit.  A cycle of the permutation is cut at "boundary" slots: a segment starts at a
+// boundary slot and follows the cycle up to, and including the write into, the next boundary slot.  In every round
+// the CTA picks up to cp_heads(D) boundary slots among the entries that are not home yet and copies their entries
+// (rows, score, position) into shared memory; after one barrier the segments are independent -- a slot inside a
+// segment is read and written by that segment's warp only, and the boundary slot a segment ends in has been saved --
+// so the warps take segments from a common counter and walk them at the same time, each with the rows of its next
+// destinations requested in batches.  Every cycle that contains a boundary slot is finished in that round.  The first
+// rounds pick boundary slots by a hash of the slot number, so that a long cycle is cut into many segments (a regular
+// choice such as every 64th slot can miss whole cycles of a regular permutation, e.g. the shift by two that two
+// evictions leave behind); the later rounds take whatever is left, until every entry is home.
+constexpr int CP_WARPS = 8;
+constexpr int CP_FLAG = 1 << 30;   // marks a boundary slot in the shared-memory copy of the permutation
+__host__ __device__ constexpr int cp_heads(int d) { return d == 256 ? 32 : 64; }   // boundary slots per round (32 KB of rows)
+
 template <int D>
-__global__ void compact_move_kernel(__half* __restrict__ K, __half* __restrict__ V, float* __restrict__ acc,
-                                    int32_t* __restrict__ pos, const int32_t* __restrict__ len,
-                                    const int32_t* __restrict__ dst, int32_t* __restrict__ place, int k, int units) {
+__global__ void __launch_bounds__(CP_WARPS * 32, 2) compact_move_kernel(__half* __restrict__ K, __half* __restrict__ V, float* __restrict__ acc,
+                                                                        int32_t* __restrict__ pos, const int32_t* __restrict__ len,
+                                                                        const int32_t* __restrict__ dst, int32_t* __restrict__ place, int k) {
   using Part = typename RowPart<D>::type;
   constexpr int CP_AHEAD = cp_ahead(D);
+  constexpr int NH = cp_heads(D);
   extern __shared__ __align__(16) int32_t cp_smem[];
+  Part* head_k = reinterpret_cast<Part*>(cp_smem);          // [NH][32] the boundary entries' K rows, one part per lane
+  Part* head_v = head_k + NH * 32;
+  float* head_a = reinterpret_cast<float*>(head_v + NH * 32);
+  int32_t* head_p = reinterpret_cast<int32_t*>(head_a + NH);
+  int32_t* head_t = head_p + NH;                            // where the boundary entry has to go
+  int32_t* head_b = head_t + NH;                            // the boundary slot itself
+  int32_t* sdst = head_b + NH;   // [k] where the entry in each slot still has to go; s itself once it is home
+  __shared__ int sb_count, sb_next;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int u = blockIdx.x * (blockDim.x >> 5) + warp;
-  if (u >= units) return;
-  int32_t* sdst = cp_smem + (size_t)warp * k;   // where the entry in each slot still has to go; s itself once it is home
+  const int u = blockIdx.x;
   const int n = min(len[u], k);
   int32_t* pos_u = pos + (size_t)u * k;
   float* acc_u = acc + (size_t)u * k;
   Part* Ku = reinterpret_cast<Part*>(K + (size_t)u * k * D);
   Part* Vu = reinterpret_cast<Part*>(V + (size_t)u * k * D);
-  for (int j = lane; j < n; j += 32) sdst[j] = dst[(size_t)u * k + j];
-  __syncwarp();
+  for (int j = threadIdx.x; j < n; j += CP_WARPS * 32) sdst[j] = dst[(size_t)u * k + j];
+  const uint32_t n_buckets = (uint32_t)max(1, n / (NH * 3 / 4));   // a hashed round expects 3/4 of the head buffer
+  const int hashed_rounds = max(1, min(8, n / (NH * 12)));          // in all about one slot in sixteen, spread by the hash
 
-  // The entry in slot j goes to slot sdst[j].  Every lane walks the same way, so there is no divergence.
-  for (int s = 0; s < n; ++s) {
-    if (sdst[s] == s) continue;
-    Part ck = Ku[(size_t)s * 32 + lane], cv = Vu[(size_t)s * 32 + lane];
-    float ca = acc_u[s];
-    int cp = pos_u[s];
-    int t = sdst[s];        // destination of the travelling entry
+  // Walks from the entry (ck, cv, ca, cp) that has to go to slot t: writes it there, picks up what was there, and so on,
+  // until the walk has written into a boundary slot (whose entry is in the head buffer).
+  auto walk = [&](int t, Part ck, Part cv, float ca, int cp) {
     bool done = false;
     while (!done) {
       int tt[CP_AHEAD];
@@ -89,13 +124,15 @@ __global__ void compact_move_kernel(__half* __restrict__ K, __half* __restrict__
         if (!done) {
           tt[i] = t;
           cnt = i + 1;
-          if (t == s) done = true;        // the cycle closes at its first slot, whose entry already travels
-          else t = sdst[t];
+          const int v = sdst[t];
+          if (v & CP_FLAG) done = true;
+          else t = v;
         }
       }
+      const int last = done ? cnt - 1 : cnt;   // the slot the walk ends in is written but not picked up
 #pragma unroll
       for (int i = 0; i < CP_AHEAD; ++i) {
-        if (i < cnt && tt[i] != s) {
+        if (i < last) {
           rk[i] = Ku[(size_t)tt[i] * 32 + lane];
           rv[i] = Vu[(size_t)tt[i] * 32 + lane];
           ra[i] = acc_u[tt[i]];
@@ -109,15 +146,51 @@ __global__ void compact_move_kernel(__half* __restrict__ K, __half* __restrict__
           Ku[(size_t)tt[i] * 32 + lane] = ck;
           Vu[(size_t)tt[i] * 32 + lane] = cv;
           if (lane == 0) { pos_u[tt[i]] = cp; acc_u[tt[i]] = ca; sdst[tt[i]] = tt[i]; }
-          if (tt[i] != s) { ck = rk[i]; cv = rv[i]; ca = ra[i]; cp = rp[i]; }
+          if (i < last) { ck = rk[i]; cv = rv[i]; ca = ra[i]; cp = rp[i]; }
         }
       }
       __syncwarp();
     }
+  };
+
+  for (int r = 0;; ++r) {
+    // ---- this round's boundary slots among the entries that are not home yet
+    if (threadIdx.x == 0) { sb_count = 0; sb_next = 0; }
+    __syncthreads();
+    const bool hashed = r < hashed_rounds;
+    for (int j = threadIdx.x; j < n; j += CP_WARPS * 32) {
+      if (sdst[j] != j && (!hashed || ((uint32_t)j * 0x9E3779B1u >> 8) % n_buckets == (uint32_t)r)) {
+        const int at = atomicAdd(&sb_count, 1);
+        if (at < NH) { head_b[at] = j; head_t[at] = sdst[j]; sdst[j] |= CP_FLAG; }
+      }
+    }
+    __syncthreads();
+    const int nb = min(sb_count, NH);   // (every thread reads the same count)
+    if (nb == 0) {
+      if (hashed) continue;
+      break;       // an unrestricted round found nothing: every entry is home
+    }
+    // ---- their entries into shared memory, before anything is overwritten
+    for (int i = warp; i < nb; i += CP_WARPS) {
+      const int b = head_b[i];
+      head_k[i * 32 + lane] = Ku[(size_t)b * 32 + lane];
+      head_v[i * 32 + lane] = Vu[(size_t)b * 32 + lane];
+      if (lane == 0) { head_a[i] = acc_u[b]; head_p[i] = pos_u[b]; }
+    }
+    __syncthreads();
+    // ---- the segments, first come first served
+    for (;;) {
+      int i = 0;
+      if (lane == 0) i = atomicAdd(&sb_next, 1);
+      i = __shfl_sync(0xffffffffu, i, 0);
+      if (i >= nb) break;
+      walk(head_t[i], head_k[i * 32 + lane], head_v[i * 32 + lane], head_a[i], head_p[i]);
+    }
+    __syncthreads();
   }
   if (place) {
     int32_t* place_u = place + (size_t)u * k;
-    for (int j = lane; j < n; j += 32) place_u[j] = j;
+    for (int j = threadIdx.x; j < n; j += CP_WARPS * 32) place_u[j] = j;
   }
 }
 
@@ -128,21 +201,23 @@ int compact_max_k() { return CP_MAX_K; }
 cudaError_t launch_compact(__half* K, __half* V, float* acc, int32_t* pos, const int32_t* len, int32_t* place,
                            int32_t* dst_scratch, int k, int head_dim, int units, cudaStream_t stream) {
   if (k < 1 || k > CP_MAX_K || units < 1 || !dst_scratch) return cudaErrorInvalidValue;
-  const size_t smem_rank = (size_t)((k + 3) & ~3) * 4;
+  int n_pow2 = 1;
+  while (n_pow2 < k) n_pow2 <<= 1;
+  const size_t smem_rank = (size_t)n_pow2 * 4;
   cudaError_t e = cudaSuccess;
   if (smem_rank > 48 * 1024) e = cudaFuncSetAttribute(compact_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_rank);
   if (e != cudaSuccess) return e;
-  compact_rank_kernel<<<units, CP_THREADS, smem_rank, stream>>>(pos, len, dst_scratch, k);
+  compact_rank_kernel<<<units, CP_THREADS, smem_rank, stream>>>(pos, len, dst_scratch, k, n_pow2);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const int wpc = k <= 4096 ? 4 : 1;                // warps (units) per CTA: at most 64 KB of destinations per CTA
-  const size_t smem = (size_t)wpc * k * 4;
+  // the head buffer (rows, scores, positions, destinations, slots of a round's boundary entries), then one destination per slot
+  const size_t smem = (size_t)cp_heads(head_dim) * ((size_t)head_dim * 4 + 16) + (size_t)k * 4;
   auto go = [&](auto kern) -> cudaError_t {
     if (smem > 48 * 1024) {
       cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e2 != cudaSuccess) return e2;
     }
-    kern<<<(units + wpc - 1) / wpc, wpc * 32, smem, stream>>>(K, V, acc, pos, len, dst_scratch, place, k, units);
+    kern<<<units, CP_WARPS * 32, smem, stream>>>(K, V, acc, pos, len, dst_scratch, place, k);
     return cudaGetLastError();
   };
   switch (head_dim) {
