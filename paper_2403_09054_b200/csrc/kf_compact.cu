@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(CP_THREADS) compact_rank_kernel(const int32_t*
   (void)n_pow2;
 }
 
-// One CTA of CP_WARPS warps per unit.  A cycle of the permutation is cut at "boundary" slots: a segment starts at a
+// One CTA of CP_WARPS (8 or 16) warps per unit.  A cycle of the permutation is cut at "boundary" slots: a segment starts at a
 // boundary slot and follows the cycle up to, and including the write into, the next boundary slot.  In every round
 // the CTA picks up to cp_heads(D) boundary slots among the entries that are not home yet and copies their entries
 // (rows, score, position) into shared memory; after one barrier the segments are independent -- a slot inside a
@@ -78,12 +78,12 @@ __global__ void __launch_bounds__(CP_THREADS) compact_rank_kernel(const int32_t*
 // rounds pick boundary slots by a hash of the slot number, so that a long cycle is cut into many segments (a regular
 // choice such as every 64th slot can miss whole cycles of a regular permutation, e.g. the shift by two that two
 // evictions leave behind); the later rounds take whatever is left, until every entry is home.
-constexpr int CP_WARPS = 8;
 constexpr int CP_FLAG = 1 << 30;   // marks a boundary slot in the shared-memory copy of the permutation
 __host__ __device__ constexpr int cp_heads(int d) { return d == 256 ? 32 : 64; }   // boundary slots per round (32 KB of rows)
 
-template <int D>
-__global__ void __launch_bounds__(CP_WARPS * 32, 2) compact_move_kernel(__half* __restrict__ K, __half* __restrict__ V, float* __restrict__ acc,
+// CP_WARPS = 8 with two CTAs per SM when there are units enough to fill the SMs twice over, 16 otherwise.
+template <int D, int CP_WARPS>
+__global__ void __launch_bounds__(CP_WARPS * 32, CP_WARPS == 8 ? 2 : 1) compact_move_kernel(__half* __restrict__ K, __half* __restrict__ V, float* __restrict__ acc,
                                                                         int32_t* __restrict__ pos, const int32_t* __restrict__ len,
                                                                         const int32_t* __restrict__ dst, int32_t* __restrict__ place, int k) {
   using Part = typename RowPart<D>::type;
@@ -212,18 +212,19 @@ cudaError_t launch_compact(__half* K, __half* V, float* acc, int32_t* pos, const
   if (e != cudaSuccess) return e;
   // the head buffer (rows, scores, positions, destinations, slots of a round's boundary entries), then one destination per slot
   const size_t smem = (size_t)cp_heads(head_dim) * ((size_t)head_dim * 4 + 16) + (size_t)k * 4;
+  const bool many = units >= 2 * 148;
   auto go = [&](auto kern) -> cudaError_t {
     if (smem > 48 * 1024) {
       cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e2 != cudaSuccess) return e2;
     }
-    kern<<<units, CP_WARPS * 32, smem, stream>>>(K, V, acc, pos, len, dst_scratch, place, k);
+    kern<<<units, many ? 256 : 512, smem, stream>>>(K, V, acc, pos, len, dst_scratch, place, k);
     return cudaGetLastError();
   };
   switch (head_dim) {
-    case 64: return go(compact_move_kernel<64>);
-    case 128: return go(compact_move_kernel<128>);
-    case 256: return go(compact_move_kernel<256>);
+    case 64: return many ? go(compact_move_kernel<64, 8>) : go(compact_move_kernel<64, 16>);
+    case 128: return many ? go(compact_move_kernel<128, 8>) : go(compact_move_kernel<128, 16>);
+    case 256: return many ? go(compact_move_kernel<256, 8>) : go(compact_move_kernel<256, 16>);
     default: return cudaErrorInvalidValue;
   }
 }
