@@ -278,13 +278,13 @@ __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
   evict_and_replace<D, NT, CPT>(P, u, len, best, best_j, z_new, kn_r, vn_r);
 }
 
-// The closing stage for G > 1 query heads on one cache, with NT = 128 * min(G, 4) threads so that the heads are worked on
-// side by side instead of one after the other: warp n merges the split statistics of head n and leaves them in shared
+// The closing stage with many threads per unit (NT = 128 * min(G, 4) for G > 1 query heads on one cache, so that the heads are
+// worked on side by side instead of one after the other; 512 for a single head with a long cache and few units): warp n merges the split statistics of head n and leaves them in shared
 // memory; then every thread owns one (head, column) of the outputs and a few entries of the score update, all of whose
 // loads are issued together.
 template <int D, int NT, int G>
 __device__ void combine_and_evict_group(const DecodeParams& P, int u, int len) {
-  static_assert(G > 1 && NT >= 32 * G && NT >= D, "one warp per head for the statistics, one thread per column of the new row");
+  static_assert(NT >= 32 * G && NT >= D, "one warp per head for the statistics, one thread per column of the new row");
   __shared__ float sh_mx[G], sh_inv_lx[G], sh_my[G], sh_inv_ly[G], sh_xnew[G], sh_ynew[G];
   __shared__ float sh_w[G][MAX_SPLITS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -685,7 +685,19 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
 }
 
 // One CTA per unit, launched behind the streaming kernel as its programmatic dependent.
+inline bool close_is_wide(int units, int k) { return units <= 148 && k >= 2048; }
 __host__ __device__ constexpr int close_threads(int d, int g) { return g == 1 ? 128 : (128 * (g < 4 ? g : 4) < d ? d : 128 * (g < 4 ? g : 4)); }
+
+// Few units with long caches (one layer of a long-context model): 128 threads would walk a unit's thousands of entries
+// in several dependent rounds while most SMs idle; 512 threads take them in one.
+template <int D>
+__global__ void __launch_bounds__(512, 1) decode_close_wide_kernel(const __grid_constant__ DecodeParams P) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int u = blockIdx.x;
+  const int len = P.len[u];
+  if (len < 0 || len > P.k) return;
+  combine_and_evict_group<D, 512, 1>(P, u, len);
+}
 
 template <int D, int G>
 __global__ void __launch_bounds__(close_threads(D, G), G == 1 ? 8 : (G == 8 ? 1 : 2)) decode_close_kernel(const __grid_constant__ DecodeParams P) {
@@ -710,6 +722,12 @@ cudaError_t launch_close(const DecodeParams& P, int units, cudaStream_t stream) 
   cfg.stream = stream;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if constexpr (G == 1) {
+    if (close_is_wide(units, P.k)) {
+      cfg.blockDim = dim3(512);
+      return cudaLaunchKernelEx(&cfg, decode_close_wide_kernel<D>, P);
+    }
+  }
   return cudaLaunchKernelEx(&cfg, decode_close_kernel<D, G>, P);
 }
 
@@ -767,7 +785,9 @@ void decode_plan(int units, int budget_k, int requested, int* splits_out, int* t
   const int tiles = (budget_k + TILE_ROWS - 1) / TILE_ROWS;
   int splits = requested;
   if (splits <= 0) {
-    const int target_ctas = 148 * 20;   // about ten waves of the two resident CTAs per SM
+    // many units (inputs larger than L2, bandwidth-bound): about ten waves of the two resident CTAs per SM;
+    // few units (cache-resident, latency-bound): one wave of CTAs that each stream a long run of tiles
+    const int target_ctas = units >= 148 ? 148 * 20 : 148 * 2;
     splits = (target_ctas + units - 1) / units;
   }
   splits = std::max(1, std::min(splits, std::min(MAX_SPLITS, (tiles + 3) / 4)));
@@ -792,8 +812,9 @@ int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, 
   int nw = 4, nstage = 2;
   decode_variant(head_dim, tiles_per_split, group, &nw, &nstage);
   if (group == 1)
-    return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d> + decode_close_kernel<%d>; units=%d k=%d splits=%d tiles_per_split=%d group=1",
-                    head_dim, nw, nstage, new_pos ? 1 : 0, head_dim, units, budget_k, splits, tiles_per_split);
+    return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d> + %s<%d>; units=%d k=%d splits=%d tiles_per_split=%d group=1",
+                    head_dim, nw, nstage, new_pos ? 1 : 0, close_is_wide(units, budget_k) ? "decode_close_wide_kernel" : "decode_close_kernel",
+                    head_dim, units, budget_k, splits, tiles_per_split);
   return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d,%d> + decode_close_kernel<%d,%d>; units=%d k=%d splits=%d tiles_per_split=%d group=%d",
                   head_dim, nw, nstage, new_pos ? 1 : 0, group, head_dim, group, units, budget_k, splits, tiles_per_split, group);
 }
