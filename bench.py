@@ -539,6 +539,49 @@ def run_prefill(args, wl):
         dist.destroy_process_group()
 
 
+def run_compact(args, wl):
+    """Times kf_compact_layer on one layer of the workload after `--scramble-steps` generation steps have left the
+    slots of every unit out of position order.  The state is exported once and imported again before every timed
+    call, so each call sorts the same permutation."""
+    import paper_2403_09054_b200 as kf
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    wl = wl.scaled(n_layers=1)
+    run = DecodeRun(wl, wl, dev, args.scramble_steps)
+    for _ in range(args.scramble_steps):
+        run.device_step()
+    torch.cuda.synchronize()
+    gpu = run.gpu
+    img = torch.empty(gpu.kf_state_bytes(), dtype=torch.uint8, device=dev)
+    n_prompt, last = gpu.kf_export_state(0, img)
+    pos = gpu.kf_view_state(0)[2]
+    displaced = int((pos.argsort(-1).argsort(-1) != torch.arange(pos.shape[-1], device=dev)).sum().item())
+    times = []
+    for _ in range(args.warmup + args.steps):
+        gpu.kf_import_state(0, img, n_prompt, last)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); gpu.kf_compact_layer(0); e1.record(); torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    times = times[args.warmup:]
+    pos = gpu.kf_view_state(0)[2]
+    assert torch.equal(pos, pos.sort(-1).values) and gpu.kf_poll_error() == 0
+    peaks, peak_kind = measured_peaks()
+    ms = statistics.mean(times)
+    moved = displaced * (4 * wl.head_dim + 8) * 2          # every displaced entry read once and written once
+    line = {"metric": "in-place compactions/sec (one layer)", "value": 1e3 / ms, "unit": "calls/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16 rows, int32 positions, f32 scores", "data": "synthetic",
+            "config": shape_config(wl, phase="compact", scramble_steps=args.scramble_steps, displaced_entries=displaced,
+                                   entries=int(pos.numel())),
+            "roofline": {"bound": "hbm", "kernel": "compact_rank_kernel + compact_move_kernel", "achieved": moved / (ms * 1e-3) / 1e9,
+                         "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s",
+                         "frac": moved / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "bytes_per_launch": moved, "traffic": None},
+            "gpu_launches": 2 * args.steps}
+    print(json.dumps(line))
+    run.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -558,8 +601,10 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="decode phase: record the timed steps into one CUDA graph and replay it once (takes the host's "
                          "launch cost out of the small, latency-bound workloads)")
-    ap.add_argument("--phase", default="decode", choices=["decode", "prefill"],
-                    help="decode: the generation step (the headline metric); prefill: the prompt phase of one layer")
+    ap.add_argument("--phase", default="decode", choices=["decode", "prefill", "compact"],
+                    help="decode: the generation step (the headline metric); prefill: the prompt phase of one layer; "
+                         "compact: kf_compact_layer on one layer")
+    ap.add_argument("--scramble-steps", type=int, default=32, help="compact phase: generation steps run before the compaction")
     ap.add_argument("--budget-frac", type=float, default=0.5, help="prefill phase: k as a fraction of the prompt")
     ap.add_argument("--with-attention", action="store_true",
                     help="prefill phase: kf_prefill_attend_score_prune (also produces the prompt's attention output)")
@@ -575,7 +620,9 @@ def main():
         wl = wl.scaled(n_layers=args.layers, name=f"{wl.name}[layers={args.layers}]")
     if args.batch > 0:
         wl = wl.scaled(batch=args.batch, name=f"{wl.name}[batch={args.batch}]")
-    if args.phase == "prefill" and args.impl == "ours":
+    if args.phase == "compact" and args.impl == "ours":
+        run_compact(args, wl)
+    elif args.phase == "prefill" and args.impl == "ours":
         run_prefill(args, wl)
     elif args.impl == "reference":
         run_reference(args, wl)
