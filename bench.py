@@ -47,8 +47,9 @@ def algorithmic_bytes_per_launch(wl: W.Workload) -> int:
 # what kf_describe_decode reports for the launch that was captured.  A launch of any other variant, split plan or
 # shape reports "traffic": null.
 CAPTURED_DECODE_TRAFFIC = {
-    # 1-layer case of the Cerebras-shaped workload (same per-launch shape as the 32-layer one)
-    "decode_kernel<128,5,2,0> + decode_close_kernel<128>; units=1024 k=2048 splits=3 tiles_per_split=24 group=1": 1.124e9,
+    # 1-layer case of the Cerebras-shaped workload (same per-launch shape as the 32-layer one): 1.0825 GB + 13.0 MB
+    # (streaming kernel, read + write) + 27.6 MB (closing kernel)
+    "decode_kernel<128,5,2,0> + decode_close_kernel<128>; units=1024 k=2048 splits=3 tiles_per_split=24 group=1": 1.1228e9,
 }
 
 
