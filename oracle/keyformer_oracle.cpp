@@ -50,6 +50,9 @@ struct ko_params {
   uint64_t noise_seed;
   const double* alibi_slopes;  // [H] or null
   int32_t n_kv_heads;    // key/value heads; H / n_kv_heads query heads share each of them (0 = H: none shared)
+  int32_t rotary_dims;   // R: 0 = the caller's Q/K carry whatever positional rotation the model uses; R > 0 (even, <= d) = they
+                         //    come without it and the rotary embedding of their first R features is applied here
+  double rotary_base;    // 10000 in the published embedding
 };
 
 // Query heads per key/value head (section 6 names multi-query / grouped-query attention as compatible with the
@@ -187,6 +190,30 @@ static double position_bias(const ko_params* P, int32_t h, int32_t i, int32_t j)
   return 0.0;
 }
 
+// Rotary position embedding (Su et al., RoFormer) in the interleaved-pair form GPT-J uses: features (2i, 2i+1), i < R/2,
+// are rotated by the angle pos * base^(-2i/R).  The paper's section 4.4.2 compares feeding a model the original
+// positions of the kept tokens ("Org Pos") with their positions inside the reduced cache ("New Pos") and runs the
+// comparison on rotary models too; for that the cache has to hold keys without rotation and the rotation is applied
+// when a logit is formed.  Reading: in the prompt phase nothing has been dropped, so every token is rotated at its own
+// position in both modes; in the generation phase Org Pos rotates the query at p and key j at its original position,
+// New Pos rotates the query at place m - 1 and the key in place j at j (this list is kept in position order).
+static void rope_row(const ko_params* P, const uint16_t* x, int pos, double* out) {
+  const int d = P->head_dim, R = P->rotary_dims;
+  for (int c = 0; c < d; ++c) out[c] = h2d(x[c]);
+  for (int i = 0; i < R / 2; ++i) {
+    const double theta = std::pow(P->rotary_base, -2.0 * (double)i / (double)R);
+    const double a = (double)pos * theta;
+    const double x0 = out[2 * i], x1 = out[2 * i + 1];
+    out[2 * i] = x0 * std::cos(a) - x1 * std::sin(a);
+    out[2 * i + 1] = x0 * std::sin(a) + x1 * std::cos(a);
+  }
+}
+static double dot_double(const double* a, const double* b, int d) {
+  double s = 0.0;
+  for (int c = 0; c < d; ++c) s += a[c] * b[c];
+  return s;
+}
+
 static double dot_half(const uint16_t* a, const uint16_t* b, int d) {
   double s = 0.0;
   for (int c = 0; c < d; ++c) s += h2d(a[c]) * h2d(b[c]);
@@ -240,14 +267,23 @@ static void prefill_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t
   const int g = group_size(P);
   const double tau = ko_tau(P, 0);
   std::vector<double> y(n), z(n);
+  std::vector<double> Kr, Qr;                                             // rows rotated at their positions (rotary_dims > 0)
+  const bool rot = P->rotary_dims > 0;
+  if (rot) {
+    Kr.resize((size_t)n * d); Qr.resize((size_t)n * d);
+    for (int j = 0; j < n; ++j) rope_row(P, K + (size_t)j * d, j, Kr.data() + (size_t)j * d);
+  }
   for (int j = 0; j < n; ++j) acc_out[j] = 0.0;
   for (int r = 0; r < g; ++r) {
     const int h = hk * g + r;                                             // query head r of this key/value head
     const uint16_t* Qh = Q + (size_t)r * n * d;
+    if (rot) for (int i = 0; i < n; ++i) rope_row(P, Qh + (size_t)i * d, i, Qr.data() + (size_t)i * d);
     for (int i = 0; i < n; ++i) {
       const int m = i + 1;
       for (int j = 0; j < m; ++j) {
-        const double x = P->logit_scale * dot_half(Qh + (size_t)i * d, K + (size_t)j * d, d)
+        const double qk = rot ? dot_double(Qr.data() + (size_t)i * d, Kr.data() + (size_t)j * d, d)
+                              : dot_half(Qh + (size_t)i * d, K + (size_t)j * d, d);
+        const double x = P->logit_scale * qk
                        + position_bias(P, h, i, j);                       // Eq. 4: x
         y[j] = (x + ko_noise(P, b, l, h, i, j)) / tau;                    // Eq. 4 then Eq. 11
       }
@@ -265,14 +301,22 @@ static void prefill_attend_unit(const ko_params* P, int32_t hk, int32_t n,
   const int d = P->head_dim;
   const int g = group_size(P);
   std::vector<double> x(n), p(n);
+  std::vector<double> Kr, qr(d);
+  const bool rot = P->rotary_dims > 0;
+  if (rot) {
+    Kr.resize((size_t)n * d);
+    for (int j = 0; j < n; ++j) rope_row(P, K + (size_t)j * d, j, Kr.data() + (size_t)j * d);
+  }
   for (int r = 0; r < g; ++r) {
     const int h = hk * g + r;
     const uint16_t* Qh = Q + (size_t)r * n * d;
     double* outh = out + (size_t)r * n * d;
     for (int i = 0; i < n; ++i) {
       const int m = i + 1;
+      if (rot) rope_row(P, Qh + (size_t)i * d, i, qr.data());
       for (int j = 0; j < m; ++j)
-        x[j] = P->logit_scale * dot_half(Qh + (size_t)i * d, K + (size_t)j * d, d) + position_bias(P, h, i, j);
+        x[j] = P->logit_scale * (rot ? dot_double(qr.data(), Kr.data() + (size_t)j * d, d)
+                                     : dot_half(Qh + (size_t)i * d, K + (size_t)j * d, d)) + position_bias(P, h, i, j);
       softmax_inplace(x.data(), p.data(), m);
       for (int c = 0; c < d; ++c) {
         double s = 0.0;
@@ -335,14 +379,22 @@ static void decode_score_unit(const ko_params* P, int32_t b, int32_t l, int32_t 
   const int m = len;
   const double tau = ko_tau(P, step);
   std::vector<double> x(m), y(m), a(m), z(m);
+  std::vector<double> Kr, qr(d);
+  const bool rot = P->rotary_dims > 0;
+  if (rot) {   // keys rotated at their original positions (Org Pos) or at their places in the reduced cache (New Pos)
+    Kr.resize((size_t)m * d);
+    for (int j = 0; j < m; ++j) rope_row(P, st_K + (size_t)j * d, P->pos_mode == 1 ? j : st_pos[j], Kr.data() + (size_t)j * d);
+  }
   for (int j = 0; j < m; ++j) z_out[j] = 0.0;
   for (int r = 0; r < g; ++r) {
     const int h = hk * g + r;                                             // query head r of this key/value head
+    if (rot) rope_row(P, q + (size_t)r * d, P->pos_mode == 1 ? m - 1 : p, qr.data());
     for (int j = 0; j < m; ++j) {
       // "New Pos" (section 4.4.2): the bias sees the entries' places in the reduced cache, which this list
       // keeps in position order, so entry j sits at place j and the current token at place m - 1.
       const double bias = P->pos_mode == 1 ? position_bias(P, h, m - 1, j) : position_bias(P, h, p, st_pos[j]);
-      x[j] = P->logit_scale * dot_half(q + (size_t)r * d, st_K + (size_t)j * d, d) + bias;
+      x[j] = P->logit_scale * (rot ? dot_double(qr.data(), Kr.data() + (size_t)j * d, d)
+                                   : dot_half(q + (size_t)r * d, st_K + (size_t)j * d, d)) + bias;
       y[j] = (x[j] + ko_noise(P, b, l, h, p, st_pos[j])) / tau;
     }
     softmax_inplace(x.data(), a.data(), m);

@@ -42,6 +42,7 @@ class _Params(C.Structure):
         ("tau_init", C.c_double), ("tau_end", C.c_double), ("logit_scale", C.c_double),
         ("noise_const", C.c_double), ("noise_mu", C.c_double), ("noise_sigma", C.c_double),
         ("noise_seed", C.c_uint64), ("alibi_slopes", C.POINTER(C.c_double)), ("n_kv_heads", C.c_int32),
+        ("rotary_dims", C.c_int32), ("rotary_base", C.c_double),
     ]
 
 
@@ -117,6 +118,8 @@ class Params:
     noise_sigma: float = 1.2825
     pos_mode: int = 0                 # 0 original positions in the bias, 1 places within the reduced cache
     n_kv_heads: int = 0               # key/value heads shared by groups of n_heads / n_kv_heads query heads (0 = none shared)
+    rotary_dims: int = 0              # > 0: Q/K come without rotary embedding; it is applied here to their first rotary_dims features
+    rotary_base: float = 10000.0
     _keep: list = field(default_factory=list, repr=False)
 
     @property
@@ -134,6 +137,7 @@ class Params:
         p.noise_const, p.noise_mu, p.noise_sigma = self.noise_const, self.noise_mu, self.noise_sigma
         p.noise_seed = self.noise_seed & 0xFFFFFFFFFFFFFFFF
         p.n_kv_heads = self.n_kv_heads
+        p.rotary_dims, p.rotary_base = self.rotary_dims, self.rotary_base
         if self.alibi_slopes is not None:
             s = np.ascontiguousarray(self.alibi_slopes, dtype=np.float64)
             self._keep.append(s)

