@@ -230,9 +230,9 @@ class DecodeRun:
         import paper_2403_09054_b200 as kf
         self.kf, self.wl, self.dev = kf, wl, dev
         self.gpu = kf.Keyformer(device=dev, n_layers=wl.n_layers, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
-                                n_kv_heads=wl.kv_heads,
+                                n_kv_heads=wl.kv_heads, rotary_dims=wl.rotary_dims if wl.rotary_in_library else 0,
                                 budget_k=wl.budget_k, recent_w=wl.recent_w, max_prompt_len=wl.prompt_len,
-                                gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
+                                gen_len_T=max(wl.gen_len_T, total_steps) if wl.rotary_in_library else wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
                                 bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
                                 alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None,
                                 decode_splits=splits, pos_mode=kf.KF_POS_NEW if new_pos else kf.KF_POS_ORIGINAL)
@@ -612,6 +612,9 @@ def main():
     ap.add_argument("--new-pos", action="store_true",
                     help="decode phase: the bias counts places within the reduced cache (only matters with ALiBi workloads)")
     ap.add_argument("--prefill-simt", action="store_true", help="prefill phase: CUDA-core scoring instead of tcgen05")
+    ap.add_argument("--library-rotary", action="store_true",
+                    help="rotary workloads: pass Q/K unrotated and let the library apply the embedding at logit time "
+                         "(a cache of unrotated keys; combine with --new-pos for positions within the reduced cache)")
     ap.add_argument("--no-extras", dest="extras", action="store_false",
                     help="decode phase: skip the blocks measured after the timed region (the three single-layer workloads, "
                          "the shared-KV-head point and the prompt phase)")
@@ -621,6 +624,8 @@ def main():
         wl = wl.scaled(n_layers=args.layers, name=f"{wl.name}[layers={args.layers}]")
     if args.batch > 0:
         wl = wl.scaled(batch=args.batch, name=f"{wl.name}[batch={args.batch}]")
+    if args.library_rotary:
+        wl = wl.scaled(rotary_in_library=True, name=f"{wl.name}[rotation by the library]")
     if args.phase == "compact" and args.impl == "ours":
         run_compact(args, wl)
     elif args.phase == "prefill" and args.impl == "ours":

@@ -100,6 +100,15 @@ typedef struct kf_config {
                               accumulates the mean of their scores.  Caches are then per (layer, batch row, key/value
                               head): wherever a shape below says [B][H] for K, V, k_new, v_new, scores, positions or entry
                               counts read [B][Hkv]; q and out stay [B][H].                                         */
+  int32_t rotary_dims;     /* R.  0: Q and K carry whatever positional rotation the model applies (the library never looks).
+                              R > 0 (a power of two, 8 <= R <= d): Q and K are passed WITHOUT rotary embedding and the cache
+                              keeps keys unrotated; the library applies the embedding to the first R features (interleaved
+                              pairs (2i, 2i+1), angle position * rotary_base^(-2i/R)) when a logit is formed -- in the prompt
+                              phase at each token's own position, in the generation phase according to pos_mode: KF_POS_ORIGINAL
+                              rotates at the positions in the text, KF_POS_NEW at the places within the reduced cache (section
+                              4.4.2 on rotary models).  Generation then accepts positions below max_prompt_len + max(T, 1)
+                              (KF_EINVAL beyond: the table of angles ends there); not available with KF_DECODE_TENSOR.   */
+  float   rotary_base;     /* > 1 when rotary_dims > 0; 10000 in the published embedding                               */
   int32_t decode_impl;     /* KF_DECODE_*                                                                              */
   int32_t debug_canaries;  /* 1: a 256-byte guard of a known pattern follows every sub-buffer of the workspace
                               (kf_workspace_bytes grows accordingly); kf_check_canaries verifies them.  0: none */

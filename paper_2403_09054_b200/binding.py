@@ -36,7 +36,7 @@ class kf_config(C.Structure):
         ("logit_scale", C.c_float), ("noise_const", C.c_float),
         ("decode_splits", C.c_int32), ("prefill_impl", C.c_int32),
         ("noise_mu", C.c_float), ("noise_sigma", C.c_float), ("pos_mode", C.c_int32),
-        ("n_kv_heads", C.c_int32), ("decode_impl", C.c_int32), ("debug_canaries", C.c_int32), ("debug_fail_first_wait", C.c_int32),
+        ("n_kv_heads", C.c_int32), ("rotary_dims", C.c_int32), ("rotary_base", C.c_float), ("decode_impl", C.c_int32), ("debug_canaries", C.c_int32), ("debug_fail_first_wait", C.c_int32),
     ]
 
 
@@ -126,7 +126,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
                 tau_init=1.0, tau_end=2.0, noise_seed=0, noise_mode=KF_NOISE_GUMBEL, bias_mode=KF_BIAS_NONE,
                 alibi_slopes=None, logit_scale=0.0, noise_const=0.5772, decode_splits=0,
                 prefill_impl=KF_PREFILL_TENSOR, noise_mu=0.5772, noise_sigma=1.2825, pos_mode=KF_POS_ORIGINAL,
-                n_kv_heads=0, decode_impl=0, debug_canaries=0, debug_fail_first_wait=0):
+                n_kv_heads=0, rotary_dims=0, rotary_base=10000.0, decode_impl=0, debug_canaries=0, debug_fail_first_wait=0):
     """Fill a kf_config; returns (config, keepalive) where keepalive holds the slopes array."""
     cfg = kf_config()
     cfg.n_layers, cfg.batch, cfg.n_heads, cfg.head_dim = n_layers, batch, n_heads, head_dim
@@ -143,6 +143,7 @@ def make_config(*, n_layers, batch, n_heads, head_dim, budget_k, recent_w, max_p
     cfg.noise_mu, cfg.noise_sigma = noise_mu, noise_sigma
     cfg.pos_mode = pos_mode
     cfg.n_kv_heads, cfg.decode_impl = n_kv_heads, decode_impl
+    cfg.rotary_dims, cfg.rotary_base = rotary_dims, rotary_base
     cfg.debug_canaries, cfg.debug_fail_first_wait = debug_canaries, debug_fail_first_wait
     return cfg, keep
 

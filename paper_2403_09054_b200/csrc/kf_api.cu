@@ -30,8 +30,11 @@ struct Layout {
   int units, max_splits;               // units = caches of a layer = batch x key/value heads
   int units_q, group;                  // batch x query heads; query heads per key/value head
   size_t acc_q;                        // group > 1 only: prompt scores per query head, before the group mean
+  size_t rope_tab, q_rot, k_rot;       // rotary_dims > 0 only: cos / sin table, rotated copies of the prompt's Q and K
+  int rope_dists;                      // distances the table covers: 0 .. max_prompt_len + max(T, 1) - 1
   // debug_canaries: a guard of GUARD_BYTES follows every sub-buffer; `guards` holds their offsets in layout order
-  // (K, V, acc, pos, len, y_scratch, partials, err, slopes, acc_full, idx, staging, lse2, lse_x, [place], [acc_q])
+  // (K, V, acc, pos, len, y_scratch, partials, err, slopes, acc_full, idx, staging, lse2, lse_x, [place], [acc_q],
+  //  [rotary table, rotated Q, rotated K])
   std::vector<size_t> guards;
 };
 
@@ -52,6 +55,11 @@ bool config_ok(const kf_config* c) {
   if ((int64_t)c->batch * c->n_heads > 65535) return false;  // grid.y limit
   if (c->n_kv_heads < 0 || c->n_kv_heads > c->n_heads) return false;
   if (c->n_kv_heads > 0 && (c->n_heads % c->n_kv_heads != 0 || !kf::decode_group_supported(c->n_heads / c->n_kv_heads))) return false;
+  if (c->rotary_dims < 0 || c->rotary_dims > c->head_dim || (c->rotary_dims & (c->rotary_dims - 1)) != 0 ||
+      (c->rotary_dims > 0 && c->rotary_dims < 8))
+    return false;   // 0, or a power of two from 8 to head_dim
+  if (c->rotary_dims > 0 && !(c->rotary_base > 1.0f)) return false;
+  if (c->rotary_dims > 0 && c->decode_impl == KF_DECODE_TENSOR) return false;   // the tensor-core kernel reads keys as stored
   if (c->decode_impl < KF_DECODE_AUTO || c->decode_impl > KF_DECODE_TENSOR) return false;
   if (c->decode_impl == KF_DECODE_TENSOR &&
       !kf::decode_tc_supported(c->head_dim, c->n_kv_heads > 0 ? c->n_heads / c->n_kv_heads : 1)) return false;
@@ -64,7 +72,7 @@ bool config_ok(const kf_config* c) {
 bool decode_uses_tensor_cores(const kf_config* c) {
   const int hkv = c->n_kv_heads > 0 ? c->n_kv_heads : c->n_heads;
   const int group = c->n_heads / hkv;
-  if (c->decode_impl == KF_DECODE_CUDA_CORES) return false;
+  if (c->decode_impl == KF_DECODE_CUDA_CORES || c->rotary_dims > 0) return false;
   if (c->decode_impl == KF_DECODE_TENSOR) return true;
   return group >= 2 && kf::decode_tc_supported(c->head_dim, group);
 }
@@ -106,6 +114,13 @@ Layout make_layout(const kf_config* c) {
   if (c->pos_mode == KF_POS_NEW) L.place = carve(nl * L.sc_layer);
   L.acc_q = off;
   if (L.group > 1) L.acc_q = carve(align_up(units_q * (size_t)c->max_prompt_len * 4));
+  L.rope_tab = L.q_rot = L.k_rot = off;
+  L.rope_dists = c->max_prompt_len + (c->gen_len_T > 1 ? c->gen_len_T : 1);
+  if (c->rotary_dims > 0) {
+    L.rope_tab = carve(align_up((size_t)L.rope_dists * (c->rotary_dims / 2) * 8));
+    L.q_rot = carve(align_up(units_q * (size_t)c->max_prompt_len * d * 2));
+    L.k_rot = carve(align_up(units * (size_t)c->max_prompt_len * d * 2));
+  }
   L.total = off;
   return L;
 }
@@ -168,6 +183,9 @@ int kf_create(const kf_config* cfg, void* d_workspace, size_t workspace_bytes, v
   if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI)
     e = cudaMemcpyAsync(ctx->ws + lay.slopes, cfg->h_alibi_slopes, (size_t)cfg->n_heads * 4, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess && cfg->bias_mode == KF_BIAS_ALIBI) e = cudaStreamSynchronize(st);  // host array may go away
+  if (e == cudaSuccess && cfg->rotary_dims > 0)
+    e = kf::launch_rope_table(reinterpret_cast<float2*>(ctx->ws + lay.rope_tab), lay.rope_dists, cfg->rotary_dims,
+                              (double)cfg->rotary_base, st);
   for (size_t g = 0; e == cudaSuccess && g < lay.guards.size(); ++g)   // after the clears above, which span some guards
     e = cudaMemsetAsync(ctx->ws + lay.guards[g], GUARD_BYTE, GUARD_BYTES, st);
   if (e != cudaSuccess) { delete ctx; return KF_ECUDA; }
@@ -194,6 +212,19 @@ static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt
   int* err = reinterpret_cast<int*>(ctx->ws + L.err);
   const float* slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   const float inv_tau = (float)(1.0 / (double)c.tau_init);  // the prompt phase is iteration t = 0 of Eq. 12
+  const void* d_k_rows = d_k;   // the cache is filled from the caller's rows (unrotated when the library applies the embedding)
+  if (c.rotary_dims > 0) {
+    // nothing has been dropped yet: every token is rotated at its own position; the scoring kernels read the copies
+    const float2* tab = reinterpret_cast<const float2*>(ctx->ws + L.rope_tab);
+    __half* qr = reinterpret_cast<__half*>(ctx->ws + L.q_rot);
+    __half* kr = reinterpret_cast<__half*>(ctx->ws + L.k_rot);
+    if (kf::launch_rope_rotate(static_cast<const __half*>(d_q), qr, tab, L.units_q, n_prompt, c.head_dim, c.rotary_dims, st) != cudaSuccess ||
+        kf::launch_rope_rotate(static_cast<const __half*>(d_k), kr, tab, L.units, n_prompt, c.head_dim, c.rotary_dims, st) != cudaSuccess)
+      return KF_ECUDA;
+    ctx->launches += 2;
+    d_q = qr;
+    d_k = kr;
+  }
   if (c.prefill_impl == KF_PREFILL_TENSOR) {
     kf::PrefillTcArgs A{};
     A.Q = static_cast<const __half*>(d_q);
@@ -242,7 +273,7 @@ static int prefill_score_prune_impl(kf_ctx* ctx, int32_t layer, int32_t n_prompt
   if (kf::launch_prefill_select(S, L.units, st) != cudaSuccess) return KF_ECUDA;
 
   kf::GatherParams G{};
-  G.K = static_cast<const __half*>(d_k);
+  G.K = static_cast<const __half*>(d_k_rows);
   G.V = static_cast<const __half*>(d_v);
   G.acc_full = acc_full;
   G.idx = S.idx;
@@ -275,6 +306,18 @@ static int prefill_attend_impl(kf_ctx* ctx, int32_t n_prompt, const void* d_q, c
        reinterpret_cast<uintptr_t>(d_out)) & 15u)
     return KF_EINVAL;
   const Layout& L = ctx->lay;
+  if (c.rotary_dims > 0) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float2* tab = reinterpret_cast<const float2*>(ctx->ws + L.rope_tab);
+    __half* qr = reinterpret_cast<__half*>(ctx->ws + L.q_rot);
+    __half* kr = reinterpret_cast<__half*>(ctx->ws + L.k_rot);
+    if (kf::launch_rope_rotate(static_cast<const __half*>(d_q), qr, tab, L.units_q, n_prompt, c.head_dim, c.rotary_dims, st) != cudaSuccess ||
+        kf::launch_rope_rotate(static_cast<const __half*>(d_k), kr, tab, L.units, n_prompt, c.head_dim, c.rotary_dims, st) != cudaSuccess)
+      return KF_ECUDA;
+    ctx->launches += 2;
+    d_q = qr;
+    d_k = kr;
+  }
   kf::PrefillAttendArgs A{};
   A.Q = static_cast<const __half*>(d_q);
   A.K = static_cast<const __half*>(d_k);
@@ -335,6 +378,8 @@ static int decode_impl(kf_ctx* ctx, int32_t layer, int32_t step, const void* d_q
   P.slopes = c.bias_mode == KF_BIAS_ALIBI ? reinterpret_cast<const float*>(ctx->ws + L.slopes) : nullptr;
   P.k = c.budget_k; P.w = c.recent_w;
   P.p = ctx->n_prompt[layer] + step - 1;
+  P.rope_tab = c.rotary_dims > 0 ? reinterpret_cast<const float2*>(ctx->ws + L.rope_tab) : nullptr;
+  P.rot_chunks = c.rotary_dims / 8;
 
   int splits = 1, tps = 4;
   kf::decode_plan(L.units, c.budget_k, c.decode_splits, &splits, &tps);
@@ -372,6 +417,8 @@ static int decode_check(kf_ctx* ctx, int32_t layer, int32_t step) {
   if (layer < 0 || layer >= ctx->cfg.n_layers || step < 1) return KF_EINVAL;
   if (ctx->n_prompt[layer] < 0) return KF_ESTATE;
   if (step != ctx->last_step[layer] + 1) return KF_ESTATE;
+  // with the rotary embedding applied here the table of angles ends at position max_prompt_len + max(T, 1) - 1
+  if (ctx->cfg.rotary_dims > 0 && ctx->n_prompt[layer] + step - 1 >= ctx->lay.rope_dists) return KF_EINVAL;
   return KF_OK;
 }
 
@@ -479,6 +526,7 @@ int kf_decode_step_static(const kf_static_step* a, void* d_K, void* d_V, int32_t
   P.inv_tau = (float)(1.0 / a->tau);
   P.noise_const = a->noise_const;
   P.first_wait_limit = kf::DECODE_WAIT_LIMIT;
+  P.rope_tab = nullptr; P.rot_chunks = 0;
   P.pk = kf::philox_expand_key(a->noise_seed);
   const cudaError_t e = kf::launch_decode_static(P, a->head_dim, units, y_bytes, partial_bytes,
                                                  static_cast<cudaStream_t>(stream));
@@ -622,7 +670,7 @@ int kf_describe_decode(const kf_ctx* ctx, char* buf, size_t n) {
     kf::decode_plan(ctx->lay.units, ctx->cfg.budget_k, ctx->cfg.decode_splits, &splits, &tps);
   }
   const int len = kf::decode_describe(buf, n, ctx->cfg.head_dim, ctx->lay.units, ctx->cfg.budget_k, splits, tps,
-                                      ctx->cfg.pos_mode == KF_POS_NEW, ctx->lay.group, ctx->decode_tc);
+                                      ctx->cfg.pos_mode == KF_POS_NEW, ctx->lay.group, ctx->decode_tc, ctx->cfg.rotary_dims > 0);
   return len < 0 ? KF_EINVAL : len;
 }
 

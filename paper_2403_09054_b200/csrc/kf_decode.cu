@@ -124,7 +124,7 @@ __device__ __forceinline__ void evict_and_replace(const DecodeParams& P, int u, 
 // adjusted logits and output row; the score added to f_theta is the mean of the heads' softmaxes (Eq. 11).
 template <int D, int NT, int G>
 __device__ void combine_and_evict(const DecodeParams& P, int u, int len) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int Hkv = P.H / G;
   const uint32_t b = (uint32_t)(u / Hkv), h0 = (uint32_t)(u % Hkv) * G, lh0 = (uint32_t)P.layer * P.H + h0;
   const __half* q = P.q + (size_t)u * G * D;
@@ -433,7 +433,9 @@ __device__ __forceinline__ void dot8_mixed(float& acc, const uint4& kv, const ui
 
 // G query heads share the unit's cache: every K and V tile is fetched once and used for all G of them
 // (G logits per row, G pairs of running softmaxes, G output rows).
-template <int D, int NW, int NSTAGE, bool NEWPOS, int G>
+// ROT: the cache holds keys without rotary embedding; the logit of a row gets the rotation by the distance between
+// the query and that key (in positions or in places) from a table of cos / sin.
+template <int D, int NW, int NSTAGE, bool NEWPOS, int G, bool ROT>
 __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__ DecodeParams P) {
   constexpr int CPR = D / 8;          // 16-byte chunks per row
   constexpr int LPR = CPR;            // lanes that share one row in the value phase
@@ -571,6 +573,32 @@ __global__ void __launch_bounds__(NW * 32) decode_kernel(const __grid_constant__
       for (int g = 0; g < G; ++g)
         x_mine[g] = ACC == 4 ? (part[g][0] + part[g][1 % ACC]) + (part[g][2 % ACC] + part[g][3 % ACC])
                              : (ACC == 2 ? part[g][0] + part[g][1 % ACC] : part[g][0]);
+      if (ROT) {
+        // The sum above took the rotary features as they are.  With q and k as complex pairs (x_2i + i x_2i+1) the rotated
+        // product of pair i is A c - B s, A + iB = q conj(k), (c, s) = cos / sin(dist theta_i): add A (c - 1) - B s.
+        const int RC = P.rot_chunks;                       // 16-byte chunks (4 pairs) that carry the rotation
+        const float2* tab = P.rope_tab + (size_t)(lane < rows ? dist : 0) * (RC * 4);
+        for (int c = 0; c < RC; ++c) {
+          const int ch = (c + lane) & (RC - 1);            // rotated order: distinct banks within a quarter warp
+          const uint4 kv = *reinterpret_cast<const uint4*>(krow + ch * 16);
+          const float4 t01 = __ldg(reinterpret_cast<const float4*>(tab + ch * 4));
+          const float4 t23 = __ldg(reinterpret_cast<const float4*>(tab + ch * 4 + 2));
+          const float cs[8] = {t01.x, t01.y, t01.z, t01.w, t23.x, t23.y, t23.z, t23.w};
+          const uint32_t kw[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const uint4 qv = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(&sh_q[g][0]) + ch * 16);
+            const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 kf2 = __half22float2(*reinterpret_cast<const __half2*>(&kw[e]));
+              const float2 qf2 = __half22float2(*reinterpret_cast<const __half2*>(&qw[e]));
+              const float A = fmaf(qf2.x, kf2.x, qf2.y * kf2.y), B = fmaf(qf2.y, kf2.x, -qf2.x * kf2.y);
+              x_mine[g] = fmaf(A, cs[2 * e] - 1.0f, fmaf(-B, cs[2 * e + 1], x_mine[g]));
+            }
+          }
+        }
+      }
       __syncwarp();
       consumed = it + 1;
       if (it + NSTAGE < n_items) issue(it + NSTAGE);
@@ -731,10 +759,10 @@ cudaError_t launch_close(const DecodeParams& P, int units, cudaStream_t stream) 
   return cudaLaunchKernelEx(&cfg, decode_close_kernel<D, G>, P);
 }
 
-template <int D, int NW, int NSTAGE, int G>
+template <int D, int NW, int NSTAGE, int G, bool ROT = false>
 cudaError_t launch_one(const DecodeParams& P, int units, cudaStream_t stream) {
   constexpr size_t smem = (size_t)NW * NSTAGE * (TILE_ROWS * D * 2) + (size_t)NW * NSTAGE * 8;
-  auto kern = P.place ? decode_kernel<D, NW, NSTAGE, true, G> : decode_kernel<D, NW, NSTAGE, false, G>;
+  auto kern = P.place ? decode_kernel<D, NW, NSTAGE, true, G, ROT> : decode_kernel<D, NW, NSTAGE, false, G, ROT>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -799,21 +827,21 @@ void decode_plan(int units, int budget_k, int requested, int* splits_out, int* t
 
 // Template arguments <D, NW, NSTAGE> of the streaming kernel launch_decode picks for a shape (one table for the
 // launcher and for kf_describe_decode).
-static void decode_variant(int head_dim, int tiles_per_split, int group, int* nw, int* nstage) {
-  *nw = (head_dim == 128 && tiles_per_split >= 16 && group == 1) ? 5 : 4;
+static void decode_variant(int head_dim, int tiles_per_split, int group, bool rotary, int* nw, int* nstage) {
+  *nw = (head_dim == 128 && tiles_per_split >= 16 && group == 1 && !rotary) ? 5 : 4;
   *nstage = head_dim == 64 ? 4 : 2;
 }
 
 int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
-                    int group, bool tensor_cores) {
+                    int group, bool tensor_cores, bool rotary) {
   if (tensor_cores)
     return snprintf(buf, n, "decode_tc_kernel<%d,%d> + decode_close_kernel<%d,%d>; units=%d k=%d ctas=%d pieces=%d group=%d",
                     head_dim, group, head_dim, group, units, budget_k, tiles_per_split, splits, group);
   int nw = 4, nstage = 2;
-  decode_variant(head_dim, tiles_per_split, group, &nw, &nstage);
+  decode_variant(head_dim, tiles_per_split, group, rotary, &nw, &nstage);
   if (group == 1)
-    return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d> + %s<%d>; units=%d k=%d splits=%d tiles_per_split=%d group=1",
-                    head_dim, nw, nstage, new_pos ? 1 : 0, close_is_wide(units, budget_k) ? "decode_close_wide_kernel" : "decode_close_kernel",
+    return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d%s> + %s<%d>; units=%d k=%d splits=%d tiles_per_split=%d group=1",
+                    head_dim, nw, nstage, new_pos ? 1 : 0, rotary ? ",1,rot" : "", close_is_wide(units, budget_k) ? "decode_close_wide_kernel" : "decode_close_kernel",
                     head_dim, units, budget_k, splits, tiles_per_split);
   return snprintf(buf, n, "decode_kernel<%d,%d,%d,%d,%d> + decode_close_kernel<%d,%d>; units=%d k=%d splits=%d tiles_per_split=%d group=%d",
                   head_dim, nw, nstage, new_pos ? 1 : 0, group, head_dim, group, units, budget_k, splits, tiles_per_split, group);
@@ -825,7 +853,15 @@ namespace {
 template <int G>
 cudaError_t launch_group(const DecodeParams& P, int head_dim, int units, cudaStream_t stream) {
   int nw = 4, nstage = 2;
-  decode_variant(head_dim, P.tiles_per_split, G, &nw, &nstage);
+  decode_variant(head_dim, P.tiles_per_split, G, P.rope_tab != nullptr, &nw, &nstage);
+  if (P.rope_tab) {
+    switch (head_dim) {
+      case 64: return launch_one<64, 4, 4, G, true>(P, units, stream);
+      case 128: return launch_one<128, 4, 2, G, true>(P, units, stream);
+      case 256: return launch_one<256, 4, 2, G, true>(P, units, stream);
+      default: return cudaErrorInvalidValue;
+    }
+  }
   switch (head_dim) {
     case 64: return launch_one<64, 4, 4, G>(P, units, stream);
     case 128:

@@ -24,6 +24,9 @@ struct DecodeParams {
   float* partials;        // [units][splits][group][4 + d]
   int* err;               // device error word
   const float* slopes;    // [H] ALiBi slopes or null
+  const float2* rope_tab; // [distance][rot_chunks * 4] (cos, sin) of distance * theta_i, or null: the rotary embedding is applied
+                          //   to the first rot_chunks * 8 features when a logit is formed (the cache holds unrotated keys)
+  int32_t rot_chunks;     // rotary features / 8 (a power of two), 0 without
   int32_t k, w, p;        // budget, recent window, position of the query token
   int32_t splits, tiles_per_split;
   int32_t H, layer, noise_mode, bias_mode;   // H = query heads
@@ -59,7 +62,7 @@ cudaError_t launch_decode(const DecodeParams& P, int head_dim, int units, cudaSt
 // Names the kernels (with their template arguments) and the split plan of a layer call of this shape; snprintf semantics.
 // For the tensor-core kernel `splits` = partials per cache and `tiles_per_split` = CTAs of the launch.
 int decode_describe(char* buf, size_t n, int head_dim, int units, int budget_k, int splits, int tiles_per_split, bool new_pos,
-                    int group, bool tensor_cores);
+                    int group, bool tensor_cores, bool rotary);
 // Tensor-core streaming kernel for query heads sharing a cache (see kf_decode_tc.cu), followed by the same closing kernel.
 // `tmK`, `tmV`: TMA maps of the layer's cache built by decode_tc_cache_maps (they depend on the cache addresses only).
 bool decode_tc_supported(int head_dim, int group);

@@ -91,6 +91,12 @@ struct PrefillAttendArgs {
 };
 cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int units, cudaStream_t stream);
 
+// Rotary embedding applied by the library (see kf_rope.cu).  `table`: [n_dist][rotary_dims / 2] (cos, sin) of dist * theta_i.
+cudaError_t launch_rope_table(float2* table, int n_dist, int rotary_dims, double base, cudaStream_t stream);
+// dst = src with the first rotary_dims features of row j of every unit ([units][n][head_dim]) rotated at position j.
+cudaError_t launch_rope_rotate(const __half* src, __half* dst, const float2* table, int units, int n, int head_dim, int rotary_dims,
+                               cudaStream_t stream);
+
 size_t prefill_tc_lse_floats(int units, int n_max);
 cudaError_t launch_prefill_score_tc(const PrefillTcArgs& a, int head_dim, int units, cudaStream_t stream);
 cudaError_t launch_prefill_score_simt(const PrefillParams& P, int head_dim, int units, cudaStream_t stream);

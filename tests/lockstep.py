@@ -30,7 +30,7 @@ def oracle_params(wl: W.Workload, noise_mode=ko.NOISE_GUMBEL, logit_scale=0.0, p
     return ko.Params(head_dim=wl.head_dim, n_heads=wl.n_heads, budget_k=wl.budget_k, recent_w=wl.recent_w,
                      gen_len_T=wl.gen_len_T, tau_init=wl.tau_init, tau_end=wl.tau_end,
                      noise_seed=wl.noise_seed, noise_mode=noise_mode, logit_scale=logit_scale, pos_mode=pos_mode,
-                     n_kv_heads=wl.n_kv_heads,
+                     n_kv_heads=wl.n_kv_heads, rotary_dims=wl.rotary_dims if wl.rotary_in_library else 0,
                      bias_mode=1 if wl.positional == "alibi" else 0,
                      alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None)
 
@@ -40,7 +40,7 @@ def make_gpu(wl: W.Workload, noise_mode=kf.KF_NOISE_GUMBEL, max_prompt_len=None,
     (see check_guards): the kernels and their launch shapes are the same with and without them."""
     kw.setdefault("debug_canaries", 1)
     return kf.Keyformer(n_layers=wl.n_layers, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim,
-                        n_kv_heads=wl.n_kv_heads, budget_k=wl.budget_k, recent_w=wl.recent_w,
+                        n_kv_heads=wl.n_kv_heads, rotary_dims=wl.rotary_dims if wl.rotary_in_library else 0, budget_k=wl.budget_k, recent_w=wl.recent_w,
                         max_prompt_len=max_prompt_len or wl.prompt_len, gen_len_T=wl.gen_len_T,
                         tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
                         noise_mode=noise_mode,

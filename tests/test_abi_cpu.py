@@ -124,3 +124,10 @@ def test_tensor_core_generation_kernel_is_refused_where_it_is_not_built():
     assert kf.kf_workspace_bytes(_cfg(decode_impl=kf.KF_DECODE_TENSOR)) > 0                 # head_dim 128
     assert kf.kf_workspace_bytes(_cfg(decode_impl=kf.KF_DECODE_TENSOR, head_dim=64)) == 0
     assert kf.kf_workspace_bytes(_cfg(decode_impl=3)) == 0
+
+
+def test_rotary_configuration_limits():
+    assert kf.kf_workspace_bytes(_cfg(rotary_dims=64)) > kf.kf_workspace_bytes(_cfg())     # table + rotated prompt copies
+    for bad in (dict(rotary_dims=4), dict(rotary_dims=48), dict(rotary_dims=256), dict(rotary_dims=64, rotary_base=1.0),
+                dict(rotary_dims=64, decode_impl=kf.KF_DECODE_TENSOR)):
+        assert kf.kf_workspace_bytes(_cfg(**bad)) == 0

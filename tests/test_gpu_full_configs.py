@@ -28,6 +28,16 @@ def test_config2_gptj_all_units_all_steps():
 
 
 @pytest.mark.parametrize("pos_mode", [0, 1])
+def test_config2_gptj_rotation_applied_by_the_library_all_units_all_steps(pos_mode):
+    """The rotary workload with Q/K passed unrotated and a cache of unrotated keys: original positions, and positions
+    within the reduced cache (section 4.4.2 on a rotary model)."""
+    wl = W.get_config("c2_gptj").scaled(rotary_in_library=True)
+    r = lockstep.run_workload(wl, check_state_every=64, pos_mode=pos_mode)
+    assert r["units"] == 16 and r["steps"] == 256
+    _report("c2_gptj, rotation by the library" + (", new positions" if pos_mode else ""), r)
+
+
+@pytest.mark.parametrize("pos_mode", [0, 1])
 def test_config3_mpt_sampled_units_all_steps(pos_mode):
     """The ALiBi workload at full size for all 512 steps, with original positions in the bias and with the bias
     counted in places of the reduced cache (section 4.4.2)."""

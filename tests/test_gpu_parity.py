@@ -556,3 +556,62 @@ def test_tensor_core_and_cuda_core_generation_kernels_agree():
         assert ((oa.float() - ob.float()).abs() <= 2e-3 * scale).all()
         assert torch.allclose(sa, sb, rtol=1e-3, atol=1e-7)
     assert torch.equal(outs[0][5][0], outs[1][5][0])        # the same entries were kept
+
+
+# ------------------------------------------------------------------ rotary embedding applied by the library (section 4.4.2 on rotary models)
+def _rot_wl(**kw):
+    base = dict(head_dim=128, n_heads=3, prompt_len=300, budget_k=150, recent_w=30, gen_len_T=16, positional="rotary", rotary_dims=64,
+                rotary_in_library=True)
+    base.update(kw)
+    return _wl(**base)
+
+
+@pytest.mark.parametrize("impl", [kf.KF_PREFILL_TENSOR, kf.KF_PREFILL_SIMT])
+@pytest.mark.parametrize("d,R", [(64, 64), (128, 32), (256, 64), (128, 128)])
+@pytest.mark.parametrize("pos_mode", [0, 1])
+def test_rotary_embedding_applied_at_logit_time(pos_mode, d, R, impl):
+    """Q and K come unrotated, the cache keeps keys unrotated; the prompt phase rotates at the tokens' positions, the
+    generation phase at original positions (Org Pos) or at places in the reduced cache (New Pos).  Lock step with the
+    oracle, which rotates in double precision; several splits and evictions."""
+    wl = _rot_wl(head_dim=d, rotary_dims=R)
+    r = lockstep.run_workload(wl, pos_mode=pos_mode, gpu_kwargs=dict(prefill_impl=impl))
+    assert r["steps"] == 16
+
+
+def test_rotary_embedding_with_shared_key_value_heads_and_alibi_free_long_positions():
+    wl = _rot_wl(n_heads=8, n_kv_heads=2, prompt_len=1500, budget_k=400, recent_w=64, gen_len_T=6, rotary_dims=32)
+    for pos_mode in (0, 1):
+        lockstep.run_workload(wl, pos_mode=pos_mode)
+
+
+def test_library_rotation_agrees_with_rotated_inputs_and_keeps_the_cache_unrotated():
+    """Org Pos with the embedding applied by the library is the ordinary rotary model: feeding tensors rotated by the
+    generator (and rounded to fp16) gives the same outputs within that rounding; the cache rows differ (rotated vs not)."""
+    plain = _rot_wl(rotary_in_library=False, gen_len_T=5)
+    inlib = _rot_wl(gen_len_T=5)
+    a, b = lockstep.make_gpu(plain), lockstep.make_gpu(inlib)
+    assert "rot" in b.kf_describe_decode() and "rot" not in a.kf_describe_decode()
+    a.kf_prefill_score_prune(0, *W.make_prompt(plain, 0, DEV))
+    Qu, Ku, Vu = W.make_prompt(inlib, 0, DEV)
+    b.kf_prefill_score_prune(0, Qu, Ku, Vu)
+    for s in range(1, 6):
+        qa, ka, va = W.make_step(plain, 0, s, DEV)
+        qb, kb, vb = W.make_step(inlib, 0, s, DEV)
+        oa, ob = torch.empty_like(qa), torch.empty_like(qb)
+        a.kf_decode_step(0, s, qa, ka, va, oa)
+        b.kf_decode_step(0, s, qb, kb, vb, ob)
+        torch.cuda.synchronize()
+        scale = oa.float().abs().amax(dim=-1, keepdim=True)
+        assert ((oa.float() - ob.float()).abs() <= 1e-2 * scale).all()
+    Kb, _, posb, _, _ = b.kf_view_state(0)
+    torch.cuda.synchronize()
+    rows = Ku.gather(2, posb.clamp(max=inlib.prompt_len - 1).long()[..., None].expand(-1, -1, -1, inlib.head_dim))
+    from_prompt = posb < inlib.prompt_len
+    assert torch.equal(Kb[from_prompt], rows[from_prompt])            # the caller's unrotated rows, bit for bit
+    with pytest.raises(kf.KeyformerError) as e:                        # the table of angles ends at n_max + T - 1
+        for s in range(6, 40):
+            qb, kb, vb = W.make_step(inlib, 0, s, DEV)
+            b.kf_decode_step(0, s, qb, kb, vb, ob)
+    assert e.value.code == kf.KF_EINVAL
+    lockstep.check_guards(a)
+    lockstep.check_guards(b)

@@ -27,6 +27,7 @@ class Workload:
     heavy_frac: float = 0.0        # fraction of key positions that are heavy hitters
     heavy_logit: float = 0.0       # logit shift those keys receive (in units of scaled logits)
     n_kv_heads: int = 0            # key/value heads shared by groups of query heads (0 = one per query head)
+    rotary_in_library: bool = False  # positional == "rotary": leave Q/K unrotated, the consumer applies the embedding itself
 
     @property
     def kv_heads(self) -> int:

@@ -71,7 +71,7 @@ def make_prompt(wl: Workload, layer: int, device="cpu"):
         mask = torch.rand((B, Hkv, n), generator=_gen(wl, layer, "hh_mask", 0, device), device=device) < wl.heavy_frac
         q = q + a * _per_query_head(wl, e)
         k = k + a * e * mask[..., None].to(torch.float32)
-    if wl.positional == "rotary":
+    if wl.positional == "rotary" and not wl.rotary_in_library:
         pos = torch.arange(n, device=device)
         q = _rotary(q, pos, wl.rotary_dims)
         k = _rotary(k, pos, wl.rotary_dims)
@@ -91,7 +91,7 @@ def make_step(wl: Workload, layer: int, step: int, device="cpu", prompt_len: int
         mask = torch.rand((B, Hkv), generator=_gen(wl, layer, "hh_mask", step, device), device=device) < wl.heavy_frac
         q = q + a * _per_query_head(wl, e)
         k = k + a * e * mask[..., None].to(torch.float32)
-    if wl.positional == "rotary":
+    if wl.positional == "rotary" and not wl.rotary_in_library:
         pos = torch.full((1,), n + step - 1, device=device)
         q = _rotary(q, pos, wl.rotary_dims)
         k = _rotary(k, pos, wl.rotary_dims)
