@@ -329,7 +329,12 @@ static int prefill_attend_impl(kf_ctx* ctx, int32_t n_prompt, const void* d_q, c
   A.n = n_prompt; A.H = c.n_heads; A.bias_mode = c.bias_mode;
   A.group = L.group;
   A.scale = ctx->scale;
-  if (kf::launch_prefill_attend(A, c.head_dim, L.units_q, static_cast<cudaStream_t>(stream)) != cudaSuccess) return KF_ECUDA;
+  // one pass over the keys where that kernel is built (head_dim 64, 128); the two-phase kernel otherwise, which can take
+  // the rows' softmax statistics from the scoring sweep
+  const cudaError_t e = (!have_lse_x && kf::prefill_attend_one_pass_supported(c.head_dim))
+                            ? kf::launch_prefill_attend_one_pass(A, c.head_dim, L.units_q, static_cast<cudaStream_t>(stream))
+                            : kf::launch_prefill_attend(A, c.head_dim, L.units_q, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return KF_ECUDA;
   ctx->launches += 1;
   return KF_OK;
 }
@@ -345,7 +350,7 @@ int kf_prefill_attend_score_prune(kf_ctx* ctx, int32_t layer, int32_t n_prompt,
     return KF_EINVAL;
   // with tensor-core scoring the first sweep also produces the rows' plain softmax statistics, so the attention
   // kernel skips its own statistics pass (one Q K^T pass fewer)
-  const bool share = ctx->cfg.prefill_impl == KF_PREFILL_TENSOR;
+  const bool share = ctx->cfg.prefill_impl == KF_PREFILL_TENSOR && !kf::prefill_attend_one_pass_supported(ctx->cfg.head_dim);
   const int rc = prefill_score_prune_impl(ctx, layer, n_prompt, d_q, d_k, d_v, d_score_opt, share, stream);
   if (rc != KF_OK) return rc;
   return prefill_attend_impl(ctx, n_prompt, d_q, d_k, d_v, d_out, share, stream);

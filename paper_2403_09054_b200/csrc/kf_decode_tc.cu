@@ -139,19 +139,6 @@ struct TileCursor {
   }
 };
 
-// Bounded wait for the single-thread roles: polls without sleeping for a while (the hop producer -> MMA -> producer
-// is on the critical path of the memory pipeline), then like wait_bar.
-__device__ __forceinline__ bool wait_bar_eager(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < TC_WAIT_LIMIT; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if (it > 4096) {
-      __nanosleep(40);
-      if ((it & 127u) == 0u && *abort_flag) return false;
-    }
-  }
-  return false;
-}
-
 // G query heads per cache, handled by HG groups of compute warps (HPT = G / HG heads per thread).
 template <int D, int G, int HG, bool GUMBEL>
 __global__ void __launch_bounds__(dt_threads(HG), 1) decode_tc_kernel(const __grid_constant__ DecodeTcParams A) {

@@ -90,6 +90,9 @@ struct PrefillAttendArgs {
   float scale;
 };
 cudaError_t launch_prefill_attend(const PrefillAttendArgs& a, int head_dim, int units, cudaStream_t stream);
+// The same output in one pass over the keys (running maximum, head_dim 64 and 128; see kf_prefill_attend1p.cu); `lse_x` is not used.
+bool prefill_attend_one_pass_supported(int head_dim);
+cudaError_t launch_prefill_attend_one_pass(const PrefillAttendArgs& a, int head_dim, int units, cudaStream_t stream);
 
 // Rotary embedding applied by the library (see kf_rope.cu).  `table`: [n_dist][rotary_dims / 2] (cos, sin) of dist * theta_i.
 cudaError_t launch_rope_table(float2* table, int n_dist, int rotary_dims, double base, cudaStream_t stream);

@@ -107,6 +107,19 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
   return false;
 }
 
+// The same for a single-thread role on the critical path of a pipeline (an MMA issuer): polls without sleeping for a
+// while before it backs off.
+__device__ __forceinline__ bool wait_bar_eager(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < TC_WAIT_LIMIT; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if (it > 4096) {
+      __nanosleep(40);
+      if ((it & 127u) == 0u && *abort_flag) return false;
+    }
+  }
+  return false;
+}
+
 // K-major binary16 operands, binary32 accumulator, M = 128, N = n.
 __host__ __device__ constexpr uint32_t umma_idesc_kk(int n) { return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24); }
 
