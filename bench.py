@@ -513,6 +513,79 @@ def prefill_point(wl, dev, budget_frac, steps, warmup, with_attention=False, sim
     return point
 
 
+def attention_point(wl, dev, steps, warmup, world=1, sampler=None):
+    """Times kf_prefill_attend alone (the prompt's causal attention output, Eq. 1, one pass over the keys on the tensor
+    cores at head_dim 64 / 128).  The roofline is the tensor one: the useful flops of the causal half (QK^T and PV over
+    j <= i) against the measured dense GEMM rate."""
+    import paper_2403_09054_b200 as kf
+    n = wl.prompt_len
+    gpu = kf.Keyformer(device=dev, n_layers=1, batch=wl.batch, n_heads=wl.n_heads, head_dim=wl.head_dim, n_kv_heads=wl.kv_heads,
+                       budget_k=max(1, n // 2), recent_w=max(1, n // 8), max_prompt_len=n, gen_len_T=0,
+                       tau_init=wl.tau_init, tau_end=wl.tau_end, noise_seed=wl.noise_seed,
+                       bias_mode=kf.KF_BIAS_ALIBI if wl.positional == "alibi" else kf.KF_BIAS_NONE,
+                       alibi_slopes=W.alibi_slopes(wl.n_heads) if wl.positional == "alibi" else None)
+    q, k, v = W.make_prompt(wl, 0, dev)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        gpu.kf_prefill_attend(q, k, v, out, stream=stream)
+    barrier(world)
+    launches0 = gpu.kf_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(steps):
+        gpu.kf_prefill_attend(q, k, v, out, stream=stream)
+    e1.record(stream)
+    barrier(world)
+    t1 = time.perf_counter()
+    launches = gpu.kf_launch_count() - launches0
+    ms = e0.elapsed_time(e1) / steps
+    assert gpu.kf_poll_error() == 0
+    gpu.kf_destroy()
+    units = wl.batch * wl.n_heads
+    logits = units * n * (n + 1) // 2
+    flops = 4 * logits * wl.head_dim
+    peaks, kind = measured_peaks()
+    achieved = flops / (ms * 1e-3) / 1e12
+    point = {"workload": wl.name, "prompt": n, "batch": wl.batch, "heads": wl.n_heads, "kv_heads": wl.kv_heads,
+             "head_dim": wl.head_dim, "ms_per_call": ms, "steps": steps, "causal_logits": logits,
+             "roofline": {"bound": "tensor", "kernel": "prefill_attend1p" if wl.head_dim in (64, 128) else "prefill_attend",
+                          "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                          "peak_kind": "%s dense bf16 GEMM, burst (binary16 runs at the same rate)" % kind,
+                          "flops": "4 x causal logits x head_dim (masked halves of the diagonal tiles not counted)",
+                          "traffic": None},
+             "gpu_launches": int(launches)}
+    if sampler is not None:
+        point["clocks"] = sampler.summary(t0, t1)
+    return point
+
+
+def run_attention(args, wl):
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    sampler = ClockSampler(local)
+    sampler.start()
+    pt = attention_point(rank_workload(wl, rank), dev, args.steps, args.warmup, world=world, sampler=sampler)
+    sampler.stop()
+    ms = max_over_ranks(pt["ms_per_call"], world, dev)
+    if rank == 0:
+        line = {"metric": "prompt attention calls/sec (one layer)", "value": world * 1e3 / ms, "unit": "calls/s",
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f16 operands and probabilities, f32 accumulate",
+                "data": "synthetic",
+                "config": {k: pt[k] for k in ("workload", "prompt", "batch", "heads", "kv_heads", "head_dim", "causal_logits")},
+                "roofline": pt["roofline"], "gpu_launches": pt["gpu_launches"], "clocks": pt.get("clocks")}
+        line["config"]["phase"] = "prefill, attention output only"
+        line["config"]["l2"] = "Q, K, V and the output of the call (%.0f MB) exceed L2" % (
+            (2 * pt["heads"] + 2 * pt["kv_heads"]) * pt["batch"] * pt["prompt"] * pt["head_dim"] * 2 / 1e6)
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
 def run_prefill(args, wl):
     rank, world, local = dist_setup(args.gpus)
     dev = torch.device("cuda", local)
@@ -609,6 +682,8 @@ def main():
     ap.add_argument("--budget-frac", type=float, default=0.5, help="prefill phase: k as a fraction of the prompt")
     ap.add_argument("--with-attention", action="store_true",
                     help="prefill phase: kf_prefill_attend_score_prune (also produces the prompt's attention output)")
+    ap.add_argument("--attention-only", action="store_true",
+                    help="prefill phase: kf_prefill_attend alone (the prompt's attention output, no scoring)")
     ap.add_argument("--new-pos", action="store_true",
                     help="decode phase: the bias counts places within the reduced cache (only matters with ALiBi workloads)")
     ap.add_argument("--prefill-simt", action="store_true", help="prefill phase: CUDA-core scoring instead of tcgen05")
@@ -628,6 +703,8 @@ def main():
         wl = wl.scaled(rotary_in_library=True, name=f"{wl.name}[rotation by the library]")
     if args.phase == "compact" and args.impl == "ours":
         run_compact(args, wl)
+    elif args.phase == "prefill" and args.impl == "ours" and args.attention_only:
+        run_attention(args, wl)
     elif args.phase == "prefill" and args.impl == "ours":
         run_prefill(args, wl)
     elif args.impl == "reference":

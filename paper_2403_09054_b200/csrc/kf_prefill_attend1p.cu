@@ -340,7 +340,8 @@ __global__ void __launch_bounds__(A1_THREADS, 1) prefill_attend1p(const __grid_c
           }
           tmem_wait_st();
         }
-        (void)a1_tile_probs<ALIBI, true>(s_addr, A, m_ref, sb, bias_t, lane, quarter, diag, packed, lt);
+        if (diag) (void)a1_tile_probs<ALIBI, true>(s_addr, A, m_ref, sb, bias_t, lane, quarter, true, packed, lt);
+        else (void)a1_tile_probs<ALIBI, false>(s_addr, A, m_ref, sb, bias_t, lane, quarter, false, packed, lt);
       }
       l += lt;
       // P over the first half of S (every logit of the tile has been read by now)
