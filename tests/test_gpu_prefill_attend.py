@@ -13,9 +13,11 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _check(wl, units=None):
+def _check(wl, units=None, edit=None):
     gpu = lockstep.make_gpu(wl)
     q, k, v = W.make_prompt(wl, 0, DEV)
+    if edit is not None:
+        edit(q, k, v)
     out = torch.empty_like(q)
     gpu.kf_prefill_attend(q, k, v, out)
     assert gpu.kf_poll_error() == 0
@@ -38,6 +40,18 @@ def _check(wl, units=None):
 @pytest.mark.parametrize("n", [1, 57, 64, 65, 128, 129, 300, 641])
 def test_prompt_attention_small(n, d):
     _check(W.Workload("attend", 1, 2, 3, d, n, max(1, n // 2), n // 8, 0, data_seed=n + d, noise_seed=1))
+
+
+@pytest.mark.parametrize("d,positional", [(128, "none"), (64, "alibi"), (128, "alibi")])
+def test_prompt_attention_when_late_keys_dwarf_the_early_ones(d, positional):
+    """Keys whose logits lie far above everything before them, first met in the third key tile and again, larger still,
+    in the seventh: a one-pass kernel has to move the rows' reference exponent (and rescale what it has accumulated)
+    in the middle of the walk, twice, and rows that end before a band must not be touched by it."""
+    def edit(q, k, v):
+        k[..., 300:340, :] *= 14.0       # logits of these keys: standard deviation 14 instead of 1
+        k[..., 800:806, :] *= 60.0
+        k[..., 1100:1101, :] *= 0.0      # and a key every row is indifferent to
+    _check(W.Workload("attend_spikes", 1, 2, 3, d, 1200, 300, 40, 0, data_seed=77, noise_seed=1, positional=positional), edit=edit)
 
 
 @pytest.mark.parametrize("positional", ["alibi", "rotary"])
