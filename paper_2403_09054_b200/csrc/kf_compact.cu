@@ -10,7 +10,9 @@
 // window, slot = place.
 //
 // Two launches.  compact_rank_kernel, one CTA per unit: the rank of every entry among the positions of its unit
-// (a sort in shared memory, then a bisection per entry) is its destination slot.  compact_move_kernel, one CTA of eight warps per unit: the
+// (a sort in shared memory, then a bisection per entry) is its destination slot.  compact_move_kernel, one CTA of eight warps per unit:
+// what the generation steps leave behind -- old entries that only have to move down, a few new ones that belong at the
+// end -- is carried over in ascending chunks by the whole CTA (see "the ordered shift" in the kernel); any other
 // permutation is applied cycle by cycle, a row travelling through the registers of a warp (each lane holds 1/32 of a
 // K row and of a V row), so no staging buffer is needed.  Long cycles are cut into segments that the warps walk at
 // the same time (see the kernel), and within a segment the rows of the next destinations are requested in batches
@@ -153,40 +155,110 @@ __global__ void __launch_bounds__(CP_WARPS * 32, CP_WARPS == 8 ? 2 : 1) compact_
     }
   };
 
-  for (int r = 0;; ++r) {
-    // ---- this round's boundary slots among the entries that are not home yet
-    if (threadIdx.x == 0) { sb_count = 0; sb_next = 0; }
+  // ---- The ordered shift: the case the generation steps leave behind.  Entries that were in the cache at the last
+  // compaction have not moved, so they are still in position order and only have to move DOWN past the slots of the
+  // entries that left; the tokens that arrived since sit in those slots and belong at the end.  Whenever the entries
+  // that have to move UP fit the head buffer, they are set aside there, every entry that moves down is carried over in
+  // ascending chunks by the whole CTA (rows of a chunk read, one barrier, rows written: a destination lies below its
+  // source, so what it holds was read in this chunk or an earlier one, or has been set aside), and the entries set
+  // aside are written last.  No cycle is followed and no load waits for another.  Any other permutation (an imported
+  // state, say) goes through the rounds below.
+  bool shifted = false;
+  {
+    constexpr int R = D == 256 ? 4 : 8;   // rows a warp carries per chunk
+    if (threadIdx.x == 0) sb_count = 0;
     __syncthreads();
-    const bool hashed = r < hashed_rounds;
     for (int j = threadIdx.x; j < n; j += CP_WARPS * 32) {
-      if (sdst[j] != j && (!hashed || ((uint32_t)j * 0x9E3779B1u >> 8) % n_buckets == (uint32_t)r)) {
+      const int t = sdst[j];
+      if (t > j) {
         const int at = atomicAdd(&sb_count, 1);
-        if (at < NH) { head_b[at] = j; head_t[at] = sdst[j]; sdst[j] |= CP_FLAG; }
+        if (at < NH) { head_b[at] = j; head_t[at] = t; }
       }
     }
     __syncthreads();
-    const int nb = min(sb_count, NH);   // (every thread reads the same count)
-    if (nb == 0) {
-      if (hashed) continue;
-      break;       // an unrestricted round found nothing: every entry is home
+    const int nup = sb_count;             // (every thread reads the same count)
+    if (nup <= NH) {
+      shifted = true;
+      for (int i = warp; i < nup; i += CP_WARPS) {
+        const int b = head_b[i];
+        head_k[i * 32 + lane] = Ku[(size_t)b * 32 + lane];
+        head_v[i * 32 + lane] = Vu[(size_t)b * 32 + lane];
+        if (lane == 0) { head_a[i] = acc_u[b]; head_p[i] = pos_u[b]; }
+      }
+      __syncthreads();
+      for (int c0 = 0; c0 < n; c0 += CP_WARPS * R) {
+        int tt[R];
+        Part rk[R], rv[R];
+        float ra[R];
+        int rp[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+          const int sl = c0 + warp * R + i;
+          const int t = sl < n ? sdst[sl] : sl;
+          tt[i] = t < sl ? t : -1;
+          if (tt[i] >= 0) {
+            rk[i] = Ku[(size_t)sl * 32 + lane];
+            rv[i] = Vu[(size_t)sl * 32 + lane];
+            ra[i] = acc_u[sl];
+            rp[i] = pos_u[sl];
+          }
+        }
+        __syncthreads();   // every row of the chunk is in registers before any slot of it is overwritten
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+          if (tt[i] >= 0) {
+            Ku[(size_t)tt[i] * 32 + lane] = rk[i];
+            Vu[(size_t)tt[i] * 32 + lane] = rv[i];
+            if (lane == 0) { pos_u[tt[i]] = rp[i]; acc_u[tt[i]] = ra[i]; }
+          }
+        }
+      }
+      __syncthreads();
+      for (int i = warp; i < nup; i += CP_WARPS) {
+        const int t = head_t[i];
+        Ku[(size_t)t * 32 + lane] = head_k[i * 32 + lane];
+        Vu[(size_t)t * 32 + lane] = head_v[i * 32 + lane];
+        if (lane == 0) { pos_u[t] = head_p[i]; acc_u[t] = head_a[i]; }
+      }
     }
-    // ---- their entries into shared memory, before anything is overwritten
-    for (int i = warp; i < nb; i += CP_WARPS) {
-      const int b = head_b[i];
-      head_k[i * 32 + lane] = Ku[(size_t)b * 32 + lane];
-      head_v[i * 32 + lane] = Vu[(size_t)b * 32 + lane];
-      if (lane == 0) { head_a[i] = acc_u[b]; head_p[i] = pos_u[b]; }
+  }
+
+  if (!shifted) {
+    for (int r = 0;; ++r) {
+      // ---- this round's boundary slots among the entries that are not home yet
+      if (threadIdx.x == 0) { sb_count = 0; sb_next = 0; }
+      __syncthreads();
+      const bool hashed = r < hashed_rounds;
+      for (int j = threadIdx.x; j < n; j += CP_WARPS * 32) {
+        if (sdst[j] != j && (!hashed || ((uint32_t)j * 0x9E3779B1u >> 8) % n_buckets == (uint32_t)r)) {
+          const int at = atomicAdd(&sb_count, 1);
+          if (at < NH) { head_b[at] = j; head_t[at] = sdst[j]; sdst[j] |= CP_FLAG; }
+        }
+      }
+      __syncthreads();
+      const int nb = min(sb_count, NH);   // (every thread reads the same count)
+      if (nb == 0) {
+        if (hashed) continue;
+        break;       // an unrestricted round found nothing: every entry is home
+      }
+      // ---- their entries into shared memory, before anything is overwritten
+      for (int i = warp; i < nb; i += CP_WARPS) {
+        const int b = head_b[i];
+        head_k[i * 32 + lane] = Ku[(size_t)b * 32 + lane];
+        head_v[i * 32 + lane] = Vu[(size_t)b * 32 + lane];
+        if (lane == 0) { head_a[i] = acc_u[b]; head_p[i] = pos_u[b]; }
+      }
+      __syncthreads();
+      // ---- the segments, first come first served
+      for (;;) {
+        int i = 0;
+        if (lane == 0) i = atomicAdd(&sb_next, 1);
+        i = __shfl_sync(0xffffffffu, i, 0);
+        if (i >= nb) break;
+        walk(head_t[i], head_k[i * 32 + lane], head_v[i * 32 + lane], head_a[i], head_p[i]);
+      }
+      __syncthreads();
     }
-    __syncthreads();
-    // ---- the segments, first come first served
-    for (;;) {
-      int i = 0;
-      if (lane == 0) i = atomicAdd(&sb_next, 1);
-      i = __shfl_sync(0xffffffffu, i, 0);
-      if (i >= nb) break;
-      walk(head_t[i], head_k[i * 32 + lane], head_v[i * 32 + lane], head_a[i], head_p[i]);
-    }
-    __syncthreads();
   }
   if (place) {
     int32_t* place_u = place + (size_t)u * k;

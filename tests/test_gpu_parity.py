@@ -193,6 +193,50 @@ def test_new_positions_differ_from_original_positions_and_survive_import():
         lockstep.check_guards(g)
 
 
+@pytest.mark.parametrize("d,k,order", [(128, 700, "random"), (64, 300, "reverse"), (256, 200, "random"), (128, 700, "rotate"),
+                                       (128, 2048, "arrivals"), (256, 333, "arrivals"), (64, 1000, "many arrivals")])
+def test_compaction_of_arbitrary_slot_orders(d, k, order):
+    """kf_compact_layer has two ways through: entries that only move down plus a few that move up (what generation
+    steps leave: `rotate`, `arrivals`) are carried over in ascending chunks; anything else (`random`, `reverse`, more
+    arrivals than the kernel sets aside) is applied cycle by cycle.  The slots of a freshly filled cache are put
+    into the given order here, through the library's own view of its state, and the call must sort them back."""
+    wl = W.Workload("compact_orders", 1, 2, 3, d, k + 60, k, k // 4, 4, data_seed=k + d, noise_seed=3)
+    gpu = lockstep.make_gpu(wl)
+    gpu.kf_prefill_score_prune(0, *W.make_prompt(wl, 0, DEV))
+    torch.cuda.synchronize()
+    K, V, pos, acc, ln = gpu.kf_view_state(0)
+    gen = torch.Generator(device="cpu").manual_seed(k)
+    U = wl.batch * wl.n_heads
+    if order in ("arrivals", "many arrivals"):
+        # entries in scattered slots become tokens that arrived later: larger positions than everything else, in any order
+        m = 40 if order == "arrivals" else 150
+        for u in range(U):
+            b, h = divmod(u, wl.n_heads)
+            sel = torch.randperm(k, generator=gen)[:m].to(DEV)
+            pos[b, h, sel] = (int(pos[b, h].max()) + 1 + torch.randperm(m, generator=gen)).to(device=DEV, dtype=torch.int32)
+    else:
+        if order == "random":
+            perm = torch.stack([torch.randperm(k, generator=gen) for _ in range(U)])
+        elif order == "reverse":
+            perm = torch.arange(k - 1, -1, -1).expand(U, k)
+        else:
+            perm = torch.arange(k).roll(-1).expand(U, k)                 # the first entry sits in the last slot
+        perm = perm.reshape(wl.batch, wl.n_heads, k).to(DEV)
+        rows = perm[..., None].expand(-1, -1, -1, d)
+        K.copy_(K.gather(2, rows)); V.copy_(V.gather(2, rows)); pos.copy_(pos.gather(-1, perm)); acc.copy_(acc.gather(-1, perm))
+    torch.cuda.synchronize()
+    before = [t.clone() for t in (K, V, pos, acc, ln)]
+    gpu.kf_compact_layer(0)
+    assert gpu.kf_poll_error() == 0
+    srt = before[2].argsort(-1)
+    rows = srt[..., None].expand(-1, -1, -1, d)
+    assert torch.equal(pos, before[2].gather(-1, srt)) and torch.equal(acc, before[3].gather(-1, srt))
+    assert torch.equal(K, before[0].gather(2, rows)) and torch.equal(V, before[1].gather(2, rows))
+    assert torch.equal(ln, before[4])
+    lockstep.check_guards(gpu)
+    gpu.kf_destroy()
+
+
 @pytest.mark.parametrize("d,pos_mode", [(64, 0), (128, 1), (256, 0)])
 def test_compaction_restores_position_order_in_place(d, pos_mode):
     """After enough steps the slots of a unit are a permutation of the position order.  kf_compact_layer must apply
