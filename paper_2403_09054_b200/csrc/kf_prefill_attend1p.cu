@@ -99,33 +99,45 @@ __device__ __forceinline__ float a1_tile_max(uint32_t s_addr, float A, float sb,
 // unrounded values) in `lsum`.  MASK = false is the common case (a tile wholly below the diagonal): it also returns
 // the row's largest x2, so that the caller can tell afterwards whether m_ref was still a valid reference.  MASK =
 // true applies the causal mask of the diagonal tile when `diag` is set (and returns nothing of use).
+#define A1_R32(r) "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),        \
+                  "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),        \
+                  "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),      \
+                  "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+// 32 lanes x 32 columns of tensor memory into r[0..32) WITHOUT waiting: the registers hold the values only after
+// a1_ld_wait(r), which also ties their later uses to the wait for the compiler.
+__device__ __forceinline__ void a1_ld_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void a1_ld_wait(uint32_t (&r)[32]) { asm volatile("tcgen05.wait::ld.sync.aligned;" : A1_R32(r)::"memory"); }
+
 template <bool ALIBI, bool MASK>
 __device__ __forceinline__ float a1_tile_probs(uint32_t s_addr, float A, float m_ref, float sb, float bias_t, int lane, int quarter,
                                                bool diag, uint32_t (&packed)[64], float& lsum) {
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    if (MASK && diag && c > quarter) {
-#pragma unroll
-      for (int e = 0; e < 16; ++e) packed[c * 16 + e] = 0u;
-      continue;
-    }
-    float v[32];
-    tmem_ld_32x32(s_addr + (uint32_t)(c * 32), v);
+  auto chunk = [&](const uint32_t (&r)[32], int c) {
     const bool edge = MASK && diag && c == quarter;
     float bias0 = 0.f;
     if (ALIBI) bias0 = fmaf(sb, (float)(c * 32), bias_t);
 #pragma unroll
     for (int e = 0; e < 32; e += 2) {
+      const float v0 = __uint_as_float(r[e]), v1 = __uint_as_float(r[e + 1]);
       float y0, y1;
       if (ALIBI) {
-        const float x0 = fmaf(sb, (float)e, fmaf(v[e], A, bias0)), x1 = fmaf(sb, (float)(e + 1), fmaf(v[e + 1], A, bias0));
+        const float x0 = fmaf(sb, (float)e, fmaf(v0, A, bias0)), x1 = fmaf(sb, (float)(e + 1), fmaf(v1, A, bias0));
         if (!MASK) { if (e & 2) m1 = a1_max3(m1, x0, x1); else m0 = a1_max3(m0, x0, x1); }
         y0 = x0 - m_ref;
         y1 = x1 - m_ref;
       } else {
-        if (!MASK) { if (e & 2) m1 = a1_max3(m1, v[e], v[e + 1]); else m0 = a1_max3(m0, v[e], v[e + 1]); }
-        a1_fma2(y0, y1, v[e], v[e + 1], A, -m_ref);
+        if (!MASK) { if (e & 2) m1 = a1_max3(m1, v0, v1); else m0 = a1_max3(m0, v0, v1); }
+        a1_fma2(y0, y1, v0, v1, A, -m_ref);
       }
       float p0 = fast_exp2(y0), p1 = fast_exp2(y1);
       if (edge) { p0 = e <= lane ? p0 : 0.f; p1 = e + 1 <= lane ? p1 : 0.f; }
@@ -133,6 +145,35 @@ __device__ __forceinline__ float a1_tile_probs(uint32_t s_addr, float A, float m
       const __half2 h = __floats2half2_rn(p0, p1);
       packed[c * 16 + (e >> 1)] = *reinterpret_cast<const uint32_t*>(&h);
     }
+  };
+  if (MASK) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      if (diag && c > quarter) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) packed[c * 16 + e] = 0u;
+        continue;
+      }
+      uint32_t r[32];
+      a1_ld_issue(s_addr + (uint32_t)(c * 32), r);
+      a1_ld_wait(r);
+      chunk(r, c);
+    }
+  } else {
+    // the logits of the next 32 columns are on their way while the current ones are worked on
+    uint32_t ra[32], rb[32];
+    a1_ld_issue(s_addr, ra);
+    a1_ld_wait(ra);
+    a1_ld_issue(s_addr + 32u, rb);
+    chunk(ra, 0);
+    a1_ld_wait(rb);
+    a1_ld_issue(s_addr + 64u, ra);
+    chunk(rb, 1);
+    a1_ld_wait(ra);
+    a1_ld_issue(s_addr + 96u, rb);
+    chunk(ra, 2);
+    a1_ld_wait(rb);
+    chunk(rb, 3);
   }
   lsum = l0 + l1;
   const float m = fmaxf(m0, m1);
