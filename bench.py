@@ -202,7 +202,7 @@ def run_reference(args, wl):
     """The slow CPU oracle as the reference arm (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    units, steps_inner = 64, 4
+    units, steps_inner = 256, 32      # one timed step of this arm: about 0.4 s of oracle work on 16 cores
     for _ in range(max(args.warmup, 1)):
         oracle_sample_rate(wl, 8, 1)
     rates, threads, desc = [], 1, ""
@@ -664,8 +664,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4_cerebras")
     ap.add_argument("--splits", type=int, default=0)
-    ap.add_argument("--cpu-units", type=int, default=512)
-    ap.add_argument("--cpu-steps", type=int, default=64)
+    ap.add_argument("--cpu-units", type=int, default=1024, help="units of the sample the CPU oracle is timed on (cpu_baseline)")
+    ap.add_argument("--cpu-steps", type=int, default=256, help="generation steps of that sample (1024 x 256 is about 12 s on 16 cores)")
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per layer call from an ncu capture (default: the stored capture of exactly the "
                          "kernel variant and shape that is launched, else null)")
