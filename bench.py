@@ -409,6 +409,9 @@ def run_ours(args, wl):
             if wl.name == "c4_cerebras":
                 line["other_workloads"].append(gqa_point(dev))
             line["prefill"] = prefill_point(W.get_config("c5_prefill_8k"), dev, budget_frac=0.5, steps=5, warmup=3)
+            both = prefill_point(W.get_config("c5_prefill_8k"), dev, budget_frac=0.5, steps=5, warmup=3, with_attention=True)
+            line["prefill"]["with_attention_output_ms_per_call"] = both["ms_per_call"]
+            line["prefill"]["attention_output_alone"] = attention_point(W.get_config("c5_prefill_8k"), dev, steps=10, warmup=3)
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
