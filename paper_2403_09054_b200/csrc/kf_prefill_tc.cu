@@ -45,7 +45,8 @@ constexpr int tc_threads(int ng) { return (2 + 4 * ng) * 32; }   // TMA warp + M
 constexpr int TC_NG = KF_TC_NG;               // compute groups for head_dim 64 / 128 (256 leaves room for 2)
 constexpr int TC_NACC = 4;                    // accumulator buffers: 4 x 128 columns = all of tensor memory
 constexpr uint32_t TC_TMEM_COLS = 512;
-constexpr int TC_XBUF_FLOATS = 4 * 32 * 4;    // per warp: 4 noise calls x 32 lanes x 4 words
+constexpr int TC_XBUF_FLOATS = 4 * 32 * 4;    // per warp and buffer: 4 noise calls x 32 lanes x 4 words
+__host__ __device__ constexpr int tc_xbufs(int d) { return d == 256 ? 1 : 2; }   // buffers per warp (two where shared memory allows)
 __host__ __device__ constexpr int tc_comb_buffers(int d) { return d == 256 ? 2 : 4; }   // what the shared memory left over allows
 constexpr float LG2_LN2 = -0.5287663729448977f;  // log2(ln 2)
 
@@ -110,7 +111,8 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
   unsigned char* sS = smem + OP_BYTES;                       // NST stages of the streamed operand
   constexpr int NCW = 4 * NG;                                // compute warps
   float* xbuf = reinterpret_cast<float*>(sS + (size_t)NST * OP_BYTES);  // [NCW][TC_XBUF_FLOATS] noise exchange
-  float* lse_s = xbuf + NCW * TC_XBUF_FLOATS;                // [NCW][128] lse2 of the current query tile
+  constexpr int XB = tc_xbufs(D);
+  float* lse_s = xbuf + NCW * XB * TC_XBUF_FLOATS;           // [NCW][128] lse2 of the current query tile
   constexpr int COMB_FLOATS = NG * 4 * 128;
   constexpr int NCB = tc_comb_buffers(D);                    // items whose hand-over may be pending at one time
   float* comb = lse_s + NCW * 128;                           // [NCB][NG][4][128] hand-over between the compute groups
@@ -249,7 +251,7 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
     const float A = P.a_scale;
     const float n_mult = NOISE == NOISE_GAUSS_T ? P.gauss_scale : -P.inv_tau;
     const float n_off = NOISE == NOISE_GUMBEL_T ? -P.inv_tau * LG2_LN2 : P.const_term;   // additive term common to all logits
-    float* my_x = xbuf + cw * TC_XBUF_FLOATS;
+    float* my_x0 = xbuf + cw * XB * TC_XBUF_FLOATS;
     float* my_lse = lse_s + cw * 128;
     bool ok = true;
 
@@ -412,8 +414,11 @@ __global__ void __launch_bounds__(tc_threads(NG), 1) prefill_tc(const __grid_con
             for (int half = 0; half < 2; ++half) {
               // Lane L draws the Philox call of key group (L & 7) of this warp and query 4 g + (L >> 3) and
               // folds that query's -lse2 into the four terms; afterwards lane L reads word (L & 3) of its
-              // own key group (L >> 2) for each query.  Both access patterns are bank-conflict free.
-              __syncwarp();
+              // own key group (L >> 2) for each query.  Both access patterns are bank-conflict free.  With two
+              // buffers the halves alternate, and the barrier after a half's writes is also what tells that the
+              // buffer written next (read one half earlier) is free.
+              float* my_x = my_x0 + (XB == 2 ? half * TC_XBUF_FLOATS : 0);
+              if (XB == 1) __syncwarp();
 #pragma unroll
               for (int g = 0; g < 4; ++g) {
                 const int ql = half * 16 + 4 * g + (lane >> 3);
@@ -576,7 +581,7 @@ namespace {
 
 template <int D, int NST, int NG>
 constexpr size_t tc_smem_bytes() {
-  size_t b = 1024 + (size_t)(1 + NST) * TC_BM * D * 2 + (size_t)4 * NG * TC_XBUF_FLOATS * 4 + (size_t)4 * NG * 128 * 4 +
+  size_t b = 1024 + (size_t)(1 + NST) * TC_BM * D * 2 + (size_t)4 * NG * tc_xbufs(D) * TC_XBUF_FLOATS * 4 + (size_t)4 * NG * 128 * 4 +
              (size_t)tc_comb_buffers(D) * NG * 4 * 128 * 4 + 40 * 8 + 64;
   return b < 120 * 1024 ? 120 * 1024 : b;   // one CTA per SM: each takes all of tensor memory
 }
