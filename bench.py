@@ -448,9 +448,9 @@ PREFILL_INT_INSTR, PREFILL_FP_INSTR, PREFILL_MUFU_INSTR = 13, 7, 3
 # dram__bytes_read.sum + dram__bytes_write.sum of the two prefill_tc launches of one call on c5_prefill_2k (B8 H32 d128,
 # n 2048: Q + K = 268 MB, each read from DRAM once per sweep), from an ncu capture.  It does not scale with the logit
 # count (re-reads are served by L2), so the other prompt lengths report no traffic figure.
-C5_2K_PREFILL_TRAFFIC_BYTES = (268.5 + 4.8 + 270.6 + 5.4) * 1e6
+C5_2K_PREFILL_TRAFFIC_BYTES = (268.6 + 8.2 + 270.9 + 5.8) * 1e6
 # sm__pipe_tensor_cycles_active / XU pipe / issue-active of the two sweeps in that capture (n = 2048), in percent
-C5_2K_PREFILL_COUNTERS = {"captured_at": "n = 2048", "tensor_pipe_pct": [8, 10], "xu_pipe_pct": [46, 56], "issue_active_pct": [57, 61]}
+C5_2K_PREFILL_COUNTERS = {"captured_at": "n = 2048", "tensor_pipe_pct": [8.4, 9.6], "xu_pipe_pct": [48, 56], "issue_active_pct": [56, 61]}
 PREFILL_LANE_INSTR_PER_LOGIT_SWEEP = 2 * PREFILL_INT_INSTR + PREFILL_FP_INSTR + PREFILL_MUFU_INSTR   # 36 FP32-lane slots
 ALU_LANES_PER_SM, N_SM = 128, 148
 
