@@ -32,9 +32,16 @@ template <> struct RowPart<64> { using type = uint32_t; };
 template <> struct RowPart<128> { using type = uint2; };
 template <> struct RowPart<256> { using type = uint4; };
 
-// dst[j] = number of the unit's positions smaller than pos[j] (positions of a unit are distinct): the positions are
-// sorted in shared memory (bitonic network, padded to a power of two with the largest value) and every entry finds
-// its own position in the sorted array by bisection.
+constexpr int CP_FAST_N = 4096;    // entries up to which the nearly-sorted shortcut of the rank kernel has its shared memory
+constexpr int CP_FAST_OUT = 128;   // out-of-order entries it handles
+
+// dst[j] = number of the unit's positions smaller than pos[j] (positions of a unit are distinct).
+// Shortcut for what generation steps leave behind: call an entry "in order" if every later slot holds a larger
+// position (a suffix minimum tells).  The in-order entries form an ascending run; if the others are few (the tokens
+// that arrived since the last compaction) every rank is a prefix count within the run plus a handful of comparisons
+// with the others, and the others find their place in the run by bisection.  Otherwise: the positions are sorted in
+// shared memory (bitonic network, padded to a power of two with the largest value) and every entry finds its own
+// position in the sorted array by bisection.
 __global__ void __launch_bounds__(CP_THREADS) compact_rank_kernel(const int32_t* __restrict__ pos, const int32_t* __restrict__ len,
                                                                   int32_t* __restrict__ dst, int k, int n_pow2) {
   extern __shared__ __align__(16) int32_t cp_smem[];
@@ -42,6 +49,73 @@ __global__ void __launch_bounds__(CP_THREADS) compact_rank_kernel(const int32_t*
   const int u = blockIdx.x, tid = threadIdx.x;
   const int n = min(len[u], k);
   const int32_t* pos_u = pos + (size_t)u * k;
+  if (n <= CP_FAST_N && n > 0) {
+    __shared__ int32_t red[CP_THREADS];
+    __shared__ int32_t opos[CP_FAST_OUT], oidx[CP_FAST_OUT];
+    __shared__ int s_out;
+    int32_t* run = key + n;          // positions of the in-order entries, ascending
+    int32_t* code = run + n;         // per slot: index within the run, or -1
+    const int per = (n + CP_THREADS - 1) / CP_THREADS;
+    const int lo = min(n, tid * per), hi = min(n, lo + per);
+    for (int j = tid; j < n; j += CP_THREADS) key[j] = pos_u[j];
+    if (tid == 0) s_out = 0;
+    __syncthreads();
+    int mn = 0x7fffffff;
+    for (int j = lo; j < hi; ++j) mn = min(mn, key[j]);
+    red[tid] = mn;
+    __syncthreads();
+    // smallest position in the slots behind this thread's range; how many in-order entries this range holds
+    int behind = 0x7fffffff;
+    for (int t = tid + 1; t < CP_THREADS; ++t) behind = min(behind, red[t]);
+    int running = behind, mine = 0;
+    for (int j = hi - 1; j >= lo; --j) {
+      const int pj = key[j];
+      const bool in_order = pj < running;
+      code[j] = in_order ? 0 : -1;
+      mine += in_order ? 1 : 0;
+      running = min(running, pj);
+    }
+    __syncthreads();                 // everybody has read red[]
+    red[tid] = mine;
+    __syncthreads();
+    int base = 0;
+    for (int t = 0; t < tid; ++t) base += red[t];
+    for (int j = lo; j < hi; ++j) {
+      if (code[j] == 0) {
+        code[j] = base;
+        run[base++] = key[j];
+      } else {
+        const int at = atomicAdd(&s_out, 1);
+        if (at < CP_FAST_OUT) { opos[at] = key[j]; oidx[at] = j; }
+      }
+    }
+    __syncthreads();
+    const int m = s_out, n_run = n - m;
+    if (m <= CP_FAST_OUT) {          // (every thread reads the same count)
+      for (int j = tid; j < n; j += CP_THREADS) {
+        const int cj = code[j];
+        if (cj >= 0) {
+          const int pj = key[j];
+          int below = 0;
+          for (int o = 0; o < m; ++o) below += opos[o] < pj ? 1 : 0;
+          dst[(size_t)u * k + j] = cj + below;
+        }
+      }
+      for (int o = tid; o < m; o += CP_THREADS) {
+        const int p = opos[o];
+        int a = 0, b = n_run;        // first index of the run whose position is not below p
+        while (a < b) {
+          const int mid = (a + b) >> 1;
+          if (run[mid] < p) a = mid + 1; else b = mid;
+        }
+        int below = 0;
+        for (int o2 = 0; o2 < m; ++o2) below += opos[o2] < p ? 1 : 0;
+        dst[(size_t)u * k + oidx[o]] = a + below;
+      }
+      return;
+    }
+    __syncthreads();                 // too many entries out of order: the general way, from the start
+  }
   int np = 1;
   while (np < n) np <<= 1;          // the network only has to cover this unit's entries (np <= n_pow2)
   for (int j = tid; j < np; j += CP_THREADS) key[j] = j < n ? pos_u[j] : 0x7fffffff;
@@ -275,9 +349,10 @@ cudaError_t launch_compact(__half* K, __half* V, float* acc, int32_t* pos, const
   if (k < 1 || k > CP_MAX_K || units < 1 || !dst_scratch) return cudaErrorInvalidValue;
   int n_pow2 = 1;
   while (n_pow2 < k) n_pow2 <<= 1;
-  const size_t smem_rank = (size_t)n_pow2 * 4;
+  const size_t smem_rank = std::max((size_t)n_pow2 * 4, (size_t)3 * std::min(k, CP_FAST_N) * 4);   // the sort, or the shortcut's three arrays
   cudaError_t e = cudaSuccess;
-  if (smem_rank > 48 * 1024) e = cudaFuncSetAttribute(compact_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_rank);
+  // (the kernel also has 2 KB of static shared memory: ask as soon as the sum could pass the 48 KB every kernel may have)
+  if (smem_rank > 40 * 1024) e = cudaFuncSetAttribute(compact_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_rank);
   if (e != cudaSuccess) return e;
   compact_rank_kernel<<<units, CP_THREADS, smem_rank, stream>>>(pos, len, dst_scratch, k, n_pow2);
   e = cudaGetLastError();

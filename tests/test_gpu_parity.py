@@ -194,7 +194,8 @@ def test_new_positions_differ_from_original_positions_and_survive_import():
 
 
 @pytest.mark.parametrize("d,k,order", [(128, 700, "random"), (64, 300, "reverse"), (256, 200, "random"), (128, 700, "rotate"),
-                                       (128, 2048, "arrivals"), (256, 333, "arrivals"), (64, 1000, "many arrivals")])
+                                       (128, 2048, "arrivals"), (256, 333, "arrivals"), (64, 1000, "many arrivals"),
+                                       (128, 4096, "arrivals"), (64, 5000, "arrivals")])
 def test_compaction_of_arbitrary_slot_orders(d, k, order):
     """kf_compact_layer has two ways through: entries that only move down plus a few that move up (what generation
     steps leave: `rotate`, `arrivals`) are carried over in ascending chunks; anything else (`random`, `reverse`, more
